@@ -1,0 +1,250 @@
+"""Pins for the CPU oracle: what the paper prints and what the mathematics fixes.
+
+Each test is chosen so that one plausible mistake in oracle/wht_oracle.py (another
+ordering of the transform, a missing or doubled 1/sqrt(d), a dropped bias, x used
+where z belongs in da, a wrong sign in a butterfly) makes it fail.
+"""
+import itertools
+import math
+import os
+
+import numpy as np
+import pytest
+import scipy.linalg
+
+import oracle
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _golden_lines(name):
+    with open(os.path.join(GOLDEN, name)) as f:
+        return [ln.strip() for ln in f if ln.strip() and not ln.startswith("#")]
+
+
+# ---------------------------------------------------------------- ordering
+
+def test_h4_matches_printed_sign_pattern():
+    # Fig. 1 prints H_4; sequency (Walsh) or dyadic (Paley) order would permute rows 1..3.
+    rows = _golden_lines("h4_sign_pattern.txt")
+    printed = np.array([[1.0 if c == "+" else -1.0 for c in r] for r in rows])
+    assert printed.shape == (4, 4)
+    np.testing.assert_array_equal(oracle.sylvester_hadamard(4), printed)
+
+
+@pytest.mark.parametrize("d", [1, 2, 4, 8, 16, 64, 256, 1024])
+def test_matches_kronecker_recursion_and_scipy(d):
+    # Sylvester's construction H_2n = [[H, H], [H, -H]] is a second, independent
+    # definition; scipy.linalg.hadamard implements it as a library routine.
+    H = oracle.sylvester_hadamard(d)
+    K = np.array([[1.0]])
+    while K.shape[0] < d:
+        K = np.block([[K, K], [K, -K]])
+    np.testing.assert_array_equal(H, K)
+    np.testing.assert_array_equal(H, scipy.linalg.hadamard(d).astype(np.float64))
+
+
+@pytest.mark.parametrize("d", [2, 8, 64, 512, 1024])
+def test_h_ht_is_d_identity_in_integers(d):
+    # Eq. 1's condition H^T H = I for the normalised matrix <=> H H^T = d I unnormalised.
+    H = oracle.sylvester_hadamard(d).astype(np.int64)
+    np.testing.assert_array_equal(H @ H.T, d * np.eye(d, dtype=np.int64))
+    np.testing.assert_array_equal(H, H.T)
+
+
+def test_d_must_be_power_of_two():
+    for bad in (0, 3, 12, 768):
+        with pytest.raises(ValueError):
+            oracle.sylvester_hadamard(bad)
+
+
+# ---------------------------------------------------------------- normalisation
+
+@pytest.mark.parametrize("d", [2, 16, 256, 2048])
+def test_norm_preserved_and_involution(d):
+    rng = np.random.default_rng(d)
+    x = rng.standard_normal((5, d))
+    z = oracle.wht_normalised(x)
+    np.testing.assert_allclose(np.linalg.norm(z, axis=1), np.linalg.norm(x, axis=1), rtol=1e-13)
+    # the normalised transform is its own inverse: H(Hx) = d x
+    np.testing.assert_allclose(oracle.wht_normalised(z), x, rtol=0, atol=1e-12)
+    ones = np.ones(d)
+    zero = np.zeros(d)
+    np.testing.assert_allclose(oracle.wht_affine_fwd(z, ones, zero), x, rtol=0, atol=1e-12)
+
+
+@pytest.mark.parametrize("d", [4, 32, 1024])
+def test_constant_and_impulse_rows(d):
+    rng = np.random.default_rng(7 + d)
+    a = rng.uniform(0.5, 1.5, d)
+    b = rng.normal(0, 0.1, d)
+    # H . 1 = d e_0  =>  y = a_0 sqrt(d) e_0 + b
+    y = oracle.wht_affine_fwd(np.ones((1, d)), a, b)[0]
+    expect = b.copy()
+    expect[0] += a[0] * math.sqrt(d)
+    np.testing.assert_allclose(y, expect, rtol=0, atol=1e-12)
+    # x = e_k  =>  y = a (.) (row k of H)/sqrt(d) + b, signs from popcount parity
+    for k in (0, 1, d // 2, d - 1):
+        e = np.zeros((1, d))
+        e[0, k] = 1.0
+        signs = np.array([(-1.0) ** bin(k & j).count("1") for j in range(d)])
+        np.testing.assert_allclose(oracle.wht_affine_fwd(e, a, b)[0],
+                                   a * signs / math.sqrt(d) + b, rtol=0, atol=1e-14)
+    # x = 0  =>  y = b
+    np.testing.assert_array_equal(oracle.wht_affine_fwd(np.zeros((2, d)), a, b),
+                                  np.broadcast_to(b, (2, d)))
+
+
+# ---------------------------------------------------------------- brute force
+
+@pytest.mark.parametrize("d", [2, 4, 8, 16])
+def test_brute_force_small(d):
+    # pure-Python triple loop from the recursive sign rule, exact rationals for the sum
+    def sign(i, j, n):
+        # entry (i, j) of H_n via the quadrant rule of Sylvester's construction
+        s = 1
+        while n > 1:
+            n //= 2
+            if i >= n and j >= n:
+                s = -s
+            i %= n
+            j %= n
+        return s
+
+    rng = np.random.default_rng(100 + d)
+    x = rng.integers(-4, 5, size=(3, d)).astype(np.float64)
+    a = rng.integers(1, 4, size=d).astype(np.float64)
+    b = rng.integers(-2, 3, size=d).astype(np.float64)
+    y = oracle.wht_affine_fwd(x, a, b)
+    for t, j in itertools.product(range(3), range(d)):
+        acc = 0
+        for i in range(d):
+            acc += int(x[t, i]) * sign(i, j, d)
+        assert y[t, j] == pytest.approx(a[j] * acc / math.sqrt(d) + b[j], abs=1e-13)
+
+
+# ---------------------------------------------------------------- Fig. 2 butterfly
+
+def test_butterfly_pairs_of_figure():
+    # the stage wiring printed in Fig. 2 for d = 8 is what fwht_butterfly walks
+    for line in _golden_lines("butterfly_pairs_d8.txt"):
+        parts = line.split()
+        stride = int(parts[0])
+        pairs = {tuple(int(p) - 1 for p in s.split("-")) for s in parts[1:]}
+        walked = {(i, i + stride) for i in range(8) if not i & stride}
+        assert pairs == walked
+
+
+@pytest.mark.parametrize("d", [2, 8, 64, 256, 1024, 4096])
+def test_butterfly_equals_matrix_and_op_count(d):
+    rng = np.random.default_rng(d + 1)
+    v = rng.standard_normal(d)
+    got, ops = oracle.fwht_butterfly(v)
+    want = v @ oracle.sylvester_hadamard(d)
+    np.testing.assert_allclose(got, want, rtol=0, atol=1e-9 * math.sqrt(d))
+    assert ops == d * int(math.log2(d))
+
+
+def test_butterfly_op_counts_match_figure():
+    for line in _golden_lines("fwht_op_counts.txt"):
+        d, count = (int(s) for s in line.split())
+        _, ops = oracle.fwht_butterfly(np.zeros(d))
+        assert ops == count
+
+
+# ---------------------------------------------------------------- gradients
+
+def _loss(x, a, b, dy):
+    return float(np.sum(dy * oracle.wht_affine_fwd(x, a, b)))
+
+
+@pytest.mark.parametrize("T,d", [(3, 8), (5, 64), (4, 256)])
+def test_gradients_by_central_differences(T, d):
+    rng = np.random.default_rng(T * 1000 + d)
+    x = rng.standard_normal((T, d))
+    dy = rng.standard_normal((T, d))
+    a = rng.uniform(0.5, 1.5, d)
+    b = rng.normal(0, 0.1, d)
+    dx, da, db = oracle.wht_affine_bwd(dy, x, a)
+    h = 1e-3  # the loss is linear in each of x, a, b alone, so the difference is exact up to rounding
+    cols = sorted(set([0, 1, d // 2, d - 1]) | set(rng.integers(0, d, 4).tolist()))
+    for j in cols:
+        ap, am = a.copy(), a.copy()
+        ap[j] += h
+        am[j] -= h
+        assert (_loss(x, ap, b, dy) - _loss(x, am, b, dy)) / (2 * h) == pytest.approx(da[j], rel=1e-8, abs=1e-8)
+        bp, bm = b.copy(), b.copy()
+        bp[j] += h
+        bm[j] -= h
+        assert (_loss(x, a, bp, dy) - _loss(x, a, bm, dy)) / (2 * h) == pytest.approx(db[j], rel=1e-8, abs=1e-8)
+    for t, i in [(0, 0), (T - 1, d - 1), (1, d // 2), (T // 2, 1)]:
+        xp, xm = x.copy(), x.copy()
+        xp[t, i] += h
+        xm[t, i] -= h
+        assert (_loss(xp, a, b, dy) - _loss(xm, a, b, dy)) / (2 * h) == pytest.approx(dx[t, i], rel=1e-8, abs=1e-8)
+
+
+@pytest.mark.parametrize("d", [16, 512])
+def test_adjoint_identity_and_db_column_sums(d):
+    rng = np.random.default_rng(d * 3)
+    T = 6
+    x = rng.standard_normal((T, d))
+    dy = rng.standard_normal((T, d))
+    a = rng.uniform(0.5, 1.5, d)
+    b = rng.normal(0, 0.1, d)
+    dx, da, db = oracle.wht_affine_bwd(dy, x, a)
+    y = oracle.wht_affine_fwd(x, a, b)
+    # <dy, y - b> = <dx, x>  (the map x -> y - b is linear with adjoint dy -> dx)
+    assert np.sum(dy * (y - b)) == pytest.approx(np.sum(dx * x), rel=1e-12)
+    # <dy, y - b> = <da, a> as well, since y - b = a (.) z
+    assert np.sum(dy * (y - b)) == pytest.approx(np.sum(da * a), rel=1e-12)
+    col = np.zeros(d)
+    for t in range(T):
+        col += dy[t]
+    np.testing.assert_allclose(db, col, rtol=0, atol=1e-13)
+
+
+def test_da_db_columns_agrees_with_full():
+    rng = np.random.default_rng(11)
+    T, d = 37, 128
+    x = rng.standard_normal((T, d)).astype(np.float32)
+    dy = rng.standard_normal((T, d)).astype(np.float32)
+    a = rng.uniform(0.5, 1.5, d)
+    _, da, db = oracle.wht_affine_bwd(dy, x, a)
+    cols = np.array([0, 5, 64, 127])
+    da_c, db_c = oracle.da_db_columns(dy, x, cols)
+    np.testing.assert_allclose(da_c, da[cols], rtol=1e-12)
+    np.testing.assert_allclose(db_c, db[cols], rtol=1e-12, atol=1e-13)
+
+
+def test_widen_bf16_bits_exact():
+    # 0x3F80 = 1.0, 0xC000 = -2.0, 0x3DCD ~ 0.100098 (bf16 nearest to 0.1), 0x0000 = 0
+    bits = np.array([0x3F80, 0xC000, 0x3DCD, 0x0000, 0x7F7F], dtype=np.uint16)
+    got = oracle.widen_bf16_bits(bits)
+    want = np.array([1.0, -2.0, 0.10009765625, 0.0, 3.3895313892515355e38])
+    np.testing.assert_array_equal(got, want)
+
+
+# ---------------------------------------------------------------- planted mistakes are caught
+
+def test_pins_catch_planted_mistakes(monkeypatch):
+    # A wrong ordering (sequency order) still satisfies H H^T = d I, so the printed
+    # pattern is what must catch it; check that it would.
+    H = oracle.sylvester_hadamard(4)
+    sequency = H[[0, 2, 3, 1]]
+    rows = _golden_lines("h4_sign_pattern.txt")
+    printed = np.array([[1.0 if c == "+" else -1.0 for c in r] for r in rows])
+    assert not np.array_equal(sequency, printed)
+    # da computed from x instead of z fails the finite-difference pin
+    rng = np.random.default_rng(5)
+    x = rng.standard_normal((3, 8))
+    dy = rng.standard_normal((3, 8))
+    a = rng.uniform(0.5, 1.5, 8)
+    b = np.zeros(8)
+    wrong_da = np.sum(dy * x, axis=0)
+    h = 1e-3
+    ap, am = a.copy(), a.copy()
+    ap[3] += h
+    am[3] -= h
+    fd = (_loss(x, ap, b, dy) - _loss(x, am, b, dy)) / (2 * h)
+    assert abs(fd - wrong_da[3]) > 1e-3
