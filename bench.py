@@ -1,0 +1,506 @@
+#!/usr/bin/env python
+"""Benchmark of the WHT + diagonal-affine path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload training|prefill|large|tiny]
+                    [--impl ours|reference] [--no-sections]
+
+A step is one pass of the whole path over one batch: the forward call
+(y = a (.) (x H)/sqrt(d) + b) followed by the backward call (dx, da, db).  The
+default workload is the training shape (65536 rows, d = 2048, bf16 rows, fp32
+parameters), whose 1 GiB working set is far larger than L2, so no flush is needed
+between iterations.  Rank 0 prints ONE JSON line.  With N > 1 ranks every rank
+transforms its own rows (rows are independent; weak scaling) and the only exchange
+is one all-reduce of da|db per step.
+
+`--impl reference` times the fp64 CPU oracle (the parity authority, a deliberately
+slow dense product) on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from paper_2603_08343_b200 import workloads as wl
+
+METRIC = "wht_affine_tokens_per_s_fwd_bwd"
+UNIT = "tokens/s"
+
+
+# ----------------------------------------------------------------------------- helpers
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json, copy bandwidth)"
+    return 6650.0, "fallback (earlier measurement on this pool)"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index = gpu_index
+        self.proc = None
+        self.lines = []
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                 "-i", str(self.gpu_index), "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._pump, daemon=True)
+        self.thread.start()
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.time(), line.strip()))
+
+    def stop(self, t0=None, t1=None):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons, power = [], [], set(), []
+        for ts, line in self.lines:
+            if t0 is not None and not (t0 - 0.05 <= ts <= t1 + 0.15):
+                continue
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 9:
+                continue
+            try:
+                sm.append(float(parts[1]))
+                mx.append(float(parts[2]))
+                power.append(float(parts[3]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"),
+                                 parts[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {
+            "sm_mhz": statistics.median(sm) if sm else None,
+            "sm_max_mhz": max(mx) if mx else None,
+            "power_w_max": max(power) if power else None,
+            "samples": len(sm),
+            "reasons": sorted(reasons),
+        }
+
+
+def f64(t: torch.Tensor) -> np.ndarray:
+    import oracle
+    t = t.detach().cpu().contiguous()
+    if t.dtype == torch.bfloat16:
+        return oracle.widen_bf16_bits(t.view(torch.int16).numpy().view(np.uint16))
+    return t.numpy().astype(np.float64)
+
+
+def blas_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"]
+        if n:
+            return int(max(n))
+    except Exception:
+        pass
+    return os.cpu_count() or 1
+
+
+def oracle_step_seconds(w: wl.Workload, rows: int, repeats: int = 1):
+    """Times the oracle's forward (+ backward when the workload has one) on `rows` rows."""
+    import oracle
+    ws = w.with_rows(rows)
+    x = f64(wl.gen_full(ws, "x"))
+    a, b = (f64(t) for t in wl.gen_params(ws))
+    dy = f64(wl.gen_full(ws, "dy")) if w.has_bwd else None
+    oracle.sylvester_hadamard(w.d)  # the constant matrix is built outside the timed region
+    best = float("inf")
+    for _ in range(repeats):
+        t0 = time.perf_counter()
+        oracle.wht_affine_fwd(x, a, b)
+        if dy is not None:
+            oracle.wht_affine_bwd(dy, x, a)
+        best = min(best, time.perf_counter() - t0)
+    return best
+
+
+# ----------------------------------------------------------------------------- reference arm
+
+def run_reference(args, rank: int, world: int):
+    if rank != 0:
+        return
+    w = wl.CONFIGS[args.workload]
+    rows = {"tiny": 64, "prefill": 2048, "training": 1024, "large": 128}[args.workload]
+    for _ in range(args.warmup):
+        oracle_step_seconds(w, min(rows, 64))
+    times = [oracle_step_seconds(w, rows) for _ in range(args.steps)]
+    total = sum(times)
+    value = rows * args.steps / total
+    cores = blas_threads()
+    sample = f"{rows} rows of the {w.name} workload per step (d={w.d}), fp64 dense product, fwd{'+bwd' if w.has_bwd else ''}"
+    out = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic", "config": {"workload": w.name, "T_sample": rows, "d": w.d},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(out))
+
+
+# ----------------------------------------------------------------------------- our arm
+
+class Timer:
+    def __init__(self):
+        self.start = torch.cuda.Event(enable_timing=True)
+        self.end = torch.cuda.Event(enable_timing=True)
+
+    def __enter__(self):
+        self.start.record()
+        return self
+
+    def __exit__(self, *exc):
+        self.end.record()
+
+    def ms(self):
+        self.end.synchronize()
+        return self.start.elapsed_time(self.end)
+
+
+def time_loop(fn, iters: int, warmup: int = 3):
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    with Timer() as t:
+        for _ in range(iters):
+            fn()
+    return t.ms() / iters
+
+
+def section_prefill(B, hbm_peak):
+    """Prefill forward; 16 buffer pairs (1 GiB) are rotated so every call misses L2."""
+    w = wl.CONFIGS["prefill"]
+    a, b = (t.cuda() for t in wl.gen_params(w))
+    x0 = wl.gen_full(w, "x").cuda()
+    nbuf = 16
+    xs = [x0.clone() for _ in range(nbuf)]
+    ys = [torch.empty_like(x0) for _ in range(nbuf)]
+    state = {"i": 0}
+
+    def call():
+        i = state["i"] % nbuf
+        state["i"] += 1
+        B.wht_affine_fwd(xs[i], a, b, ys[i], w.T, w.d, w.dtype)
+
+    def copy():
+        i = state["i"] % nbuf
+        state["i"] += 1
+        B.wht_copy_rows(xs[i], ys[i], w.T, w.d, w.dtype)
+
+    ms = time_loop(call, 20 * nbuf, warmup=nbuf)
+    ms_copy = time_loop(copy, 20 * nbuf, warmup=nbuf)
+    warm = time_loop(lambda: B.wht_affine_fwd(xs[0], a, b, ys[0], w.T, w.d, w.dtype), 200, warmup=10)
+    gb = 2 * w.T * w.d * w.io_bytes / 1e9
+    return {"T": w.T, "d": w.d, "dtype": "bf16", "l2": "16 rotating buffer pairs (1 GiB)",
+            "fwd_us": 1e3 * ms, "fwd_tokens_per_s": w.T / (ms * 1e-3), "fwd_GBps": gb / (ms * 1e-3),
+            "fwd_frac_of_measured_peak": gb / (ms * 1e-3) / hbm_peak,
+            "fwd_frac_of_8000": gb / (ms * 1e-3) / 8000.0,
+            "copy_rows_GBps": gb / (ms_copy * 1e-3), "fwd_us_l2_warm": 1e3 * warm}
+
+
+def section_decode(B):
+    w0 = wl.CONFIGS["decode"]
+    a, b = (t.cuda() for t in wl.gen_params(w0))
+    out = {}
+    for T in wl.DECODE_T:
+        w = w0.with_rows(T)
+        x = wl.gen_full(w, "x").cuda()
+        y = torch.empty_like(x)
+        fn = lambda: B.wht_affine_fwd_decode(x, a, b, y, w.T, w.d, w.dtype)  # noqa: E731
+        loop_us = 1e3 * time_loop(fn, 2000, warmup=20)
+        # CUDA-graph replay of 50 back-to-back calls: per-call device time without launch overhead
+        s = torch.cuda.Stream()
+        with torch.cuda.stream(s):
+            for _ in range(3):
+                B.wht_affine_fwd_decode(x, a, b, y, w.T, w.d, w.dtype)
+            torch.cuda.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=s):
+                for _ in range(50):
+                    B.wht_affine_fwd_decode(x, a, b, y, w.T, w.d, w.dtype)
+            graph_us = 1e3 * time_loop(g.replay, 40, warmup=3) / 50
+        out[f"T{T}"] = {"stream_loop_us_per_call": loop_us, "graph_replay_us_per_call": graph_us}
+    out["d"] = w0.d
+    return out
+
+
+def section_fwd_bwd(B, name, hbm_peak, iters):
+    """Forward and backward timed separately on a workload larger than L2."""
+    w = wl.CONFIGS[name]
+    base_rows = min(w.T, 8192)
+    a, b = (t.cuda() for t in wl.gen_params(w))
+    xb = wl.gen_full(w.with_rows(base_rows), "x").cuda()
+    dyb = wl.gen_full(w.with_rows(base_rows), "dy").cuda()
+    reps = w.T // base_rows
+    x = xb.repeat(reps, 1)
+    dy = dyb.repeat(reps, 1)
+    del xb, dyb
+    y = torch.empty_like(x)
+    da = torch.empty(w.d, dtype=torch.float32, device="cuda")
+    db = torch.empty_like(da)
+    f_ms = time_loop(lambda: B.wht_affine_fwd(x, a, b, y, w.T, w.d, w.dtype), iters)
+    b_ms = time_loop(lambda: B.wht_affine_bwd(dy, x, a, y, da, db, w.T, w.d, w.dtype), iters)
+    c_ms = time_loop(lambda: B.wht_copy_rows(x, y, w.T, w.d, w.dtype), iters)
+    fb = 2 * w.T * w.d * w.io_bytes / 1e9
+    bb = 3 * w.T * w.d * w.io_bytes / 1e9
+    res = {"T": w.T, "d": w.d, "rows_drawn": base_rows, "rows_tiled": reps,
+           "fwd_us": 1e3 * f_ms, "fwd_GBps": fb / (f_ms * 1e-3), "fwd_frac_of_measured_peak": fb / (f_ms * 1e-3) / hbm_peak,
+           "fwd_frac_of_8000": fb / (f_ms * 1e-3) / 8000.0, "fwd_tokens_per_s": w.T / (f_ms * 1e-3),
+           "bwd_us": 1e3 * b_ms, "bwd_GBps": bb / (b_ms * 1e-3), "bwd_frac_of_measured_peak": bb / (b_ms * 1e-3) / hbm_peak,
+           "bwd_frac_of_8000": bb / (b_ms * 1e-3) / 8000.0, "bwd_tokens_per_s": w.T / (b_ms * 1e-3),
+           "copy_rows_GBps": fb / (c_ms * 1e-3)}
+    # the dense projection this path replaces, as context: cuBLAS bf16 [T x d] x [d x d]
+    if w.dtype != wl.WHT_F32:
+        wmat = torch.randn(w.d, w.d, device="cuda", dtype=torch.bfloat16)
+        g_ms = time_loop(lambda: torch.matmul(x, wmat, out=y), max(3, iters // 4))
+        res["dense_gemm_bf16_us"] = 1e3 * g_ms
+        res["dense_gemm_tflops"] = 2.0 * w.T * w.d * w.d / (g_ms * 1e-3) / 1e12
+    return res
+
+
+def run_ours(args, rank: int, world: int, local_rank: int):
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    import torch.distributed as dist
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    from paper_2603_08343_b200 import build as _build
+    if rank == 0:
+        _build.build()
+    if world > 1:
+        dist.barrier()
+    from paper_2603_08343_b200 import binding as B
+    if args.variant:
+        B.wht_affine_set_variant(args.variant)
+
+    hbm_peak, peak_src = load_peaks()
+    w = wl.CONFIGS[args.workload]
+    # every rank draws its own rows (weak scaling): the seed is offset by the rank
+    wr = wl.Workload(w.name, w.T, w.d, w.dtype, w.dist, w.seed + 1000 * rank, w.has_bwd, w.note)
+    base_rows = min(w.T, 8192) if w.dist != "normal" else w.T
+    a_h, b_h = wl.gen_params(wr)
+    x_h = wl.gen_full(wr.with_rows(base_rows), "x", threads=16)
+    dy_h = wl.gen_full(wr.with_rows(base_rows), "dy", threads=16) if w.has_bwd else None
+    reps = w.T // base_rows
+    a, b = a_h.cuda(), b_h.cuda()
+    x = x_h.cuda().repeat(reps, 1)
+    dy = dy_h.cuda().repeat(reps, 1) if w.has_bwd else None
+    y = torch.empty_like(x)
+    dx = torch.empty_like(x) if w.has_bwd else None
+    da = torch.empty(w.d, dtype=torch.float32, device="cuda")
+    db = torch.empty_like(da)
+    grads = torch.empty(2 * w.d, dtype=torch.float32, device="cuda")
+
+    # small working sets are rotated through enough buffers to exceed L2 (126 MB)
+    step_bytes = (4 if w.has_bwd else 2) * w.T * w.d * w.io_bytes
+    nbuf = 1 if step_bytes > 400e6 else int(np.ceil(1.0e9 / step_bytes))
+    xs, ys, dys, dxs = [x], [y], [dy], [dx]
+    for _ in range(nbuf - 1):
+        xs.append(x.clone())
+        ys.append(torch.empty_like(x))
+        dys.append(dy.clone() if w.has_bwd else None)
+        dxs.append(torch.empty_like(x) if w.has_bwd else None)
+    l2_note = ("working set %.0f MB per step, larger than L2" % (step_bytes / 1e6)) if nbuf == 1 else \
+        f"{nbuf} rotating buffer sets ({nbuf * step_bytes / 1e6:.0f} MB), larger than L2"
+    counter = {"i": 0}
+    launches_per_step = 1 + (2 if w.has_bwd else 0)
+
+    def step(ev=None):
+        i = counter["i"] % nbuf
+        counter["i"] += 1
+        if ev is not None:
+            ev[0].record()
+        B.wht_affine_fwd(xs[i], a, b, ys[i], w.T, w.d, w.dtype)
+        if ev is not None:
+            ev[1].record()
+        if w.has_bwd:
+            B.wht_affine_bwd(dys[i], xs[i], a, dxs[i], da, db, w.T, w.d, w.dtype)
+            if ev is not None:
+                ev[2].record()
+            if world > 1:
+                grads[:w.d].copy_(da)
+                grads[w.d:].copy_(db)
+                dist.all_reduce(grads)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    torch.cuda.synchronize()
+    events = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    t_wall0 = time.time()
+    with Timer() as total:
+        for k in range(args.steps):
+            step(events[k])
+    total_ms = total.ms()
+    torch.cuda.synchronize()
+    t_wall1 = time.time()
+    if world > 1:
+        dist.barrier()
+        tmax = torch.tensor([total_ms], device="cuda")
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+        total_ms = float(tmax.item())
+    clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
+
+    fwd_ms = [e[0].elapsed_time(e[1]) for e in events]
+    bwd_ms = [e[1].elapsed_time(e[2]) for e in events] if w.has_bwd else []
+    ms_per_step = total_ms / args.steps
+    value = world * w.T / (ms_per_step * 1e-3)
+
+    # roofline of the dominant kernel: the backward main kernel when there is one
+    if w.has_bwd:
+        dom, dom_ms = "wht_affine_bwd (main kernel + the small finalize pass)", statistics.mean(bwd_ms)
+        bytes_per_launch = 3 * w.T * w.d * w.io_bytes
+    else:
+        dom, dom_ms = "wht_affine_fwd", statistics.mean(fwd_ms)
+        bytes_per_launch = 2 * w.T * w.d * w.io_bytes
+    achieved = bytes_per_launch / 1e9 / (dom_ms * 1e-3)
+    roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": hbm_peak, "unit": "GB/s",
+                "frac": achieved / hbm_peak, "peak_source": peak_src, "traffic": None,
+                "algorithmic_bytes_per_launch": bytes_per_launch, "avg_launch_ms": dom_ms,
+                "frac_of_nominal_8000": achieved / 8000.0}
+    fwd_gbps = 2 * w.T * w.d * w.io_bytes / 1e9 / (statistics.mean(fwd_ms) * 1e-3)
+
+    # ---- end to end: pinned host buffers in, results back to the host, every step
+    e2e = None
+    staging = {"x": x, "a": a, "b": b, "y": y, "dy": dy, "dx": dx, "da": da, "db": db}
+    xp, ap, bp = x_h.repeat(reps, 1).pin_memory(), a_h.pin_memory(), b_h.pin_memory()
+    yp = torch.empty_like(xp).pin_memory()
+    h2d = xp.numel() * xp.element_size() + 2 * ap.numel() * ap.element_size()
+    d2h = yp.numel() * yp.element_size()
+    if w.has_bwd:
+        dyp = dy_h.repeat(reps, 1).pin_memory()
+        dxp = torch.empty_like(xp).pin_memory()
+        dap = torch.empty(w.d, dtype=torch.float32).pin_memory()
+        dbp = torch.empty(w.d, dtype=torch.float32).pin_memory()
+        h2d += dyp.numel() * dyp.element_size() + xp.numel() * xp.element_size() + ap.numel() * ap.element_size()
+        d2h += dxp.numel() * dxp.element_size() + 8 * w.d
+
+    def e2e_step():
+        B.forward_host(xp, ap, bp, yp, staging)
+        if w.has_bwd:
+            B.backward_host(dyp, xp, ap, dxp, dap, dbp, staging)
+
+    e2e_steps = max(2, min(args.steps, 5))
+    e2e_ms = time_loop(e2e_step, e2e_steps, warmup=1)
+    if world > 1:
+        tmax = torch.tensor([e2e_ms], device="cuda")
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+        e2e_ms = float(tmax.item())
+    e2e = {"value": world * w.T / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
+           "d2h_bytes_per_step": int(d2h), "ms_per_step": e2e_ms, "steps": e2e_steps,
+           "api": "binding.forward_host + binding.backward_host (pinned host -> device -> C ABI -> pinned host)"}
+    del xp, yp, staging
+    if w.has_bwd:
+        del dyp, dxp
+    if world > 1:
+        dist.barrier()
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+        "data": "synthetic",
+        "config": {"workload": w.name, "T_per_gpu": w.T, "d": w.d,
+                   "storage": {0: "fp32", 1: "bf16 rows, bf16 params", 2: "bf16 rows, fp32 params"}[w.dtype],
+                   "step": "wht_affine_fwd + wht_affine_bwd" if w.has_bwd else "wht_affine_fwd",
+                   "l2": l2_note, "variant": B.wht_affine_get_variant(),
+                   "parallelism": f"dp{world} (rows sharded; all-reduce of da|db only)" if world > 1 else "single GPU"},
+        "fwd": {"ms": statistics.mean(fwd_ms), "GBps": fwd_gbps, "frac_of_measured_peak": fwd_gbps / hbm_peak,
+                "frac_of_nominal_8000": fwd_gbps / 8000.0, "tokens_per_s": w.T / (statistics.mean(fwd_ms) * 1e-3)},
+        "roofline": roofline, "e2e": e2e, "gpu_launches": launches_per_step * args.steps, "clocks": clocks,
+    }
+    if w.has_bwd:
+        out["bwd"] = {"ms": dom_ms, "GBps": achieved, "frac_of_measured_peak": achieved / hbm_peak,
+                      "frac_of_nominal_8000": achieved / 8000.0, "tokens_per_s": w.T / (dom_ms * 1e-3)}
+
+    # ---- CPU baseline: the oracle as it stands, on a bounded sample of the same workload
+    rows = {"tiny": 64, "prefill": 4096, "training": 2048, "large": 256}[w.name]
+    sec = oracle_step_seconds(w, rows)
+    out["cpu_baseline"] = {"value": rows / sec, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+                           "seconds": sec,
+                           "sample": f"{rows} rows of the {w.name} workload (d={w.d}), fp64 dense product, "
+                                     f"fwd{'+bwd' if w.has_bwd else ''}; tokens/s from that sample (per-row cost is constant)"}
+
+    if not args.no_sections and world == 1:
+        del xs, ys, dys, dxs, x, y, dy, dx
+        torch.cuda.empty_cache()
+        sections = {}
+        sections["prefill"] = section_prefill(B, hbm_peak)
+        sections["decode"] = section_decode(B)
+        sections["training"] = section_fwd_bwd(B, "training", hbm_peak, 20)
+        sections["large"] = section_fwd_bwd(B, "large", hbm_peak, 5)
+        out["sections"] = sections
+    print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default="training", choices=["tiny", "prefill", "training", "large"])
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--variant", type=int, default=0)
+    ap.add_argument("--no-sections", action="store_true")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank, world)
+        return
+    run_ours(args, rank, world, local_rank)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,141 @@
+/*
+ * wht_affine.h -- C ABI of the B200 (sm_100a) Walsh-Hadamard head-mixing library.
+ *
+ * The operation is the paper's replacement for the dense attention output
+ * projection (Eq. 1):
+ *
+ *     y[t, :] = a (.) ( x[t, :] H_d ) / sqrt(d) + b          for every row t < T
+ *
+ * H_d is the d x d Walsh-Hadamard matrix in Sylvester (natural) order,
+ * H[i][j] = (-1)^popcount(i & j) -- the ordering of the 4x4 sign pattern printed
+ * in Fig. 1 and of the in-place butterfly of Fig. 2 -- and the 1/sqrt(d) factor
+ * makes it orthonormal (the condition H^T H = I stated under Eq. 1).  a and b are
+ * the trainable per-channel scale and bias (alpha and beta in Eq. 1).
+ *
+ * Conventions common to every entry point
+ *   - All tensor pointers are DEVICE pointers owned by the caller.  x, y, dy, dx
+ *     are row-major contiguous [T x d] (row stride = d elements); a, b, da, db
+ *     have d elements.  Every pointer must be 16-byte aligned.
+ *   - d must be a power of two with 8 <= d <= 32768.  T >= 0; T == 0 is a no-op
+ *     for the forward calls, and makes the backward call write zeros to da, db
+ *     (the row tensors may then be NULL; a, b, da, db are always required).
+ *   - `dtype` selects the storage types (wht_dtype below).  All arithmetic is
+ *     fp32 whatever the storage type; bf16 outputs are rounded once, to nearest
+ *     even, at the store.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ *     Calls are asynchronous: they enqueue work and return without synchronising.
+ *   - Exact aliasing y == x and dx == dy is allowed (a row is read completely
+ *     before it is written).  Any other overlap is undefined.
+ *   - Return value: WHT_OK (0) or a negative wht_status.  On error nothing has
+ *     been launched.  No exception crosses this boundary and no kernel traps.
+ */
+#ifndef WHT_AFFINE_H_
+#define WHT_AFFINE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    WHT_F32 = 0,       /* x, y, dy, dx, a, b : float32                              */
+    WHT_BF16 = 1,      /* x, y, dy, dx, a, b : bfloat16            (inference)      */
+    WHT_BF16_PF32 = 2  /* x, y, dy, dx : bfloat16 ;  a, b : float32 (training)      */
+} wht_dtype;           /* da and db are float32 for every dtype                      */
+
+typedef enum {
+    WHT_OK = 0,
+    WHT_ERR_NULL = -1,        /* a required pointer is NULL                          */
+    WHT_ERR_BAD_DIM = -2,     /* d is not a power of two in [8, 32768]               */
+    WHT_ERR_BAD_T = -3,       /* T < 0                                               */
+    WHT_ERR_BAD_DTYPE = -4,   /* dtype is not a wht_dtype                            */
+    WHT_ERR_MISALIGNED = -5,  /* a pointer is not 16-byte aligned                    */
+    WHT_ERR_WORKSPACE = -6,   /* workspace missing, too small, or allocation failed  */
+    WHT_ERR_CUDA = -7,        /* a CUDA runtime call failed; see wht_affine_last_cuda_error */
+    WHT_ERR_BAD_VARIANT = -8  /* unknown kernel variant id                           */
+} wht_status;
+
+/*
+ * Forward pass (Eq. 1): y = a (.) (x H_d)/sqrt(d) + b on T rows.
+ *   x [T x d] in, a [d] in, b [d] in, y [T x d] out.  Reads x once, writes y once.
+ */
+int wht_affine_fwd(const void* x, const void* a, const void* b, void* y,
+                   int64_t T, int32_t d, int dtype, void* stream);
+
+/*
+ * Forward pass tuned for a handful of rows (the decode regime of the paper's
+ * inference benchmark: one new token per sequence).  Same arguments, semantics
+ * and results as wht_affine_fwd; any T is legal, T <= 256 is what it is shaped
+ * for.  Uses no workspace and makes no allocation.
+ */
+int wht_affine_fwd_decode(const void* x, const void* a, const void* b, void* y,
+                          int64_t T, int32_t d, int dtype, void* stream);
+
+/*
+ * Backward pass of Eq. 1 (the paper states only its O(d log d) cost in the table
+ * comparing the dense and Hadamard projections; the formulas are the chain rule
+ * applied to Eq. 1, with z = (x H_d)/sqrt(d) recomputed from x):
+ *     dx[t, :] = ( (a (.) dy[t, :]) H_d ) / sqrt(d)         (H is symmetric)
+ *     da[j]    = sum_t dy[t, j] * z[t, j]
+ *     db[j]    = sum_t dy[t, j]
+ *   dy [T x d] in, x [T x d] in, a [d] in, dx [T x d] out, da [d] out, db [d] out.
+ * da and db are OVERWRITTEN (not accumulated) and are float32.  The column sums
+ * are taken in a fixed order, so results are bit-identical from run to run.
+ *
+ * This call uses a per-device scratch buffer owned by the library, allocated
+ * with cudaMalloc on first use (and grown when a larger problem arrives), so the
+ * first call for a given size synchronises and must not happen during stream
+ * capture.  Concurrent backward calls on one device through this entry point
+ * share that buffer and must be serialised by the caller; use wht_affine_bwd_ws
+ * to give each call site its own.
+ */
+int wht_affine_bwd(const void* dy, const void* x, const void* a,
+                   void* dx, float* da, float* db,
+                   int64_t T, int32_t d, int dtype, void* stream);
+
+/*
+ * Backward pass with caller-owned scratch: identical results to wht_affine_bwd.
+ * `workspace` is a 16-byte aligned device buffer of at least
+ * wht_affine_bwd_workspace_bytes(T, d, dtype) bytes; its contents on entry are
+ * ignored and undefined on exit.  Never allocates.
+ */
+int wht_affine_bwd_ws(const void* dy, const void* x, const void* a,
+                      void* dx, float* da, float* db,
+                      int64_t T, int32_t d, int dtype,
+                      void* workspace, size_t workspace_bytes, void* stream);
+
+/* Scratch bytes wht_affine_bwd_ws needs on the current device (0 on bad arguments). */
+size_t wht_affine_bwd_workspace_bytes(int64_t T, int32_t d, int dtype);
+
+/*
+ * Kernel family used by the three compute calls (for A/B measurements):
+ *   0 = automatic (default), 1 = butterfly (registers + warp shuffles + shared
+ *   memory), 2 = tensor-core assisted (H_16 factors through mma, bf16 storage only).
+ * A variant that does not support the requested (d, dtype) falls back to 1.
+ * Process-wide; not meant to be changed while calls are in flight.
+ */
+int wht_affine_set_variant(int variant);
+int wht_affine_get_variant(void);
+
+/*
+ * Bandwidth yardstick with the same access pattern as the forward pass: copies
+ * T rows of d elements (element size from dtype) from src to dst.  Used only by
+ * the benchmark to report a practical copy ceiling next to the kernels.
+ */
+int wht_copy_rows(const void* src, void* dst, int64_t T, int32_t d, int dtype, void* stream);
+
+/* cudaError_t of the most recent failing CUDA call on this thread (0 if none). */
+int wht_affine_last_cuda_error(void);
+
+/* Human-readable name of a wht_status. */
+const char* wht_affine_status_string(int status);
+
+/* Frees the library-owned scratch buffers of all devices.  Safe to call twice. */
+int wht_affine_shutdown(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* WHT_AFFINE_H_ */

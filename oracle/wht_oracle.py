@@ -27,6 +27,7 @@ for the gradients.  No function here is "parity unpinned".
 """
 from __future__ import annotations
 
+import functools
 import math
 
 import numpy as np
@@ -38,20 +39,24 @@ def _log2_exact(d: int) -> int:
     return d.bit_length() - 1
 
 
+@functools.lru_cache(maxsize=3)
 def sylvester_hadamard(d: int) -> np.ndarray:
     """Unnormalised d x d matrix of +-1 in Sylvester order (Fig. 1 sign pattern).
 
-    H[i][j] = +1 when popcount(i & j) is even, -1 when it is odd.
+    H[i][j] = +1 when popcount(i & j) is even, -1 when it is odd.  The matrix is
+    a constant of d, so the last few sizes are kept (read-only) between calls.
     """
     _log2_exact(d)
-    idx = np.arange(d, dtype=np.int64)
+    idx = np.arange(d, dtype=np.int32)
     both = idx[:, None] & idx[None, :]
-    parity = np.zeros((d, d), dtype=np.int64)
+    parity = np.zeros((d, d), dtype=np.int8)
     bit = 1
     while bit < d:
-        parity ^= (both & bit) != 0
+        parity ^= ((both & bit) != 0).astype(np.int8)
         bit <<= 1
-    return (1 - 2 * parity).astype(np.float64)
+    H = (1 - 2 * parity).astype(np.float64)
+    H.setflags(write=False)
+    return H
 
 
 def widen_bf16_bits(bits: np.ndarray) -> np.ndarray:

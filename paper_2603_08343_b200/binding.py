@@ -1,0 +1,199 @@
+"""ctypes binding of libwht_affine.so: same names and argument order as include/wht_affine.h.
+
+Argument marshalling only -- every step of the path runs in the library's CUDA
+kernels.  torch is used for device memory and the current stream.  If the shared
+library is missing or cannot be loaded, importing this module raises; there is
+no CPU fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+from .workloads import WHT_BF16, WHT_BF16_PF32, WHT_F32
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libwht_affine.so")
+
+EXPORTS = (
+    "wht_affine_fwd", "wht_affine_fwd_decode", "wht_affine_bwd", "wht_affine_bwd_ws",
+    "wht_affine_bwd_workspace_bytes", "wht_affine_set_variant", "wht_affine_get_variant",
+    "wht_copy_rows", "wht_affine_last_cuda_error", "wht_affine_status_string",
+    "wht_affine_shutdown",
+)
+
+
+class WhtError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        msg = _lib.wht_affine_status_string(status).decode()
+        cuda = _lib.wht_affine_last_cuda_error()
+        super().__init__(f"{where}: {msg} (status {status}, cuda error {cuda})")
+
+
+def _load() -> ctypes.CDLL:
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(
+            f"{LIB_PATH} is missing: build it with `python -m paper_2603_08343_b200.build` "
+            "(there is no CPU fallback)")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, i64, i32, ci, sz = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32, ctypes.c_int, ctypes.c_size_t
+    lib.wht_affine_fwd.argtypes = [vp, vp, vp, vp, i64, i32, ci, vp]
+    lib.wht_affine_fwd_decode.argtypes = [vp, vp, vp, vp, i64, i32, ci, vp]
+    lib.wht_affine_bwd.argtypes = [vp, vp, vp, vp, vp, vp, i64, i32, ci, vp]
+    lib.wht_affine_bwd_ws.argtypes = [vp, vp, vp, vp, vp, vp, i64, i32, ci, vp, sz, vp]
+    lib.wht_affine_bwd_workspace_bytes.argtypes = [i64, i32, ci]
+    lib.wht_affine_bwd_workspace_bytes.restype = sz
+    lib.wht_affine_set_variant.argtypes = [ci]
+    lib.wht_affine_get_variant.argtypes = []
+    lib.wht_copy_rows.argtypes = [vp, vp, i64, i32, ci, vp]
+    lib.wht_affine_last_cuda_error.argtypes = []
+    lib.wht_affine_status_string.argtypes = [ci]
+    lib.wht_affine_status_string.restype = ctypes.c_char_p
+    lib.wht_affine_shutdown.argtypes = []
+    for name in EXPORTS:
+        fn = getattr(lib, name)
+        if fn.restype is ctypes.c_int or fn.restype is None:
+            fn.restype = ctypes.c_int
+    return lib
+
+
+_lib = _load()
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded shared library (for tests that call the C ABI with raw pointers)."""
+    return _lib
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _check(status: int, where: str) -> None:
+    if status != 0:
+        raise WhtError(status, where)
+
+
+def _require_cuda(*tensors):
+    for t in tensors:
+        if t is not None and not t.is_cuda:
+            raise ValueError("tensors must live on a CUDA device")
+        if t is not None and not t.is_contiguous():
+            raise ValueError("tensors must be contiguous")
+
+
+def wht_affine_fwd(x, a, b, y, T: int, d: int, dtype: int, stream=None) -> None:
+    _require_cuda(x, a, b, y)
+    _check(_lib.wht_affine_fwd(_ptr(x), _ptr(a), _ptr(b), _ptr(y), T, d, dtype, _stream(stream)),
+           "wht_affine_fwd")
+
+
+def wht_affine_fwd_decode(x, a, b, y, T: int, d: int, dtype: int, stream=None) -> None:
+    _require_cuda(x, a, b, y)
+    _check(_lib.wht_affine_fwd_decode(_ptr(x), _ptr(a), _ptr(b), _ptr(y), T, d, dtype, _stream(stream)),
+           "wht_affine_fwd_decode")
+
+
+def wht_affine_bwd(dy, x, a, dx, da, db, T: int, d: int, dtype: int, stream=None) -> None:
+    _require_cuda(dy, x, a, dx, da, db)
+    _check(_lib.wht_affine_bwd(_ptr(dy), _ptr(x), _ptr(a), _ptr(dx), _ptr(da), _ptr(db), T, d, dtype,
+                               _stream(stream)), "wht_affine_bwd")
+
+
+def wht_affine_bwd_ws(dy, x, a, dx, da, db, T: int, d: int, dtype: int, workspace, stream=None) -> None:
+    _require_cuda(dy, x, a, dx, da, db, workspace)
+    nbytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(_lib.wht_affine_bwd_ws(_ptr(dy), _ptr(x), _ptr(a), _ptr(dx), _ptr(da), _ptr(db), T, d, dtype,
+                                  _ptr(workspace), nbytes, _stream(stream)), "wht_affine_bwd_ws")
+
+
+def wht_affine_bwd_workspace_bytes(T: int, d: int, dtype: int) -> int:
+    return int(_lib.wht_affine_bwd_workspace_bytes(T, d, dtype))
+
+
+def wht_affine_set_variant(variant: int) -> None:
+    _check(_lib.wht_affine_set_variant(variant), "wht_affine_set_variant")
+
+
+def wht_affine_get_variant() -> int:
+    return int(_lib.wht_affine_get_variant())
+
+
+def wht_copy_rows(src, dst, T: int, d: int, dtype: int, stream=None) -> None:
+    _require_cuda(src, dst)
+    _check(_lib.wht_copy_rows(_ptr(src), _ptr(dst), T, d, dtype, _stream(stream)), "wht_copy_rows")
+
+
+def wht_affine_shutdown() -> None:
+    _check(_lib.wht_affine_shutdown(), "wht_affine_shutdown")
+
+
+# ---- convenience wrappers that infer T, d and the dtype code from the tensors ----
+
+def dtype_code(x: torch.Tensor, a: torch.Tensor) -> int:
+    if x.dtype == torch.float32 and a.dtype == torch.float32:
+        return WHT_F32
+    if x.dtype == torch.bfloat16 and a.dtype == torch.bfloat16:
+        return WHT_BF16
+    if x.dtype == torch.bfloat16 and a.dtype == torch.float32:
+        return WHT_BF16_PF32
+    raise ValueError(f"unsupported storage types x={x.dtype}, a={a.dtype}")
+
+
+def forward(x, a, b, out=None, decode: bool = False, stream=None):
+    """y = a (.) (x H)/sqrt(d) + b for x[..., d]; returns `out` (allocated if None)."""
+    d = x.shape[-1]
+    T = x.numel() // d if d else 0
+    y = torch.empty_like(x) if out is None else out
+    fn = wht_affine_fwd_decode if decode else wht_affine_fwd
+    fn(x, a, b, y, T, d, dtype_code(x, a), stream)
+    return y
+
+
+def backward(dy, x, a, stream=None):
+    """(dx, da, db) for the forward above; da, db are fp32."""
+    d = x.shape[-1]
+    T = x.numel() // d if d else 0
+    dx = torch.empty_like(x)
+    da = torch.empty(d, dtype=torch.float32, device=x.device)
+    db = torch.empty(d, dtype=torch.float32, device=x.device)
+    wht_affine_bwd(dy, x, a, dx, da, db, T, d, dtype_code(x, a), stream)
+    return dx, da, db
+
+
+def forward_host(x_host, a_host, b_host, y_host, staging, stream=None):
+    """End-to-end forward from pinned host memory: copy in, transform, copy out.
+
+    `staging` is a dict of preallocated device tensors {"x", "a", "b", "y"}.
+    All copies are asynchronous on the current stream.
+    """
+    staging["x"].copy_(x_host, non_blocking=True)
+    staging["a"].copy_(a_host, non_blocking=True)
+    staging["b"].copy_(b_host, non_blocking=True)
+    forward(staging["x"], staging["a"], staging["b"], out=staging["y"], stream=stream)
+    y_host.copy_(staging["y"], non_blocking=True)
+    return y_host
+
+
+def backward_host(dy_host, x_host, a_host, dx_host, da_host, db_host, staging, stream=None):
+    """End-to-end backward from pinned host memory; `staging` holds device tensors
+    {"dy", "x", "a", "dx", "da", "db"}."""
+    st = staging
+    st["dy"].copy_(dy_host, non_blocking=True)
+    st["x"].copy_(x_host, non_blocking=True)
+    st["a"].copy_(a_host, non_blocking=True)
+    d = st["x"].shape[-1]
+    T = st["x"].numel() // d
+    wht_affine_bwd(st["dy"], st["x"], st["a"], st["dx"], st["da"], st["db"], T, d,
+                   dtype_code(st["x"], st["a"]), stream)
+    dx_host.copy_(st["dx"], non_blocking=True)
+    da_host.copy_(st["da"], non_blocking=True)
+    db_host.copy_(st["db"], non_blocking=True)

@@ -1,0 +1,316 @@
+// Butterfly kernel family: the FWHT of Fig. 2 on one row per thread group.
+//
+// Index bits of a row of d = 2^LOGD elements are split as
+//     [ chunk c (log2 C) | thread t in group (log2 G) | element e (3) ]
+// A thread owns C chunks of 8 contiguous elements (one 128-bit access each for
+// bf16).  Stages on the e bits and the c bits run in registers, stages on the
+// low 5 bits of t run across lanes with __shfl_xor_sync, and stages on the
+// remaining bits of t (rows wider than one warp) run through a shared-memory
+// copy of the row in radix-8 rounds.  The 1/sqrt(d) scale, a and b are applied
+// when the row is written out.  Works for every power of two 8 <= d <= 32768
+// and every storage type; it is also the only family for fp32 storage.
+#pragma once
+#include "wht_common.cuh"
+
+namespace wht {
+
+template <int LOGD>
+struct BflyGeo {
+    static constexpr int D = 1 << LOGD;
+    static constexpr int C = imax_c(1, D / 8192);      // chunks of 8 per thread
+    static constexpr int G = D / (8 * C);              // threads per row, 1..1024
+    static constexpr int LOGG = ilog2_c(G);
+    static constexpr int THREADS = imax_c(G, 256);
+    static constexpr int R = THREADS / G;              // rows per CTA tile
+    static constexpr int LANE_BITS = imin_c(5, LOGG);
+    static constexpr int WARP_BITS = LOGG - LANE_BITS; // stages that cross warps
+    static constexpr int SMEM_ROW_BYTES = D * 4;
+    static constexpr int SMEM_FWD = WARP_BITS > 0 ? R * D * 4 : 0;
+    static constexpr int SMEM_BWD = R * D * 4;
+};
+
+// One radix-2^NB round on row bits [P, P+NB) through shared memory.
+template <int LOGD, int P, int NB>
+__device__ __forceinline__ void bfly_smem_round(float* srow, int t) {
+    using Geo = BflyGeo<LOGD>;
+    constexpr int SETS = (8 * Geo::C) >> NB;
+    constexpr int N = 1 << NB;
+#pragma unroll
+    for (int k = 0; k < SETS; ++k) {
+        const int s = t + Geo::G * k;
+        const int base = ((s >> P) << (P + NB)) | (s & ((1 << P) - 1));
+        float r[N];
+#pragma unroll
+        for (int j = 0; j < N; ++j) r[j] = srow[base + (j << P)];
+#pragma unroll
+        for (int h = 1; h < N; h <<= 1) {
+#pragma unroll
+            for (int j = 0; j < N; ++j) {
+                if ((j & h) == 0) {
+                    const float lo = r[j], hi = r[j + h];
+                    r[j] = lo + hi;
+                    r[j + h] = lo - hi;
+                }
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < N; ++j) srow[base + (j << P)] = r[j];
+    }
+}
+
+template <int LOGD, int P, int REM>
+struct BflyCrossRounds {
+    static __device__ __forceinline__ void run(float* srow, int t) {
+        constexpr int NB = imin_c(3, REM);
+        bfly_smem_round<LOGD, P, NB>(srow, t);
+        __syncthreads();
+        BflyCrossRounds<LOGD, P + NB, REM - NB>::run(srow, t);
+    }
+};
+template <int LOGD, int P>
+struct BflyCrossRounds<LOGD, P, 0> {
+    static __device__ __forceinline__ void run(float*, int) {}
+};
+
+// Unnormalised H_d applied in place to the row held by one thread group.
+// Every thread of the CTA must call this (it contains __syncthreads when the
+// row spans several warps).
+template <int LOGD>
+__device__ __forceinline__ void bfly_row_transform(float (&v)[BflyGeo<LOGD>::C][8], float* srow, int t) {
+    using Geo = BflyGeo<LOGD>;
+#pragma unroll
+    for (int c = 0; c < Geo::C; ++c) bfly8(v[c]);
+    // chunk bits (the top log2 C bits of the row index)
+#pragma unroll
+    for (int h = 1; h < Geo::C; h <<= 1) {
+#pragma unroll
+        for (int c = 0; c < Geo::C; ++c) {
+            if ((c & h) == 0) {
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    const float lo = v[c][e], hi = v[c + h][e];
+                    v[c][e] = lo + hi;
+                    v[c + h][e] = lo - hi;
+                }
+            }
+        }
+    }
+    // lane bits: the partner's value arrives by shuffle; the upper lane of a
+    // pair keeps (partner - own), the lower (own + partner)
+#pragma unroll
+    for (int m = 1; m < (1 << Geo::LANE_BITS); m <<= 1) {
+        const float sgn = (t & m) ? -1.0f : 1.0f;
+#pragma unroll
+        for (int c = 0; c < Geo::C; ++c) {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                const float other = __shfl_xor_sync(kFullMask, v[c][e], m);
+                v[c][e] = fmaf(v[c][e], sgn, other);
+            }
+        }
+    }
+    if constexpr (Geo::WARP_BITS > 0) {
+#pragma unroll
+        for (int c = 0; c < Geo::C; ++c) {
+            float4* dst = reinterpret_cast<float4*>(srow + (c * Geo::G + t) * 8);
+            dst[0] = make_float4(v[c][0], v[c][1], v[c][2], v[c][3]);
+            dst[1] = make_float4(v[c][4], v[c][5], v[c][6], v[c][7]);
+        }
+        __syncthreads();
+        BflyCrossRounds<LOGD, 3 + Geo::LANE_BITS, Geo::WARP_BITS>::run(srow, t);
+#pragma unroll
+        for (int c = 0; c < Geo::C; ++c) {
+            const float4* src = reinterpret_cast<const float4*>(srow + (c * Geo::G + t) * 8);
+            const float4 q0 = src[0], q1 = src[1];
+            v[c][0] = q0.x; v[c][1] = q0.y; v[c][2] = q0.z; v[c][3] = q0.w;
+            v[c][4] = q1.x; v[c][5] = q1.y; v[c][6] = q1.z; v[c][7] = q1.w;
+        }
+    }
+}
+
+// Streaming row access: rows are touched once, so mark them evict-first.
+__device__ __forceinline__ void load8_stream(const float* p, float (&v)[8]) {
+    const float4 q0 = __ldcs(reinterpret_cast<const float4*>(p));
+    const float4 q1 = __ldcs(reinterpret_cast<const float4*>(p) + 1);
+    v[0] = q0.x; v[1] = q0.y; v[2] = q0.z; v[3] = q0.w;
+    v[4] = q1.x; v[5] = q1.y; v[6] = q1.z; v[7] = q1.w;
+}
+__device__ __forceinline__ void load8_stream(const __nv_bfloat16* p, float (&v)[8]) {
+    const uint4 q = __ldcs(reinterpret_cast<const uint4*>(p));
+    v[0] = bf16lo_to_f32(q.x); v[1] = bf16hi_to_f32(q.x);
+    v[2] = bf16lo_to_f32(q.y); v[3] = bf16hi_to_f32(q.y);
+    v[4] = bf16lo_to_f32(q.z); v[5] = bf16hi_to_f32(q.z);
+    v[6] = bf16lo_to_f32(q.w); v[7] = bf16hi_to_f32(q.w);
+}
+__device__ __forceinline__ void store8_stream(float* p, const float (&v)[8]) {
+    __stcs(reinterpret_cast<float4*>(p), make_float4(v[0], v[1], v[2], v[3]));
+    __stcs(reinterpret_cast<float4*>(p) + 1, make_float4(v[4], v[5], v[6], v[7]));
+}
+__device__ __forceinline__ void store8_stream(__nv_bfloat16* p, const float (&v)[8]) {
+    uint4 q;
+    q.x = pack_bf16x2(v[0], v[1]);
+    q.y = pack_bf16x2(v[2], v[3]);
+    q.z = pack_bf16x2(v[4], v[5]);
+    q.w = pack_bf16x2(v[6], v[7]);
+    __stcs(reinterpret_cast<uint4*>(p), q);
+}
+
+// ---- forward: y = a (.) (x H)/sqrt(d) + b ------------------------------------
+template <int LOGD, typename TIO, typename TP>
+__global__ void __launch_bounds__(BflyGeo<LOGD>::THREADS)
+bfly_fwd_kernel(const TIO* x, const TP* __restrict__ a, const TP* __restrict__ b, TIO* y,
+                long long T, float inv_sqrt_d) {
+    using Geo = BflyGeo<LOGD>;
+    extern __shared__ __align__(16) float smem[];
+    const int rg = threadIdx.x / Geo::G;  // row group inside the CTA
+    const int t = threadIdx.x % Geo::G;
+    float* srow = smem + (Geo::WARP_BITS > 0 ? rg * Geo::D : 0);
+
+    float as[Geo::C][8], bs[Geo::C][8];
+#pragma unroll
+    for (int c = 0; c < Geo::C; ++c) {
+        load8(a + (c * Geo::G + t) * 8, as[c]);
+        load8(b + (c * Geo::G + t) * 8, bs[c]);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) as[c][e] *= inv_sqrt_d;
+    }
+
+    const long long tiles = (T + Geo::R - 1) / Geo::R;
+    for (long long tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
+        const long long row = tile * Geo::R + rg;
+        const bool valid = row < T;
+        float v[Geo::C][8];
+#pragma unroll
+        for (int c = 0; c < Geo::C; ++c) {
+            if (valid) {
+                load8_stream(x + row * Geo::D + (c * Geo::G + t) * 8, v[c]);
+            } else {
+#pragma unroll
+                for (int e = 0; e < 8; ++e) v[c][e] = 0.0f;
+            }
+        }
+        bfly_row_transform<LOGD>(v, srow, t);
+        if (valid) {
+#pragma unroll
+            for (int c = 0; c < Geo::C; ++c) {
+#pragma unroll
+                for (int e = 0; e < 8; ++e) v[c][e] = fmaf(v[c][e], as[c][e], bs[c][e]);
+                store8_stream(y + row * Geo::D + (c * Geo::G + t) * 8, v[c]);
+            }
+        }
+    }
+}
+
+// ---- backward: dx = ((a (.) dy) H)/sqrt(d); per-CTA partial da, db -------------
+// partials layout: [gridDim.x][2][D] fp32; slot 0 holds sum_t dy (.) (x H) WITHOUT
+// the 1/sqrt(d) factor (the finalize pass applies it), slot 1 holds sum_t dy.
+template <int LOGD, typename TIO, typename TP>
+__global__ void __launch_bounds__(BflyGeo<LOGD>::THREADS)
+bfly_bwd_kernel(const TIO* dy, const TIO* x, const TP* __restrict__ a, TIO* dx,
+                float* __restrict__ partials, long long T, float inv_sqrt_d) {
+    using Geo = BflyGeo<LOGD>;
+    extern __shared__ __align__(16) float smem[];
+    const int rg = threadIdx.x / Geo::G;
+    const int t = threadIdx.x % Geo::G;
+    float* srow = smem + rg * Geo::D;
+
+    float da_acc[Geo::C][8], db_acc[Geo::C][8];
+#pragma unroll
+    for (int c = 0; c < Geo::C; ++c) {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) { da_acc[c][e] = 0.0f; db_acc[c][e] = 0.0f; }
+    }
+
+    const long long tiles = (T + Geo::R - 1) / Geo::R;
+    for (long long tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
+        const long long row = tile * Geo::R + rg;
+        const bool valid = row < T;
+        float v[Geo::C][8], w[Geo::C][8];
+#pragma unroll
+        for (int c = 0; c < Geo::C; ++c) {
+            if (valid) {
+                load8_stream(x + row * Geo::D + (c * Geo::G + t) * 8, v[c]);
+                load8_stream(dy + row * Geo::D + (c * Geo::G + t) * 8, w[c]);
+            } else {
+#pragma unroll
+                for (int e = 0; e < 8; ++e) { v[c][e] = 0.0f; w[c][e] = 0.0f; }
+            }
+        }
+        bfly_row_transform<LOGD>(v, srow, t);  // v = x H (unnormalised)
+#pragma unroll
+        for (int c = 0; c < Geo::C; ++c) {
+            float as[8];
+            load8(a + (c * Geo::G + t) * 8, as);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                da_acc[c][e] = fmaf(w[c][e], v[c][e], da_acc[c][e]);
+                db_acc[c][e] += w[c][e];
+                v[c][e] = as[e] * w[c][e];
+            }
+        }
+        if constexpr (Geo::WARP_BITS > 0) __syncthreads();  // srow is reused by the second transform
+        bfly_row_transform<LOGD>(v, srow, t);  // v = (a (.) dy) H
+        if (valid) {
+#pragma unroll
+            for (int c = 0; c < Geo::C; ++c) {
+#pragma unroll
+                for (int e = 0; e < 8; ++e) v[c][e] *= inv_sqrt_d;
+                store8_stream(dx + row * Geo::D + (c * Geo::G + t) * 8, v[c]);
+            }
+        }
+    }
+
+    // fold the R row groups of this CTA in a fixed order, then publish
+    float* out = partials + static_cast<size_t>(blockIdx.x) * 2 * Geo::D;
+#pragma unroll
+    for (int which = 0; which < 2; ++which) {
+        __syncthreads();
+#pragma unroll
+        for (int c = 0; c < Geo::C; ++c) {
+            float4* dst = reinterpret_cast<float4*>(srow + (c * Geo::G + t) * 8);
+            const float (&src)[8] = which == 0 ? da_acc[c] : db_acc[c];
+            dst[0] = make_float4(src[0], src[1], src[2], src[3]);
+            dst[1] = make_float4(src[4], src[5], src[6], src[7]);
+        }
+        __syncthreads();
+        for (int j = threadIdx.x; j < Geo::D; j += Geo::THREADS) {
+            float s = 0.0f;
+#pragma unroll
+            for (int r = 0; r < Geo::R; ++r) s += smem[r * Geo::D + j];
+            out[which * Geo::D + j] = s;
+        }
+    }
+}
+
+// ---- second pass: da[j] = inv_sqrt_d * sum_p partials[p][0][j], db[j] likewise --
+__global__ void __launch_bounds__(256)
+dadb_finalize_kernel(const float* __restrict__ partials, int nparts, int d, float inv_sqrt_d,
+                     float* __restrict__ da, float* __restrict__ db) {
+    const int j = blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= 2 * d) return;
+    const int which = j / d;
+    const int col = j - which * d;
+    const float* src = partials + static_cast<size_t>(which) * d + col;
+    const size_t stride = static_cast<size_t>(2) * d;
+    float s0 = 0.0f, s1 = 0.0f, s2 = 0.0f, s3 = 0.0f;
+    int p = 0;
+    for (; p + 4 <= nparts; p += 4) {
+        s0 += src[(p + 0) * stride];
+        s1 += src[(p + 1) * stride];
+        s2 += src[(p + 2) * stride];
+        s3 += src[(p + 3) * stride];
+    }
+    for (; p < nparts; ++p) s0 += src[p * stride];
+    const float s = (s0 + s1) + (s2 + s3);
+    if (which == 0) da[col] = s * inv_sqrt_d; else db[col] = s;
+}
+
+// ---- bandwidth yardstick: copy rows with the forward pass's access pattern ----
+__global__ void __launch_bounds__(256)
+copy_rows_kernel(const uint4* src, uint4* dst, long long n16) {
+    const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
+    for (long long i = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; i < n16; i += stride)
+        __stcs(dst + i, __ldcs(src + i));
+}
+
+}  // namespace wht

@@ -1,0 +1,291 @@
+"""CUDA path vs the fp64 oracle, element by element, through the C ABI (ctypes binding).
+
+Tolerances (written out in tests/helpers.py):
+  fp32 storage : max_j |err| <= 1e-5 * ||transform input row||_2      per row
+  bf16 storage : max_j |err| <= 1e-2 * max_j |reference row|           per row
+  da, db       : max_j |err| <= 1e-4 * max_j |reference|               per vector
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from helpers import assert_grad_vec, assert_rows_bf16, assert_rows_fp32, to_f64
+from paper_2603_08343_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+VARIANTS = [1, 2]  # 1 = butterfly family, 2 = tensor-core assisted (falls back to 1 where unsupported)
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2603_08343_b200 import build
+    build.build()
+    from paper_2603_08343_b200 import binding
+    yield binding
+    binding.wht_affine_set_variant(0)
+
+
+def _check_fwd(w, y_gpu, x_cpu, a_cpu, b_cpu, what):
+    ref = oracle.wht_affine_fwd(to_f64(x_cpu), to_f64(a_cpu), to_f64(b_cpu))
+    got = to_f64(y_gpu)
+    if w.dtype == wl.WHT_F32:
+        return assert_rows_fp32(got, ref, to_f64(x_cpu), what)
+    return assert_rows_bf16(got, ref, what)
+
+
+def _check_bwd(w, dx_gpu, da_gpu, db_gpu, dy_cpu, x_cpu, a_cpu, what):
+    dy64, x64, a64 = to_f64(dy_cpu), to_f64(x_cpu), to_f64(a_cpu)
+    dx, da, db = oracle.wht_affine_bwd(dy64, x64, a64)
+    got = to_f64(dx_gpu)
+    if w.dtype == wl.WHT_F32:
+        assert_rows_fp32(got, dx, a64[None, :] * dy64, what + " dx")
+    else:
+        assert_rows_bf16(got, dx, what + " dx")
+    assert_grad_vec(to_f64(da_gpu), da, what + " da")
+    assert_grad_vec(to_f64(db_gpu), db, what + " db")
+
+
+def _run_case(B, w, variant, decode=False, bwd=True):
+    B.wht_affine_set_variant(variant)
+    x = wl.gen_full(w, "x")
+    a, b = wl.gen_params(w)
+    xd, ad, bd = x.cuda(), a.cuda(), b.cuda()
+    y = B.forward(xd, ad, bd, decode=decode)
+    torch.cuda.synchronize()
+    _check_fwd(w, y.cpu(), x, a, b, f"{w.name} T={w.T} d={w.d} v{variant} fwd")
+    if bwd:
+        dy = wl.gen_full(w, "dy")
+        dx, da, db = B.backward(dy.cuda(), xd, ad)
+        torch.cuda.synchronize()
+        _check_bwd(w, dx.cpu(), da.cpu(), db.cpu(), dy, x, a, f"{w.name} T={w.T} d={w.d} v{variant} bwd")
+
+
+# ------------------------------------------------------------------ configs[0]: Tiny
+
+@pytest.mark.parametrize("variant", VARIANTS)
+def test_tiny_fwd_bwd(B, variant):
+    _run_case(B, wl.CONFIGS["tiny"], variant)
+
+
+# ------------------------------------------------------------------ every supported d, every dtype, ragged T
+
+@pytest.mark.parametrize("variant", VARIANTS)
+@pytest.mark.parametrize("dtype", [wl.WHT_F32, wl.WHT_BF16, wl.WHT_BF16_PF32])
+@pytest.mark.parametrize("logd", list(range(3, 14)))
+def test_all_sizes_ragged_rows(B, logd, dtype, variant):
+    d = 1 << logd
+    # row counts that leave a ragged last tile for every rows-per-CTA setting, over several tiles
+    T = 1031 if d <= 64 else (257 if d <= 1024 else 37)
+    w = wl.Workload("sweep", T, d, dtype, "normal", 100 + logd, True, "")
+    _run_case(B, w, variant)
+
+
+@pytest.mark.parametrize("dtype", [wl.WHT_F32, wl.WHT_BF16_PF32])
+def test_d16384(B, dtype):
+    w = wl.Workload("sweep", 5, 16384, dtype, "normal", 77, True, "")
+    _run_case(B, w, 0)
+
+
+@pytest.mark.parametrize("T", [1, 2, 3, 7, 8, 9, 255, 256, 300])
+def test_row_count_tails(B, T):
+    for d, dtype in [(256, wl.WHT_F32), (1024, wl.WHT_BF16), (2048, wl.WHT_BF16_PF32)]:
+        w = wl.Workload("tails", T, d, dtype, "normal", 200 + T, True, "")
+        for variant in VARIANTS:
+            _run_case(B, w, variant)
+
+
+# ------------------------------------------------------------------ configs[1]: Prefill, every row
+
+@pytest.mark.parametrize("variant", VARIANTS)
+def test_prefill_full(B, variant):
+    _run_case(B, wl.CONFIGS["prefill"], variant, bwd=False)
+
+
+# ------------------------------------------------------------------ configs[2]: Decode
+
+@pytest.mark.parametrize("variant", VARIANTS)
+@pytest.mark.parametrize("T", wl.DECODE_T)
+def test_decode(B, T, variant):
+    w = wl.CONFIGS["decode"].with_rows(T)
+    _run_case(B, w, variant, decode=True, bwd=False)
+
+
+def test_decode_equals_fwd_bitwise(B):
+    B.wht_affine_set_variant(0)
+    w = wl.CONFIGS["decode"].with_rows(64)
+    x = wl.gen_full(w, "x").cuda()
+    a, b = (t.cuda() for t in wl.gen_params(w))
+    y1 = B.forward(x, a, b, decode=True)
+    y2 = B.forward(x, a, b, decode=False)
+    torch.cuda.synchronize()
+    # both run fp32 accumulation over the same 4096 terms; orders may differ, the rounding target not
+    assert_rows_bf16(to_f64(y1.cpu()), to_f64(y2.cpu()), "decode vs fwd")
+
+
+# ------------------------------------------------------------------ configs[3], [4]: full size, sampled
+
+def _sample_rows(T, n, seed):
+    rng = np.random.default_rng(seed)
+    rows = set(range(64)) | set(range(T - 64, T)) | set(rng.integers(0, T, n).tolist())
+    return np.array(sorted(rows))
+
+
+def _full_size_case(B, w, n_rows, n_cols, variant):
+    B.wht_affine_set_variant(variant)
+    a, b = wl.gen_params(w)
+    ad, bd = a.cuda(), b.cuda()
+    x = wl.gen_full(w, "x", out=torch.empty(w.T, w.d, dtype=w.io_torch_dtype).pin_memory(), threads=32)
+    dy = wl.gen_full(w, "dy", out=torch.empty(w.T, w.d, dtype=w.io_torch_dtype).pin_memory(), threads=32)
+    xd, dyd = x.cuda(), dy.cuda()
+    y = B.forward(xd, ad, bd)
+    dx, da, db = B.backward(dyd, xd, ad)
+    torch.cuda.synchronize()
+    rows = _sample_rows(w.T, n_rows, w.seed)
+    ridx = torch.from_numpy(rows)
+    xs, dys = x[ridx], dy[ridx]
+    ys, dxs = y[ridx.cuda()].cpu(), dx[ridx.cuda()].cpu()
+    a64 = to_f64(a)
+    ref_y = oracle.wht_affine_fwd(to_f64(xs), a64, to_f64(b))
+    assert_rows_bf16(to_f64(ys), ref_y, f"{w.name} fwd sampled rows")
+    ref_dx, _, _ = oracle.wht_affine_bwd(to_f64(dys), to_f64(xs), a64)
+    assert_rows_bf16(to_f64(dxs), ref_dx, f"{w.name} dx sampled rows")
+    # da, db need every row: the oracle's column form, summed over row blocks
+    rng = np.random.default_rng(w.seed + 1)
+    cols = np.array(sorted(set([0, 1, w.d // 2, w.d - 1]) | set(rng.integers(0, w.d, n_cols).tolist())))
+    da_ref = np.zeros(cols.size)
+    db_ref = np.zeros(cols.size)
+    blk = 8192
+    for r0 in range(0, w.T, blk):
+        pa, pb = oracle.da_db_columns(to_f64(dy[r0:r0 + blk]), to_f64(x[r0:r0 + blk]), cols)
+        da_ref += pa
+        db_ref += pb
+    da_got = to_f64(da.cpu())[cols]
+    db_got = to_f64(db.cpu())[cols]
+    # the bound is 1e-4 * max|g_ref| over the vector; the sampled columns give a lower
+    # estimate of that maximum, which only makes the check stricter
+    assert_grad_vec(da_got, da_ref, f"{w.name} da sampled columns")
+    assert_grad_vec(db_got, db_ref, f"{w.name} db sampled columns")
+    # db over ALL columns against plain column sums in fp64 (cheap at any size)
+    db_all = np.zeros(w.d)
+    for r0 in range(0, w.T, blk):
+        db_all += to_f64(dy[r0:r0 + blk]).sum(axis=0)
+    assert_grad_vec(to_f64(db.cpu()), db_all, f"{w.name} db all columns")
+
+
+@pytest.mark.parametrize("variant", VARIANTS)
+def test_training_full_size(B, variant):
+    _full_size_case(B, wl.CONFIGS["training"], n_rows=1024, n_cols=96, variant=variant)
+
+
+def test_large_full_size(B):
+    _full_size_case(B, wl.CONFIGS["large"], n_rows=256, n_cols=28, variant=0)
+
+
+# ------------------------------------------------------------------ structure that needs no oracle
+
+@pytest.mark.parametrize("variant", VARIANTS)
+@pytest.mark.parametrize("d", [256, 4096, 32768])
+def test_impulse_rows_closed_form(B, d, variant):
+    # x = e_k  =>  y = a (.) (row k of H)/sqrt(d) + b with sign (-1)^popcount(k & j)
+    B.wht_affine_set_variant(variant)
+    ks = [0, 1, 5, d // 2, d - 1]
+    x = torch.zeros(len(ks), d, dtype=torch.float32)
+    for r, k in enumerate(ks):
+        x[r, k] = 1.0
+    w = wl.Workload("imp", len(ks), d, wl.WHT_F32, "normal", 9, False, "")
+    a, b = wl.gen_params(w)
+    y = B.forward(x.cuda(), a.cuda(), b.cuda()).cpu().numpy().astype(np.float64)
+    j = np.arange(d)
+    for r, k in enumerate(ks):
+        par = np.zeros(d, dtype=np.int64)
+        v = j & k
+        while np.any(v):
+            par ^= v & 1
+            v >>= 1
+        want = a.numpy().astype(np.float64) * (1 - 2 * par) / math.sqrt(d) + b.numpy().astype(np.float64)
+        assert np.max(np.abs(y[r] - want)) <= 1e-5
+
+
+@pytest.mark.parametrize("variant", VARIANTS)
+@pytest.mark.parametrize("d,dtype", [(32768, torch.float32), (8192, torch.float32), (1024, torch.float32)])
+def test_involution_and_norm(B, d, dtype, variant):
+    B.wht_affine_set_variant(variant)
+    g = torch.Generator().manual_seed(d)
+    x = torch.randn(9, d, generator=g, dtype=dtype).cuda()
+    one = torch.ones(d, dtype=dtype).cuda()
+    zero = torch.zeros(d, dtype=dtype).cuda()
+    z = B.forward(x, one, zero)
+    back = B.forward(z, one, zero)
+    torch.cuda.synchronize()
+    xn = x.double().norm(dim=1)
+    assert torch.all((z.double().norm(dim=1) - xn).abs() <= 1e-5 * xn)
+    assert torch.all((back.double() - x.double()).abs().amax(dim=1) <= 2e-5 * xn)
+
+
+@pytest.mark.parametrize("variant", VARIANTS)
+def test_in_place_and_empty(B, variant):
+    B.wht_affine_set_variant(variant)
+    for name in ("tiny", "prefill"):
+        w = wl.CONFIGS[name].with_rows(300)
+        x = wl.gen_full(w, "x").cuda()
+        a, b = (t.cuda() for t in wl.gen_params(w))
+        y = B.forward(x, a, b)
+        x2 = x.clone()
+        B.forward(x2, a, b, out=x2)
+        assert torch.equal(y, x2)
+        dy = wl.gen_full(w, "dy").cuda()
+        dx, da, db = B.backward(dy, x, a)
+        dy2 = dy.clone()
+        da2, db2 = torch.empty_like(da), torch.empty_like(db)
+        B.wht_affine_bwd(dy2, x, a, dy2, da2, db2, w.T, w.d, w.dtype)
+        assert torch.equal(dx, dy2) and torch.equal(da, da2) and torch.equal(db, db2)
+        # T == 0: forward is a no-op, backward writes zeros
+        e = torch.empty(0, w.d, dtype=x.dtype, device="cuda")
+        B.forward(e, a, b)
+        da0 = torch.full((w.d,), 3.0, device="cuda")
+        db0 = torch.full((w.d,), 3.0, device="cuda")
+        B.wht_affine_bwd(e, e, a, e, da0, db0, 0, w.d, w.dtype)
+        torch.cuda.synchronize()
+        assert torch.count_nonzero(da0) == 0 and torch.count_nonzero(db0) == 0
+
+
+@pytest.mark.parametrize("variant", VARIANTS)
+def test_bwd_reproducible_and_workspace_forms_agree(B, variant):
+    B.wht_affine_set_variant(variant)
+    w = wl.CONFIGS["training"].with_rows(5000)
+    x = wl.gen_full(w, "x").cuda()
+    dy = wl.gen_full(w, "dy").cuda()
+    a, _ = wl.gen_params(w)
+    a = a.cuda()
+    dx1, da1, db1 = B.backward(dy, x, a)
+    dx2, da2, db2 = B.backward(dy, x, a)
+    assert torch.equal(dx1, dx2) and torch.equal(da1, da2) and torch.equal(db1, db2)
+    need = B.wht_affine_bwd_workspace_bytes(w.T, w.d, w.dtype)
+    assert need > 0
+    ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+    dx3 = torch.empty_like(dx1)
+    da3, db3 = torch.empty_like(da1), torch.empty_like(db1)
+    B.wht_affine_bwd_ws(dy, x, a, dx3, da3, db3, w.T, w.d, w.dtype, ws)
+    assert torch.equal(dx1, dx3) and torch.equal(da1, da3) and torch.equal(db1, db3)
+    small = torch.empty(max(need // 2, 16), dtype=torch.uint8, device="cuda")
+    with pytest.raises(B.WhtError) as err:
+        B.wht_affine_bwd_ws(dy, x, a, dx3, da3, db3, w.T, w.d, w.dtype, small)
+    assert err.value.status == -6
+
+
+def test_heavy_tailed_rows(B):
+    # Student-t(3) rows in bf16: single spikes dominate a row; fp32 accumulation must hold the bound
+    for variant in VARIANTS:
+        w = wl.CONFIGS["large"].with_rows(48)
+        _run_case(B, w, variant)
+
+
+def test_copy_rows(B):
+    src = torch.arange(3 * 1024, dtype=torch.float32, device="cuda").view(3, 1024)
+    dst = torch.zeros_like(src)
+    B.wht_copy_rows(src, dst, 3, 1024, wl.WHT_F32)
+    assert torch.equal(src, dst)
