@@ -8,6 +8,7 @@
 #include <mutex>
 
 #include "bfly_kernels.cuh"
+#include "mma_kernels.cuh"
 
 namespace {
 
@@ -157,14 +158,105 @@ int dispatch_bfly_bwd(int logd, const void* dy, const void* x, const void* a, vo
     return WHT_ERR_BAD_DIM;
 }
 
+
+// ------------------------------------------------------------------ tensor-core family
+template <int LOGD, int TB, int RG, typename TP>
+int launch_mma_fwd(const void* x, const void* a, const void* b, void* y, int64_t T,
+                   int dev, int sms, cudaStream_t s) {
+    using Geo = MmaGeo<LOGD, TB, RG>;
+    static int occ[kMaxDevices] = {};
+    auto kernel = mma_fwd_kernel<LOGD, TB, RG, TP>;
+    const int per_sm = resident_ctas(kernel, Geo::THREADS, Geo::SMEM_FWD, dev, occ);
+    if (per_sm <= 0) return cuda_fail(cudaGetLastError());
+    const long long tiles = ceil_div(T, RG);
+    const long long cap = static_cast<long long>(sms) * per_sm;
+    const unsigned grid = static_cast<unsigned>(tiles < cap ? tiles : cap);
+    const float rs = static_cast<float>(1.0 / sqrt(static_cast<double>(Geo::D)));
+    kernel<<<grid, Geo::THREADS, Geo::SMEM_FWD, s>>>(
+        static_cast<const __nv_bfloat16*>(x), static_cast<const TP*>(a), static_cast<const TP*>(b),
+        static_cast<__nv_bfloat16*>(y), static_cast<long long>(T), rs);
+    WHT_CUDA_TRY(cudaGetLastError());
+    return WHT_OK;
+}
+
+template <int LOGD, int TB, int RG, typename TP>
+int launch_mma_bwd(const void* dy, const void* x, const void* a, void* dx, float* da, float* db,
+                   int64_t T, void* ws, size_t ws_bytes, bool query_only, size_t* need,
+                   int dev, int sms, cudaStream_t s) {
+    using Geo = MmaGeo<LOGD, TB, RG>;
+    static int occ[kMaxDevices] = {};
+    auto kernel = mma_bwd_kernel<LOGD, TB, RG, TP>;
+    const int per_sm = resident_ctas(kernel, Geo::THREADS, Geo::SMEM_BWD, dev, occ);
+    if (per_sm <= 0) return cuda_fail(cudaGetLastError());
+    const long long tiles = ceil_div(T, RG);
+    const long long cap = static_cast<long long>(sms) * per_sm;
+    const int grid = static_cast<int>(tiles < cap ? tiles : cap);
+    *need = static_cast<size_t>(grid) * 2 * Geo::D * sizeof(float);
+    if (query_only) return WHT_OK;
+    if (*need > 0 && (ws == nullptr || ws_bytes < *need)) return WHT_ERR_WORKSPACE;
+    const float rs = static_cast<float>(1.0 / sqrt(static_cast<double>(Geo::D)));
+    if (grid > 0) {
+        kernel<<<grid, Geo::THREADS, Geo::SMEM_BWD, s>>>(
+            static_cast<const __nv_bfloat16*>(dy), static_cast<const __nv_bfloat16*>(x),
+            static_cast<const TP*>(a), static_cast<__nv_bfloat16*>(dx), static_cast<float*>(ws),
+            static_cast<long long>(T), rs);
+        WHT_CUDA_TRY(cudaGetLastError());
+    }
+    dadb_finalize_kernel<<<(2 * Geo::D + 255) / 256, 256, 0, s>>>(
+        static_cast<const float*>(ws), grid, Geo::D, rs, da, db);
+    WHT_CUDA_TRY(cudaGetLastError());
+    return WHT_OK;
+}
+
+// Row splits (LOGD, TB, RG) of the tensor-core family.  `wide` spreads a row over
+// more warps (lower latency per row, used for decode and as tuning alternative).
+template <typename TP>
+int dispatch_mma_fwd(int logd, bool wide, const void* x, const void* a, const void* b, void* y,
+                     int64_t T, int dev, int sms, cudaStream_t s) {
+    switch (logd) {
+        case 9: return launch_mma_fwd<9, 1, 4, TP>(x, a, b, y, T, dev, sms, s);
+        case 10: return wide ? launch_mma_fwd<10, 1, 2, TP>(x, a, b, y, T, dev, sms, s)
+                             : launch_mma_fwd<10, 2, 4, TP>(x, a, b, y, T, dev, sms, s);
+        case 11: return wide ? launch_mma_fwd<11, 2, 2, TP>(x, a, b, y, T, dev, sms, s)
+                             : launch_mma_fwd<11, 3, 4, TP>(x, a, b, y, T, dev, sms, s);
+        case 12: return wide ? launch_mma_fwd<12, 2, 1, TP>(x, a, b, y, T, dev, sms, s)
+                             : launch_mma_fwd<12, 3, 2, TP>(x, a, b, y, T, dev, sms, s);
+        case 13: return launch_mma_fwd<13, 3, 1, TP>(x, a, b, y, T, dev, sms, s);
+    }
+    return WHT_ERR_BAD_DIM;
+}
+
+template <typename TP>
+int dispatch_mma_bwd(int logd, bool wide, const void* dy, const void* x, const void* a, void* dx,
+                     float* da, float* db, int64_t T, void* ws, size_t ws_bytes, bool query_only,
+                     size_t* need, int dev, int sms, cudaStream_t s) {
+#define WHT_BWD_ARGS dy, x, a, dx, da, db, T, ws, ws_bytes, query_only, need, dev, sms, s
+    switch (logd) {
+        case 9: return launch_mma_bwd<9, 1, 8, TP>(WHT_BWD_ARGS);
+        case 10: return wide ? launch_mma_bwd<10, 1, 4, TP>(WHT_BWD_ARGS) : launch_mma_bwd<10, 2, 8, TP>(WHT_BWD_ARGS);
+        case 11: return wide ? launch_mma_bwd<11, 2, 4, TP>(WHT_BWD_ARGS) : launch_mma_bwd<11, 3, 4, TP>(WHT_BWD_ARGS);
+        case 12: return wide ? launch_mma_bwd<12, 2, 2, TP>(WHT_BWD_ARGS) : launch_mma_bwd<12, 3, 2, TP>(WHT_BWD_ARGS);
+        case 13: return launch_mma_bwd<13, 3, 1, TP>(WHT_BWD_ARGS);
+    }
+#undef WHT_BWD_ARGS
+    return WHT_ERR_BAD_DIM;
+}
+
+bool mma_supported(int logd, int dtype) { return dtype != WHT_F32 && logd >= 9 && logd <= 13; }
+
 // ------------------------------------------------------------------ selection
 int run_fwd(const void* x, const void* a, const void* b, void* y, int64_t T, int32_t d, int dtype,
             cudaStream_t s, bool decode) {
-    (void)decode;
     int dev = 0, sms = 0;
     int rc = current_device(&dev, &sms);
     if (rc != WHT_OK) return rc;
     const int logd = log2_of(d);
+    if (g_variant != 1 && mma_supported(logd, dtype)) {
+        const bool wide = decode || g_variant == 3;
+        return dtype == WHT_BF16
+                   ? dispatch_mma_fwd<__nv_bfloat16>(logd, wide, x, a, b, y, T, dev, sms, s)
+                   : dispatch_mma_fwd<float>(logd, wide, x, a, b, y, T, dev, sms, s);
+    }
     switch (dtype) {
         case WHT_F32: return dispatch_bfly_fwd<float, float>(logd, x, a, b, y, T, dev, sms, s);
         case WHT_BF16: return dispatch_bfly_fwd<__nv_bfloat16, __nv_bfloat16>(logd, x, a, b, y, T, dev, sms, s);
@@ -179,6 +271,12 @@ int run_bwd(const void* dy, const void* x, const void* a, void* dx, float* da, f
     int rc = current_device(&dev, &sms);
     if (rc != WHT_OK) return rc;
     const int logd = log2_of(d);
+    if (g_variant != 1 && mma_supported(logd, dtype)) {
+        const bool wide = g_variant != 3;
+        return dtype == WHT_BF16
+                   ? dispatch_mma_bwd<__nv_bfloat16>(logd, wide, dy, x, a, dx, da, db, T, ws, ws_bytes, query_only, need, dev, sms, s)
+                   : dispatch_mma_bwd<float>(logd, wide, dy, x, a, dx, da, db, T, ws, ws_bytes, query_only, need, dev, sms, s);
+    }
     switch (dtype) {
         case WHT_F32:
             return dispatch_bfly_bwd<float, float>(logd, dy, x, a, dx, da, db, T, ws, ws_bytes, query_only, need, dev, sms, s);
@@ -290,7 +388,7 @@ int wht_affine_bwd(const void* dy, const void* x, const void* a, void* dx, float
 }
 
 int wht_affine_set_variant(int variant) {
-    if (variant < 0 || variant > 2) return WHT_ERR_BAD_VARIANT;
+    if (variant < 0 || variant > 3) return WHT_ERR_BAD_VARIANT;
     g_variant = variant;
     return WHT_OK;
 }
