@@ -54,7 +54,8 @@ typedef enum {
     WHT_ERR_MISALIGNED = -5,  /* a pointer is not 16-byte aligned                    */
     WHT_ERR_WORKSPACE = -6,   /* workspace missing, too small, or allocation failed  */
     WHT_ERR_CUDA = -7,        /* a CUDA runtime call failed; see wht_affine_last_cuda_error */
-    WHT_ERR_BAD_VARIANT = -8  /* unknown kernel variant id                           */
+    WHT_ERR_BAD_VARIANT = -8, /* unknown kernel variant id                           */
+    WHT_ERR_DEVICE_WAIT = -9  /* a kernel's bounded wait for an async copy expired   */
 } wht_status;
 
 /*
@@ -111,8 +112,12 @@ size_t wht_affine_bwd_workspace_bytes(int64_t T, int32_t d, int dtype);
 
 /*
  * Kernel family used by the three compute calls (for A/B measurements):
- *   0 = automatic (default), 1 = butterfly (registers + warp shuffles + shared
- *   memory), 2 = tensor-core assisted (H_16 factors through mma, bf16 storage only).
+ *   0 = automatic (default): tensor-core assisted kernels for bf16 rows with
+ *       512 <= d <= 8192 (rows streamed through a shared-memory ring when there
+ *       are many, loaded directly when there are few), butterfly otherwise;
+ *   1 = butterfly (registers + warp shuffles + shared memory), every d and dtype;
+ *   2 = tensor-core assisted with direct row loads;
+ *   3 = tensor-core assisted with streamed rows.
  * A variant that does not support the requested (d, dtype) falls back to 1.
  * Process-wide; not meant to be changed while calls are in flight.
  */
@@ -125,6 +130,16 @@ int wht_affine_get_variant(void);
  * the benchmark to report a practical copy ceiling next to the kernels.
  */
 int wht_copy_rows(const void* src, void* dst, int64_t T, int32_t d, int dtype, void* stream);
+
+/*
+ * The streamed kernels wait for their async copies with a bound; a wait that
+ * expires does not hang or trap, it sets a flag on the device and the launch's
+ * results are invalid.  This call synchronises with the current device's work
+ * (it copies the flag back), returns WHT_ERR_DEVICE_WAIT if the flag was set
+ * since the last query and clears it, else WHT_OK.  Never expected in normal
+ * operation; meant for tests and for debugging after a suspicious result.
+ */
+int wht_affine_device_status(void);
 
 /* cudaError_t of the most recent failing CUDA call on this thread (0 if none). */
 int wht_affine_last_cuda_error(void);

@@ -20,7 +20,7 @@ LIB_PATH = os.path.join(_HERE, "libwht_affine.so")
 EXPORTS = (
     "wht_affine_fwd", "wht_affine_fwd_decode", "wht_affine_bwd", "wht_affine_bwd_ws",
     "wht_affine_bwd_workspace_bytes", "wht_affine_set_variant", "wht_affine_get_variant",
-    "wht_copy_rows", "wht_affine_last_cuda_error", "wht_affine_status_string",
+    "wht_copy_rows", "wht_affine_device_status", "wht_affine_last_cuda_error", "wht_affine_status_string",
     "wht_affine_shutdown",
 )
 
@@ -49,6 +49,7 @@ def _load() -> ctypes.CDLL:
     lib.wht_affine_set_variant.argtypes = [ci]
     lib.wht_affine_get_variant.argtypes = []
     lib.wht_copy_rows.argtypes = [vp, vp, i64, i32, ci, vp]
+    lib.wht_affine_device_status.argtypes = []
     lib.wht_affine_last_cuda_error.argtypes = []
     lib.wht_affine_status_string.argtypes = [ci]
     lib.wht_affine_status_string.restype = ctypes.c_char_p
@@ -130,6 +131,11 @@ def wht_affine_get_variant() -> int:
 def wht_copy_rows(src, dst, T: int, d: int, dtype: int, stream=None) -> None:
     _require_cuda(src, dst)
     _check(_lib.wht_copy_rows(_ptr(src), _ptr(dst), T, d, dtype, _stream(stream)), "wht_copy_rows")
+
+
+def wht_affine_device_status() -> None:
+    """Synchronises and raises WhtError if a kernel's bounded wait expired since the last query."""
+    _check(_lib.wht_affine_device_status(), "wht_affine_device_status")
 
 
 def wht_affine_shutdown() -> None:

@@ -32,17 +32,36 @@
 //           with the top WB chunk bits through shared memory (fp32, conflict-free
 //           128-bit accesses, one named barrier per exchange, double-buffered),
 //           then finished with fp32 butterflies in registers.
+//
+// All fp32 arithmetic outside the mma is done on register pairs with the packed
+// f32x2 add / fma of sm_100, which halves its issue slots.
 #pragma once
 #include "wht_common.cuh"
 
 namespace wht {
 
-__device__ __forceinline__ void mma_bf16_m16n8k16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0,
+using F2 = float2;
+
+__device__ __forceinline__ F2 f2(float x, float y) { return make_float2(x, y); }
+__device__ __forceinline__ F2 add2(F2 a, F2 b) { return __fadd2_rn(a, b); }
+__device__ __forceinline__ F2 sub2(F2 a, F2 b) { return __ffma2_rn(b, f2(-1.0f, -1.0f), a); }  // a - b, exact product
+__device__ __forceinline__ F2 mul2(F2 a, F2 b) { return __fmul2_rn(a, b); }
+__device__ __forceinline__ F2 fma2(F2 a, F2 b, F2 c) { return __ffma2_rn(a, b, c); }
+__device__ __forceinline__ void bfly2(F2& lo, F2& hi) {
+    const F2 s = add2(lo, hi);
+    hi = sub2(lo, hi);
+    lo = s;
+}
+__device__ __forceinline__ F2 unpack_bf16x2(uint32_t u) { return f2(bf16lo_to_f32(u), bf16hi_to_f32(u)); }
+__device__ __forceinline__ uint32_t pack_bf16x2(F2 v) { return pack_bf16x2(v.x, v.y); }
+
+// D(16x8, fp32) += A(16x16, bf16) * B(16x8, bf16); d01 = (c0, c1), d23 = (c2, c3)
+__device__ __forceinline__ void mma_bf16_m16n8k16(F2& d01, F2& d23, const uint32_t (&a)[4], uint32_t b0,
                                                   uint32_t b1) {
     asm volatile(
         "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
         "{%0,%1,%2,%3};"
-        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "+f"(d01.x), "+f"(d01.y), "+f"(d23.x), "+f"(d23.y)
         : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
@@ -56,10 +75,11 @@ __device__ __forceinline__ void make_h16_fragment(uint32_t (&a)[4], int lane) {
     a[3] = s(g + 8, 2 * q + 8) | (s(g + 8, 2 * q + 9) << 16);
 }
 
-// fp32 pair -> bf16x2 hi (round to nearest) and bf16x2 lo (rounded remainder)
-__device__ __forceinline__ void split_hi_lo(float v0, float v1, uint32_t& hi, uint32_t& lo) {
-    hi = pack_bf16x2(v0, v1);
-    lo = pack_bf16x2(v0 - bf16lo_to_f32(hi), v1 - bf16hi_to_f32(hi));
+// fp32 pair -> bf16x2 hi (round to nearest) and bf16x2 lo (rounded remainder):
+// hi + lo carries the pair to a relative error of 2^-17.
+__device__ __forceinline__ void split_hi_lo(F2 v, uint32_t& hi, uint32_t& lo) {
+    hi = pack_bf16x2(v);
+    lo = pack_bf16x2(sub2(v, unpack_bf16x2(hi)));
 }
 
 __device__ __forceinline__ void named_barrier(int id, int threads) {
@@ -96,50 +116,47 @@ __device__ __forceinline__ int chunk_of(int w, int idx) {
     }
 }
 
+// Thread-local views of a row slice:
+//   m[t][h][p]  (after pass 1)  pair r = (x, y) <-> index bit 5, p <-> bit 1, h <-> bit 2
+//   v[t][j]     (load layout)   pair (x, y) = elements 2j, 2j+1 of chunk slot t
 template <class Geo>
 struct MmaXform {
     static constexpr int NT = Geo::NT;
 
-    // pass 1 on stored bf16: m[t][h][2p + r] <- bits {0,3,4,1} transformed
-    static __device__ __forceinline__ void pass1_raw(const uint4 (&raw)[NT], float (&m)[NT][2][4],
+    // pass 1 on stored bf16 (bits {0,3,4,1})
+    static __device__ __forceinline__ void pass1_raw(const uint4 (&raw)[NT], F2 (&m)[NT][2][2],
                                                      const uint32_t (&hf)[4]) {
 #pragma unroll
         for (int t = 0; t < NT; ++t) {
-#pragma unroll
-            for (int i = 0; i < 4; ++i) { m[t][0][i] = 0.0f; m[t][1][i] = 0.0f; }
-            mma_bf16_m16n8k16(m[t][0], hf, raw[t].x, raw[t].y);
-            mma_bf16_m16n8k16(m[t][1], hf, raw[t].z, raw[t].w);
+            m[t][0][0] = m[t][0][1] = m[t][1][0] = m[t][1][1] = f2(0.0f, 0.0f);
+            mma_bf16_m16n8k16(m[t][0][0], m[t][0][1], hf, raw[t].x, raw[t].y);
+            mma_bf16_m16n8k16(m[t][1][0], m[t][1][1], hf, raw[t].z, raw[t].w);
         }
     }
 
-    // pass 1 on fp32 values in load layout v[t][e] (hi/lo split operands)
-    static __device__ __forceinline__ void pass1_f32(const float (&v)[NT][8], float (&m)[NT][2][4],
+    // pass 1 on fp32 values in load layout (hi/lo split operands)
+    static __device__ __forceinline__ void pass1_f32(const F2 (&v)[NT][4], F2 (&m)[NT][2][2],
                                                      const uint32_t (&hf)[4]) {
 #pragma unroll
         for (int t = 0; t < NT; ++t) {
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
                 uint32_t b0h, b0l, b1h, b1l;
-                split_hi_lo(v[t][4 * h + 0], v[t][4 * h + 1], b0h, b0l);
-                split_hi_lo(v[t][4 * h + 2], v[t][4 * h + 3], b1h, b1l);
-#pragma unroll
-                for (int i = 0; i < 4; ++i) m[t][h][i] = 0.0f;
-                mma_bf16_m16n8k16(m[t][h], hf, b0h, b1h);
-                mma_bf16_m16n8k16(m[t][h], hf, b0l, b1l);
+                split_hi_lo(v[t][2 * h + 0], b0h, b0l);
+                split_hi_lo(v[t][2 * h + 1], b1h, b1l);
+                m[t][h][0] = m[t][h][1] = f2(0.0f, 0.0f);
+                mma_bf16_m16n8k16(m[t][h][0], m[t][h][1], hf, b0h, b1h);
+                mma_bf16_m16n8k16(m[t][h][0], m[t][h][1], hf, b0l, b1l);
             }
         }
     }
 
     // fp32 butterflies on bit 2 (h) and on chunk-slot bits 1..TB-1
-    static __device__ __forceinline__ void mid_stages(float (&m)[NT][2][4]) {
+    static __device__ __forceinline__ void mid_stages(F2 (&m)[NT][2][2]) {
 #pragma unroll
         for (int t = 0; t < NT; ++t) {
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const float lo = m[t][0][i], hi = m[t][1][i];
-                m[t][0][i] = lo + hi;
-                m[t][1][i] = lo - hi;
-            }
+            bfly2(m[t][0][0], m[t][1][0]);
+            bfly2(m[t][0][1], m[t][1][1]);
         }
 #pragma unroll
         for (int bit = 2; bit < NT; bit <<= 1) {
@@ -148,20 +165,16 @@ struct MmaXform {
                 if ((t & bit) == 0) {
 #pragma unroll
                     for (int h = 0; h < 2; ++h) {
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            const float lo = m[t][h][i], hi = m[t + bit][h][i];
-                            m[t][h][i] = lo + hi;
-                            m[t + bit][h][i] = lo - hi;
-                        }
+                        bfly2(m[t][h][0], m[t + bit][h][0]);
+                        bfly2(m[t][h][1], m[t + bit][h][1]);
                     }
                 }
             }
         }
     }
 
-    // pass 2 on bits {5,6,7} and chunk-slot bit 0; result v[t][e] is in load layout
-    static __device__ __forceinline__ void pass2(const float (&m)[NT][2][4], float (&v)[NT][8],
+    // pass 2 on bits {5,6,7} and chunk-slot bit 0; the result is in load layout
+    static __device__ __forceinline__ void pass2(const F2 (&m)[NT][2][2], F2 (&v)[NT][4],
                                                  const uint32_t (&hf)[4]) {
 #pragma unroll
         for (int u = 0; u < NT / 2; ++u) {
@@ -170,15 +183,13 @@ struct MmaXform {
 #pragma unroll
                 for (int p = 0; p < 2; ++p) {
                     uint32_t b0h, b0l, b1h, b1l;
-                    split_hi_lo(m[2 * u][h][2 * p], m[2 * u][h][2 * p + 1], b0h, b0l);
-                    split_hi_lo(m[2 * u + 1][h][2 * p], m[2 * u + 1][h][2 * p + 1], b1h, b1l);
-                    float d[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-                    mma_bf16_m16n8k16(d, hf, b0h, b1h);
-                    mma_bf16_m16n8k16(d, hf, b0l, b1l);
-                    v[2 * u][4 * h + 2 * p + 0] = d[0];
-                    v[2 * u][4 * h + 2 * p + 1] = d[1];
-                    v[2 * u + 1][4 * h + 2 * p + 0] = d[2];
-                    v[2 * u + 1][4 * h + 2 * p + 1] = d[3];
+                    split_hi_lo(m[2 * u][h][p], b0h, b0l);
+                    split_hi_lo(m[2 * u + 1][h][p], b1h, b1l);
+                    F2 d01 = f2(0.0f, 0.0f), d23 = f2(0.0f, 0.0f);
+                    mma_bf16_m16n8k16(d01, d23, hf, b0h, b1h);
+                    mma_bf16_m16n8k16(d01, d23, hf, b0l, b1l);
+                    v[2 * u][2 * h + p] = d01;
+                    v[2 * u + 1][2 * h + p] = d23;
                 }
             }
         }
@@ -187,15 +198,15 @@ struct MmaXform {
     // Swap the warp bits with the top WB chunk-slot bits through shared memory
     // (layout A -> B when FROM_A, else B -> A) and finish those stages in registers.
     template <bool FROM_A>
-    static __device__ __forceinline__ void exchange_and_top(float (&v)[NT][8], float* xbuf, int w, int lane,
+    static __device__ __forceinline__ void exchange_and_top(F2 (&v)[NT][4], float* xbuf, int w, int lane,
                                                             int barrier_id) {
         if constexpr (Geo::WB > 0) {
 #pragma unroll
             for (int idx = 0; idx < NT; ++idx) {
                 const int c = chunk_of<Geo, !FROM_A>(w, idx);
                 float4* p = reinterpret_cast<float4*>(xbuf + c * 256 + lane * 4);
-                p[0] = make_float4(v[idx][0], v[idx][1], v[idx][2], v[idx][3]);
-                p[32] = make_float4(v[idx][4], v[idx][5], v[idx][6], v[idx][7]);
+                p[0] = make_float4(v[idx][0].x, v[idx][0].y, v[idx][1].x, v[idx][1].y);
+                p[32] = make_float4(v[idx][2].x, v[idx][2].y, v[idx][3].x, v[idx][3].y);
             }
             named_barrier(barrier_id, Geo::GROUP_THREADS);
 #pragma unroll
@@ -203,8 +214,8 @@ struct MmaXform {
                 const int c = chunk_of<Geo, FROM_A>(w, idx);
                 const float4* p = reinterpret_cast<const float4*>(xbuf + c * 256 + lane * 4);
                 const float4 q0 = p[0], q1 = p[32];
-                v[idx][0] = q0.x; v[idx][1] = q0.y; v[idx][2] = q0.z; v[idx][3] = q0.w;
-                v[idx][4] = q1.x; v[idx][5] = q1.y; v[idx][6] = q1.z; v[idx][7] = q1.w;
+                v[idx][0] = f2(q0.x, q0.y); v[idx][1] = f2(q0.z, q0.w);
+                v[idx][2] = f2(q1.x, q1.y); v[idx][3] = f2(q1.z, q1.w);
             }
 #pragma unroll
             for (int bit = Geo::NREST; bit < NT; bit <<= 1) {
@@ -212,11 +223,7 @@ struct MmaXform {
                 for (int idx = 0; idx < NT; ++idx) {
                     if ((idx & bit) == 0) {
 #pragma unroll
-                        for (int e = 0; e < 8; ++e) {
-                            const float lo = v[idx][e], hi = v[idx + bit][e];
-                            v[idx][e] = lo + hi;
-                            v[idx + bit][e] = lo - hi;
-                        }
+                        for (int j = 0; j < 4; ++j) bfly2(v[idx][j], v[idx + bit][j]);
                     }
                 }
             }
@@ -224,18 +231,86 @@ struct MmaXform {
     }
 };
 
-// 8 parameters at a column offset, widened to fp32
-__device__ __forceinline__ void load_params8(const float* __restrict__ p, float (&v)[8]) { load8(p, v); }
-__device__ __forceinline__ void load_params8(const __nv_bfloat16* __restrict__ p, float (&v)[8]) { load8(p, v); }
-
-__device__ __forceinline__ void unpack8(const uint4& q, float (&v)[8]) {
-    v[0] = bf16lo_to_f32(q.x); v[1] = bf16hi_to_f32(q.x);
-    v[2] = bf16lo_to_f32(q.y); v[3] = bf16hi_to_f32(q.y);
-    v[4] = bf16lo_to_f32(q.z); v[5] = bf16hi_to_f32(q.z);
-    v[6] = bf16lo_to_f32(q.w); v[7] = bf16hi_to_f32(q.w);
+// 8 parameters at a column offset in global memory, widened to fp32 pairs
+__device__ __forceinline__ void load_params8(const float* __restrict__ p, F2 (&v)[4]) {
+    const float4 q0 = __ldg(reinterpret_cast<const float4*>(p));
+    const float4 q1 = __ldg(reinterpret_cast<const float4*>(p) + 1);
+    v[0] = f2(q0.x, q0.y); v[1] = f2(q0.z, q0.w);
+    v[2] = f2(q1.x, q1.y); v[3] = f2(q1.z, q1.w);
+}
+__device__ __forceinline__ void load_params8(const __nv_bfloat16* __restrict__ p, F2 (&v)[4]) {
+    const uint4 q = __ldg(reinterpret_cast<const uint4*>(p));
+    v[0] = unpack_bf16x2(q.x); v[1] = unpack_bf16x2(q.y);
+    v[2] = unpack_bf16x2(q.z); v[3] = unpack_bf16x2(q.w);
 }
 
-// ---- forward -------------------------------------------------------------------
+// In every helper below `as` is a / sqrt(d): the normalisation rides on the scale
+// vector, so the forward epilogue is one fma and the backward needs no final scale
+// (H is linear: ((a/sqrt(d)) (.) dy) H = ((a (.) dy) H)/sqrt(d)).
+
+// y chunk = as (.) v + b, rounded to bf16 and stored (128-bit, streaming)
+__device__ __forceinline__ void fwd_store_chunk(const F2 (&v)[4], const F2 (&as)[4], const F2 (&bs)[4],
+                                                uint4* dst) {
+    uint4 o;
+    o.x = pack_bf16x2(fma2(v[0], as[0], bs[0]));
+    o.y = pack_bf16x2(fma2(v[1], as[1], bs[1]));
+    o.z = pack_bf16x2(fma2(v[2], as[2], bs[2]));
+    o.w = pack_bf16x2(fma2(v[3], as[3], bs[3]));
+    __stcs(dst, o);
+}
+
+// backward, between the two transforms, one chunk: da += dy (.) u, db += dy, v <- as (.) dy
+__device__ __forceinline__ void bwd_mid_chunk(F2 (&v)[4], const uint4& rawdy, const F2 (&as)[4],
+                                              F2 (&da_acc)[4], F2 (&db_acc)[4]) {
+    const uint32_t w[4] = {rawdy.x, rawdy.y, rawdy.z, rawdy.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const F2 dyv = unpack_bf16x2(w[j]);
+        da_acc[j] = fma2(dyv, v[j], da_acc[j]);
+        db_acc[j] = add2(db_acc[j], dyv);
+        v[j] = mul2(as[j], dyv);
+    }
+}
+
+__device__ __forceinline__ void bwd_store_chunk(const F2 (&v)[4], uint4* dst) {
+    uint4 o;
+    o.x = pack_bf16x2(v[0]);
+    o.y = pack_bf16x2(v[1]);
+    o.z = pack_bf16x2(v[2]);
+    o.w = pack_bf16x2(v[3]);
+    __stcs(dst, o);
+}
+
+// Fold the RG row groups' partial sums of one CTA in a fixed order and publish them.
+// partials layout: [gridDim.x][2][D] fp32 (slot 0: sum_t dy (.) (x H) without the
+// 1/sqrt(d) factor, slot 1: sum_t dy).  `fold` is RG*D floats of shared memory.
+template <class Geo>
+__device__ __forceinline__ void bwd_publish_partials(const F2 (&da_acc)[Geo::NT][4], const F2 (&db_acc)[Geo::NT][4],
+                                                     float* fold, float* __restrict__ partials, int rg, int w,
+                                                     int lane) {
+    float* out = partials + static_cast<size_t>(blockIdx.x) * 2 * Geo::D;
+#pragma unroll
+    for (int which = 0; which < 2; ++which) {
+        __syncthreads();
+#pragma unroll
+        for (int idx = 0; idx < Geo::NT; ++idx) {
+            const int c = chunk_of<Geo, true>(w, idx);
+            float4* p = reinterpret_cast<float4*>(fold + rg * Geo::D + (c * 32 + lane) * 8);
+            const F2 (&src)[4] = which == 0 ? da_acc[idx] : db_acc[idx];
+            p[0] = make_float4(src[0].x, src[0].y, src[1].x, src[1].y);
+            p[1] = make_float4(src[2].x, src[2].y, src[3].x, src[3].y);
+        }
+        __syncthreads();
+        for (int j = threadIdx.x; j < Geo::D; j += Geo::THREADS) {
+            float s = 0.0f;
+#pragma unroll
+            for (int r = 0; r < Geo::RG; ++r) s += fold[r * Geo::D + j];
+            out[which * Geo::D + j] = s;
+        }
+    }
+}
+
+// ---- forward, rows loaded straight from global memory (few rows / decode) ----------
 template <int LOGD, int TB, int RG, typename TP>
 __global__ void __launch_bounds__(MmaGeo<LOGD, TB, RG>::THREADS)
 mma_fwd_kernel(const __nv_bfloat16* x, const TP* __restrict__ a, const TP* __restrict__ b,
@@ -251,6 +326,7 @@ mma_fwd_kernel(const __nv_bfloat16* x, const TP* __restrict__ a, const TP* __res
     float* xbuf = smem + rg * Geo::XCHG_FLOATS;
     uint32_t hf[4];
     make_h16_fragment(hf, lane);
+    const F2 rs2 = f2(inv_sqrt_d, inv_sqrt_d);
 
     int parity = 0;
     const long long stride = static_cast<long long>(gridDim.x) * RG;
@@ -259,8 +335,8 @@ mma_fwd_kernel(const __nv_bfloat16* x, const TP* __restrict__ a, const TP* __res
         uint4 raw[NT];
 #pragma unroll
         for (int t = 0; t < NT; ++t) raw[t] = __ldcs(src + chunk_of<Geo, false>(w, t) * 32 + lane);
-        float m[NT][2][4];
-        float v[NT][8];
+        F2 m[NT][2][2];
+        F2 v[NT][4];
         X::pass1_raw(raw, m, hf);
         X::mid_stages(m);
         X::pass2(m, v, hf);
@@ -270,22 +346,17 @@ mma_fwd_kernel(const __nv_bfloat16* x, const TP* __restrict__ a, const TP* __res
 #pragma unroll
         for (int idx = 0; idx < NT; ++idx) {
             const int c = chunk_of<Geo, true>(w, idx);
-            float as[8], bs[8];
+            F2 as[4], bs[4];
             load_params8(a + (c * 32 + lane) * 8, as);
             load_params8(b + (c * 32 + lane) * 8, bs);
-            uint4 o;
-            o.x = pack_bf16x2(fmaf(v[idx][0] * inv_sqrt_d, as[0], bs[0]), fmaf(v[idx][1] * inv_sqrt_d, as[1], bs[1]));
-            o.y = pack_bf16x2(fmaf(v[idx][2] * inv_sqrt_d, as[2], bs[2]), fmaf(v[idx][3] * inv_sqrt_d, as[3], bs[3]));
-            o.z = pack_bf16x2(fmaf(v[idx][4] * inv_sqrt_d, as[4], bs[4]), fmaf(v[idx][5] * inv_sqrt_d, as[5], bs[5]));
-            o.w = pack_bf16x2(fmaf(v[idx][6] * inv_sqrt_d, as[6], bs[6]), fmaf(v[idx][7] * inv_sqrt_d, as[7], bs[7]));
-            __stcs(dst + c * 32 + lane, o);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) as[j] = mul2(as[j], rs2);
+            fwd_store_chunk(v[idx], as, bs, dst + c * 32 + lane);
         }
     }
 }
 
-// ---- backward ------------------------------------------------------------------
-// partials layout: [gridDim.x][2][D] fp32 as in the butterfly family (slot 0 holds
-// sum_t dy (.) (x H) without the 1/sqrt(d) factor, slot 1 holds sum_t dy).
+// ---- backward, rows loaded straight from global memory ------------------------------
 template <int LOGD, int TB, int RG, typename TP>
 __global__ void __launch_bounds__(MmaGeo<LOGD, TB, RG>::THREADS)
 mma_bwd_kernel(const __nv_bfloat16* dy, const __nv_bfloat16* x, const TP* __restrict__ a,
@@ -301,12 +372,13 @@ mma_bwd_kernel(const __nv_bfloat16* dy, const __nv_bfloat16* x, const TP* __rest
     float* xbuf = smem + rg * Geo::XCHG_FLOATS;
     uint32_t hf[4];
     make_h16_fragment(hf, lane);
+    const F2 rs2 = f2(inv_sqrt_d, inv_sqrt_d);
 
-    float da_acc[NT][8], db_acc[NT][8];
+    F2 da_acc[NT][4], db_acc[NT][4];
 #pragma unroll
     for (int t = 0; t < NT; ++t) {
 #pragma unroll
-        for (int e = 0; e < 8; ++e) { da_acc[t][e] = 0.0f; db_acc[t][e] = 0.0f; }
+        for (int j = 0; j < 4; ++j) { da_acc[t][j] = f2(0.0f, 0.0f); db_acc[t][j] = f2(0.0f, 0.0f); }
     }
 
     const long long stride = static_cast<long long>(gridDim.x) * RG;
@@ -318,8 +390,8 @@ mma_bwd_kernel(const __nv_bfloat16* dy, const __nv_bfloat16* x, const TP* __rest
         for (int t = 0; t < NT; ++t) raw[t] = __ldcs(xsrc + chunk_of<Geo, false>(w, t) * 32 + lane);
 #pragma unroll
         for (int t = 0; t < NT; ++t) rawdy[t] = __ldcs(dysrc + chunk_of<Geo, true>(w, t) * 32 + lane);
-        float m[NT][2][4];
-        float v[NT][8];
+        F2 m[NT][2][2];
+        F2 v[NT][4];
         // u = x H, delivered in layout B
         X::pass1_raw(raw, m, hf);
         X::mid_stages(m);
@@ -329,15 +401,11 @@ mma_bwd_kernel(const __nv_bfloat16* dy, const __nv_bfloat16* x, const TP* __rest
 #pragma unroll
         for (int idx = 0; idx < NT; ++idx) {
             const int c = chunk_of<Geo, true>(w, idx);
-            float as[8], wv[8];
+            F2 as[4];
             load_params8(a + (c * 32 + lane) * 8, as);
-            unpack8(rawdy[idx], wv);
 #pragma unroll
-            for (int e = 0; e < 8; ++e) {
-                da_acc[idx][e] = fmaf(wv[e], v[idx][e], da_acc[idx][e]);
-                db_acc[idx][e] += wv[e];
-                v[idx][e] = as[e] * wv[e];
-            }
+            for (int j = 0; j < 4; ++j) as[j] = mul2(as[j], rs2);
+            bwd_mid_chunk(v[idx], rawdy[idx], as, da_acc[idx], db_acc[idx]);
         }
         // dx = (g H)/sqrt(d): layout B in, layout A out
         X::pass1_f32(v, m, hf);
@@ -346,38 +414,10 @@ mma_bwd_kernel(const __nv_bfloat16* dy, const __nv_bfloat16* x, const TP* __rest
         X::template exchange_and_top<false>(v, xbuf + Geo::D, w, lane, 1 + rg);
         uint4* dst = reinterpret_cast<uint4*>(dx + row * Geo::D);
 #pragma unroll
-        for (int idx = 0; idx < NT; ++idx) {
-            const int c = chunk_of<Geo, false>(w, idx);
-            uint4 o;
-            o.x = pack_bf16x2(v[idx][0] * inv_sqrt_d, v[idx][1] * inv_sqrt_d);
-            o.y = pack_bf16x2(v[idx][2] * inv_sqrt_d, v[idx][3] * inv_sqrt_d);
-            o.z = pack_bf16x2(v[idx][4] * inv_sqrt_d, v[idx][5] * inv_sqrt_d);
-            o.w = pack_bf16x2(v[idx][6] * inv_sqrt_d, v[idx][7] * inv_sqrt_d);
-            __stcs(dst + c * 32 + lane, o);
-        }
+        for (int idx = 0; idx < NT; ++idx)
+            bwd_store_chunk(v[idx], dst + chunk_of<Geo, false>(w, idx) * 32 + lane);
     }
-
-    // fold the RG row groups of this CTA in a fixed order, then publish (layout B columns)
-    float* out = partials + static_cast<size_t>(blockIdx.x) * 2 * Geo::D;
-#pragma unroll
-    for (int which = 0; which < 2; ++which) {
-        __syncthreads();
-#pragma unroll
-        for (int idx = 0; idx < NT; ++idx) {
-            const int c = chunk_of<Geo, true>(w, idx);
-            float4* p = reinterpret_cast<float4*>(smem + rg * Geo::D + (c * 32 + lane) * 8);
-            const float (&src)[8] = which == 0 ? da_acc[idx] : db_acc[idx];
-            p[0] = make_float4(src[0], src[1], src[2], src[3]);
-            p[1] = make_float4(src[4], src[5], src[6], src[7]);
-        }
-        __syncthreads();
-        for (int j = threadIdx.x; j < Geo::D; j += Geo::THREADS) {
-            float s = 0.0f;
-#pragma unroll
-            for (int r = 0; r < RG; ++r) s += smem[r * Geo::D + j];
-            out[which * Geo::D + j] = s;
-        }
-    }
+    bwd_publish_partials<Geo>(da_acc, db_acc, smem, partials, rg, w, lane);
 }
 
 }  // namespace wht

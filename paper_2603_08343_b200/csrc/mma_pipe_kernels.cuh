@@ -1,0 +1,320 @@
+// Streaming versions of the tensor-core assisted kernels: rows are brought into a
+// shared-memory ring by the bulk async-copy engine (cp.async.bulk + mbarrier), so
+// the bytes in flight per SM are set by the ring depth and not by registers or
+// occupancy.  One elected lane per row group issues the copies; every wait on an
+// mbarrier is bounded -- if it ever gives up, the kernel records that in
+// g_wht_device_error and carries on (all barriers are still reached, copies that
+// were issued are still waited for, bounded again), so a fault in the pipeline
+// shows up as a status the host can read instead of a hang.
+//
+// No copy uses cluster multicast and every source is this GPU's own memory.
+#pragma once
+#include "mma_kernels.cuh"
+
+namespace wht {
+
+// set to a non-zero code by a kernel whose bounded wait expired
+__device__ unsigned int g_wht_device_error = 0;
+constexpr unsigned int kDeviceErrWaitExpired = 1;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void fence_mbar_init() {
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
+                 : "memory");
+}
+// 1-D bulk copy global -> this CTA's shared memory, completion counted on `bar`.
+// dst, src 16-byte aligned; bytes a multiple of 16.
+__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+            smem_u32(dst)),
+        "l"(src), "r"(bytes), "r"(smem_u32(bar))
+        : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait: about a quarter of a second of polling at the very least, far
+// beyond any real copy latency.  Returns false when it gave up.
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity) {
+    for (uint32_t i = 0; i < (1u << 22); ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (i > 32) __nanosleep(64);
+    }
+    atomicExch(&g_wht_device_error, kDeviceErrWaitExpired);
+    return false;
+}
+
+template <int LOGD, int TB, int RG, int S_, bool BWD>
+struct PipeGeo : MmaGeo<LOGD, TB, RG> {
+    using Base = MmaGeo<LOGD, TB, RG>;
+    static constexpr int S = S_;                              // ring depth (rows in flight per row group)
+    static constexpr int ROW_BYTES = Base::D * 2;
+    static constexpr int STAGE_BYTES = ROW_BYTES * (BWD ? 2 : 1);  // bwd: x row then dy row
+    static constexpr int RING_BYTES = RG * S * STAGE_BYTES;
+    static constexpr int XCHG_BYTES = RG * Base::XCHG_FLOATS * 4;
+    static constexpr int BAR_BYTES = RG * S * 8;
+    static constexpr int FOLD_BYTES = BWD ? RG * Base::D * 4 : 0;
+    static constexpr int PARAM_OFFSET = imax_c(RING_BYTES + XCHG_BYTES, FOLD_BYTES);
+    static constexpr int PARAM_BYTES = Base::D * 4 * (BWD ? 1 : 2);  // a/sqrt(d) [, b] as fp32
+    static constexpr int BAR_OFFSET = PARAM_OFFSET + PARAM_BYTES;
+    static constexpr int SMEM = BAR_OFFSET + BAR_BYTES;
+};
+
+// Per-channel vector -> shared memory as fp32 (times `scale`), in the order the
+// threads read it: chunk c, half h, lane l hold elements c*256 + l*8 + h*4 .. +3 at
+// float offset c*256 + h*128 + l*4, so a warp's 128-bit reads are conflict-free.
+template <int D, int THREADS>
+__device__ __forceinline__ void stage_params(const float* __restrict__ src, float* dst, float scale) {
+    for (int i = threadIdx.x; i < D / 4; i += THREADS) {
+        const float4 q = __ldg(reinterpret_cast<const float4*>(src) + i);
+        const int e0 = i * 4, c = e0 >> 8, l = (e0 & 255) >> 3, h = (e0 & 7) >> 2;
+        *reinterpret_cast<float4*>(dst + c * 256 + h * 128 + l * 4) =
+            make_float4(q.x * scale, q.y * scale, q.z * scale, q.w * scale);
+    }
+}
+template <int D, int THREADS>
+__device__ __forceinline__ void stage_params(const __nv_bfloat16* __restrict__ src, float* dst, float scale) {
+    for (int i = threadIdx.x; i < D / 4; i += THREADS) {
+        const uint2 q = __ldg(reinterpret_cast<const uint2*>(src) + i);
+        const int e0 = i * 4, c = e0 >> 8, l = (e0 & 255) >> 3, h = (e0 & 7) >> 2;
+        *reinterpret_cast<float4*>(dst + c * 256 + h * 128 + l * 4) =
+            make_float4(bf16lo_to_f32(q.x) * scale, bf16hi_to_f32(q.x) * scale, bf16lo_to_f32(q.y) * scale,
+                        bf16hi_to_f32(q.y) * scale);
+    }
+}
+__device__ __forceinline__ void read_staged8(const float* base, int c, int lane, F2 (&v)[4]) {
+    const float4* p = reinterpret_cast<const float4*>(base + c * 256 + lane * 4);
+    const float4 q0 = p[0], q1 = p[32];
+    v[0] = f2(q0.x, q0.y); v[1] = f2(q0.z, q0.w);
+    v[2] = f2(q1.x, q1.y); v[3] = f2(q1.z, q1.w);
+}
+
+// ---- forward, streamed ----------------------------------------------------------
+template <int LOGD, int TB, int RG, int S, int MINB, typename TP>
+__global__ void __launch_bounds__(MmaGeo<LOGD, TB, RG>::THREADS, MINB)
+mma_fwd_pipe_kernel(const __nv_bfloat16* x, const TP* __restrict__ a, const TP* __restrict__ b,
+                    __nv_bfloat16* y, long long T, float inv_sqrt_d) {
+    using Geo = PipeGeo<LOGD, TB, RG, S, false>;
+    using X = MmaXform<Geo>;
+    constexpr int NT = Geo::NT;
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
+    const int rg = warp / Geo::W;
+    const int w = warp % Geo::W;
+    unsigned char* ring = smem_raw + rg * (S * Geo::STAGE_BYTES);
+    float* xbuf = reinterpret_cast<float*>(smem_raw + Geo::RING_BYTES) + rg * Geo::XCHG_FLOATS;
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem_raw + Geo::BAR_OFFSET) + rg * S;
+    const bool elected = (w == 0 && lane == 0);
+
+    float* pa = reinterpret_cast<float*>(smem_raw + Geo::PARAM_OFFSET);
+    float* pb = pa + Geo::D;
+
+    if (elected) {
+#pragma unroll
+        for (int s = 0; s < S; ++s) mbar_init(full + s, 1);
+        fence_mbar_init();
+    }
+    stage_params<Geo::D, Geo::THREADS>(a, pa, inv_sqrt_d);
+    stage_params<Geo::D, Geo::THREADS>(b, pb, 1.0f);
+    __syncthreads();
+
+    uint32_t hf[4];
+    make_h16_fragment(hf, lane);
+
+    const long long stride = static_cast<long long>(gridDim.x) * RG;
+    const long long first = static_cast<long long>(blockIdx.x) * RG + rg;
+    auto issue = [&](int s, long long r) {
+        mbar_expect_tx(full + s, Geo::ROW_BYTES);
+        bulk_load(ring + s * Geo::STAGE_BYTES, x + r * Geo::D, Geo::ROW_BYTES, full + s);
+    };
+    if (elected) {
+#pragma unroll
+        for (int s = 0; s < S; ++s) {
+            const long long r = first + s * stride;
+            if (r < T) issue(s, r);
+        }
+    }
+
+    int stage = 0;
+    uint32_t phase = 0;
+    int parity = 0;
+    for (long long row = first; row < T; row += stride) {
+        mbar_wait_bounded(full + stage, phase);
+        const uint4* st = reinterpret_cast<const uint4*>(ring + stage * Geo::STAGE_BYTES);
+        uint4 raw[NT];
+#pragma unroll
+        for (int t = 0; t < NT; ++t) raw[t] = st[chunk_of<Geo, false>(w, t) * 32 + lane];
+        F2 m[NT][2][2];
+        F2 v[NT][4];
+        X::pass1_raw(raw, m, hf);  // warp-synchronous: every lane's reads of the stage are done here
+        const long long next_row = row + S * stride;
+        if constexpr (Geo::WB == 0) {
+            __syncwarp();
+            if (elected && next_row < T) issue(stage, next_row);
+        }
+        X::mid_stages(m);
+        X::pass2(m, v, hf);
+        X::template exchange_and_top<true>(v, xbuf + parity * Geo::D, w, lane, 1 + rg);
+        parity ^= 1;
+        if constexpr (Geo::WB > 0) {
+            // every warp of the row group has passed the exchange barrier, each after
+            // its pass 1: the stage is free
+            if (elected && next_row < T) issue(stage, next_row);
+        }
+        uint4* dst = reinterpret_cast<uint4*>(y + row * Geo::D);
+#pragma unroll
+        for (int idx = 0; idx < NT; ++idx) {
+            const int c = chunk_of<Geo, true>(w, idx);
+            F2 as[4], bs[4];
+            read_staged8(pa, c, lane, as);
+            read_staged8(pb, c, lane, bs);
+            fwd_store_chunk(v[idx], as, bs, dst + c * 32 + lane);
+        }
+        if (++stage == S) { stage = 0; phase ^= 1; }
+    }
+}
+
+// ---- backward, streamed -----------------------------------------------------------
+template <int LOGD, int TB, int RG, int S, int MINB, typename TP>
+__global__ void __launch_bounds__(MmaGeo<LOGD, TB, RG>::THREADS, MINB)
+mma_bwd_pipe_kernel(const __nv_bfloat16* dy, const __nv_bfloat16* x, const TP* __restrict__ a,
+                    __nv_bfloat16* dx, float* __restrict__ partials, long long T, float inv_sqrt_d) {
+    using Geo = PipeGeo<LOGD, TB, RG, S, true>;
+    using X = MmaXform<Geo>;
+    constexpr int NT = Geo::NT;
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
+    const int rg = warp / Geo::W;
+    const int w = warp % Geo::W;
+    unsigned char* ring = smem_raw + rg * (S * Geo::STAGE_BYTES);
+    float* xbuf = reinterpret_cast<float*>(smem_raw + Geo::RING_BYTES) + rg * Geo::XCHG_FLOATS;
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem_raw + Geo::BAR_OFFSET) + rg * S;
+    const bool elected = (w == 0 && lane == 0);
+
+    float* pa = reinterpret_cast<float*>(smem_raw + Geo::PARAM_OFFSET);
+
+    if (elected) {
+#pragma unroll
+        for (int s = 0; s < S; ++s) mbar_init(full + s, 1);
+        fence_mbar_init();
+    }
+    stage_params<Geo::D, Geo::THREADS>(a, pa, inv_sqrt_d);
+    __syncthreads();
+
+    uint32_t hf[4];
+    make_h16_fragment(hf, lane);
+
+    F2 da_acc[NT][4], db_acc[NT][4];
+#pragma unroll
+    for (int t = 0; t < NT; ++t) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) { da_acc[t][j] = f2(0.0f, 0.0f); db_acc[t][j] = f2(0.0f, 0.0f); }
+    }
+
+    const long long stride = static_cast<long long>(gridDim.x) * RG;
+    const long long first = static_cast<long long>(blockIdx.x) * RG + rg;
+    auto issue = [&](int s, long long r) {
+        mbar_expect_tx(full + s, Geo::STAGE_BYTES);
+        bulk_load(ring + s * Geo::STAGE_BYTES, x + r * Geo::D, Geo::ROW_BYTES, full + s);
+        bulk_load(ring + s * Geo::STAGE_BYTES + Geo::ROW_BYTES, dy + r * Geo::D, Geo::ROW_BYTES, full + s);
+    };
+    if (elected) {
+#pragma unroll
+        for (int s = 0; s < S; ++s) {
+            const long long r = first + s * stride;
+            if (r < T) issue(s, r);
+        }
+    }
+
+    int stage = 0;
+    uint32_t phase = 0;
+    for (long long row = first; row < T; row += stride) {
+        mbar_wait_bounded(full + stage, phase);
+        const uint4* stx = reinterpret_cast<const uint4*>(ring + stage * Geo::STAGE_BYTES);
+        const uint4* stdy = reinterpret_cast<const uint4*>(ring + stage * Geo::STAGE_BYTES + Geo::ROW_BYTES);
+        uint4 raw[NT];
+#pragma unroll
+        for (int t = 0; t < NT; ++t) raw[t] = stx[chunk_of<Geo, false>(w, t) * 32 + lane];
+        F2 m[NT][2][2];
+        F2 v[NT][4];
+        // u = x H, delivered in layout B
+        X::pass1_raw(raw, m, hf);
+        X::mid_stages(m);
+        X::pass2(m, v, hf);
+        X::template exchange_and_top<true>(v, xbuf, w, lane, 1 + rg);
+        // da, db partial sums and g = a (.) dy, all in layout B
+#pragma unroll
+        for (int idx = 0; idx < NT; ++idx) {
+            const int c = chunk_of<Geo, true>(w, idx);
+            F2 as[4];
+            read_staged8(pa, c, lane, as);
+            bwd_mid_chunk(v[idx], stdy[c * 32 + lane], as, da_acc[idx], db_acc[idx]);
+        }
+        // dx = (g H)/sqrt(d): layout B in, layout A out
+        X::pass1_f32(v, m, hf);  // warp-synchronous: this warp's reads of the stage are done here
+        const long long next_row = row + S * stride;
+        if constexpr (Geo::WB == 0) {
+            __syncwarp();
+            if (elected && next_row < T) issue(stage, next_row);
+        }
+        X::mid_stages(m);
+        X::pass2(m, v, hf);
+        X::template exchange_and_top<false>(v, xbuf + Geo::D, w, lane, 1 + rg);
+        if constexpr (Geo::WB > 0) {
+            if (elected && next_row < T) issue(stage, next_row);
+        }
+        uint4* dst = reinterpret_cast<uint4*>(dx + row * Geo::D);
+#pragma unroll
+        for (int idx = 0; idx < NT; ++idx)
+            bwd_store_chunk(v[idx], dst + chunk_of<Geo, false>(w, idx) * 32 + lane);
+        if (++stage == S) { stage = 0; phase ^= 1; }
+    }
+    bwd_publish_partials<Geo>(da_acc, db_acc, reinterpret_cast<float*>(smem_raw), partials, rg, w, lane);
+}
+
+// ---- second pass of the backward, parallel over slices of the partials -------------
+// block = 32 columns x 32 slices; slice s adds partials s, s+32, ... in order, then
+// the 32 slice sums are added in order: a fixed association, bit-reproducible.
+__global__ void __launch_bounds__(1024)
+dadb_finalize32_kernel(const float* __restrict__ partials, int nparts, int d, float inv_sqrt_d,
+                       float* __restrict__ da, float* __restrict__ db) {
+    __shared__ float red[32][33];
+    const int cx = threadIdx.x & 31;
+    const int sl = threadIdx.x >> 5;
+    const int j = blockIdx.x * 32 + cx;  // column in [0, 2d): da columns then db columns
+    const int which = j / d;
+    const int col = j - which * d;
+    const size_t stride = static_cast<size_t>(2) * d;
+    const float* src = partials + static_cast<size_t>(which) * d + col;
+    float s = 0.0f;
+    for (int p = sl; p < nparts; p += 32) s += src[p * stride];
+    red[sl][cx] = s;
+    __syncthreads();
+    if (sl == 0) {
+        float t = 0.0f;
+#pragma unroll
+        for (int k = 0; k < 32; ++k) t += red[k][cx];
+        if (which == 0) da[col] = t * inv_sqrt_d; else db[col] = t;
+    }
+}
+
+}  // namespace wht

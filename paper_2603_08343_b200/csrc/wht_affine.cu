@@ -9,6 +9,7 @@
 
 #include "bfly_kernels.cuh"
 #include "mma_kernels.cuh"
+#include "mma_pipe_kernels.cuh"
 
 namespace {
 
@@ -53,6 +54,7 @@ int current_device(int* dev, int* sms) {
 bool is_pow2(int32_t d) { return d > 0 && (d & (d - 1)) == 0; }
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 int log2_of(int32_t d) { int l = 0; while ((1 << l) < d) ++l; return l; }
+long long ceil_div(long long a, long long b) { return (a + b - 1) / b; }
 
 int check_common(int64_t T, int32_t d, int dtype) {
     if (dtype != WHT_F32 && dtype != WHT_BF16 && dtype != WHT_BF16_PF32) return WHT_ERR_BAD_DTYPE;
@@ -70,76 +72,136 @@ int resident_ctas(Kernel kernel, int threads, size_t smem, int dev, int* cache) 
                                  static_cast<int>(smem)) != cudaSuccess)
             return 0;
     }
+    if (smem > 0) {
+        // first see how many CTAs fit when shared memory takes all it may ...
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                 cudaSharedmemCarveoutMaxShared) != cudaSuccess)
+            return 0;
+    }
     int n = 0;
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kernel, threads, smem) != cudaSuccess) return 0;
+    if (smem > 0 && n > 0) {
+        // ... then ask for no more than those CTAs need, so that what is left stays L1
+        // (the per-channel parameters are re-read from L1 for every row)
+        int max_smem_sm = 0;
+        if (cudaDeviceGetAttribute(&max_smem_sm, cudaDevAttrMaxSharedMemoryPerMultiprocessor, dev) != cudaSuccess)
+            return 0;
+        const size_t want = static_cast<size_t>(n) * (smem + 1024);
+        int pct = static_cast<int>((want * 100 + max_smem_sm - 1) / max_smem_sm);
+        if (pct > 100) pct = 100;
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, pct) != cudaSuccess)
+            return 0;
+        int n2 = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n2, kernel, threads, smem) != cudaSuccess) return 0;
+        if (n2 < n) {
+            if (cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                     cudaSharedmemCarveoutMaxShared) != cudaSuccess)
+                return 0;
+        }
+    }
     cache[dev] = n > 0 ? n : 0;
     return cache[dev];
 }
 
-long long ceil_div(long long a, long long b) { return (a + b - 1) / b; }
+float inv_sqrt(int d) { return static_cast<float>(1.0 / sqrt(static_cast<double>(d))); }
 
-// ------------------------------------------------------------------ butterfly family
-template <int LOGD, typename TIO, typename TP>
-int launch_bfly_fwd(const void* x, const void* a, const void* b, void* y, int64_t T,
-                    int dev, int sms, cudaStream_t s) {
-    using Geo = BflyGeo<LOGD>;
-    static int occ[kMaxDevices] = {};
-    auto kernel = bfly_fwd_kernel<LOGD, TIO, TP>;
-    const int per_sm = resident_ctas(kernel, Geo::THREADS, Geo::SMEM_FWD, dev, occ);
-    if (per_sm <= 0) return cuda_fail(cudaGetLastError());
-    const long long tiles = ceil_div(T, Geo::R);
-    const long long cap = static_cast<long long>(sms) * per_sm;
-    const unsigned grid = static_cast<unsigned>(tiles < cap ? tiles : cap);
-    const float rs = static_cast<float>(1.0 / sqrt(static_cast<double>(Geo::D)));
-    kernel<<<grid, Geo::THREADS, Geo::SMEM_FWD, s>>>(
-        static_cast<const TIO*>(x), static_cast<const TP*>(a), static_cast<const TP*>(b),
-        static_cast<TIO*>(y), static_cast<long long>(T), rs);
+// Everything a launcher needs besides the tensors.
+struct Ctx {
+    int64_t T;
+    int dev;
+    int sms;
+    cudaStream_t stream;
+};
+
+struct FwdArgs {
+    const void* x;
+    const void* a;
+    const void* b;
+    void* y;
+};
+
+struct BwdArgs {
+    const void* dy;
+    const void* x;
+    const void* a;
+    void* dx;
+    float* da;
+    float* db;
+    void* ws;
+    size_t ws_bytes;
+    bool query_only;  // only report the scratch size in *need
+    size_t* need;
+};
+
+int launch_finalize(const BwdArgs& g, int nparts, int d, cudaStream_t s) {
+    if (d >= 32) {
+        dadb_finalize32_kernel<<<2 * d / 32, 1024, 0, s>>>(static_cast<const float*>(g.ws), nparts, d,
+                                                          inv_sqrt(d), g.da, g.db);
+    } else {
+        dadb_finalize_kernel<<<(2 * d + 255) / 256, 256, 0, s>>>(static_cast<const float*>(g.ws), nparts, d,
+                                                                inv_sqrt(d), g.da, g.db);
+    }
     WHT_CUDA_TRY(cudaGetLastError());
     return WHT_OK;
 }
 
-template <int LOGD>
-int bfly_bwd_grid(int64_t T, int sms, int per_sm) {
-    using Geo = BflyGeo<LOGD>;
-    const long long tiles = ceil_div(T, Geo::R);
+// Common tail of every backward launcher: size the scratch, check it, launch.
+template <typename Launch>
+int run_bwd_with_grid(const BwdArgs& g, const Ctx& c, int grid, int d, Launch launch) {
+    *g.need = static_cast<size_t>(grid) * 2 * d * sizeof(float);
+    if (g.query_only) return WHT_OK;
+    if (*g.need > 0 && (g.ws == nullptr || g.ws_bytes < *g.need)) return WHT_ERR_WORKSPACE;
+    if (grid > 0) {
+        launch(grid);
+        WHT_CUDA_TRY(cudaGetLastError());
+    }
+    return launch_finalize(g, grid, d, c.stream);
+}
+
+int capped_grid(int64_t tiles, int sms, int per_sm) {
     const long long cap = static_cast<long long>(sms) * per_sm;
     return static_cast<int>(tiles < cap ? tiles : cap);
 }
 
+// ------------------------------------------------------------------ butterfly family
 template <int LOGD, typename TIO, typename TP>
-int launch_bfly_bwd(const void* dy, const void* x, const void* a, void* dx, float* da, float* db,
-                    int64_t T, void* ws, size_t ws_bytes, bool query_only, size_t* need,
-                    int dev, int sms, cudaStream_t s) {
+int launch_bfly_fwd(const FwdArgs& f, const Ctx& c) {
+    using Geo = BflyGeo<LOGD>;
+    static int occ[kMaxDevices] = {};
+    auto kernel = bfly_fwd_kernel<LOGD, TIO, TP>;
+    const int per_sm = resident_ctas(kernel, Geo::THREADS, Geo::SMEM_FWD, c.dev, occ);
+    if (per_sm <= 0) return cuda_fail(cudaGetLastError());
+    const int grid = capped_grid(ceil_div(c.T, Geo::R), c.sms, per_sm);
+    kernel<<<grid, Geo::THREADS, Geo::SMEM_FWD, c.stream>>>(
+        static_cast<const TIO*>(f.x), static_cast<const TP*>(f.a), static_cast<const TP*>(f.b),
+        static_cast<TIO*>(f.y), static_cast<long long>(c.T), inv_sqrt(Geo::D));
+    WHT_CUDA_TRY(cudaGetLastError());
+    return WHT_OK;
+}
+
+template <int LOGD, typename TIO, typename TP>
+int launch_bfly_bwd(const BwdArgs& g, const Ctx& c) {
     using Geo = BflyGeo<LOGD>;
     static int occ[kMaxDevices] = {};
     auto kernel = bfly_bwd_kernel<LOGD, TIO, TP>;
-    const int per_sm = resident_ctas(kernel, Geo::THREADS, Geo::SMEM_BWD, dev, occ);
+    const int per_sm = resident_ctas(kernel, Geo::THREADS, Geo::SMEM_BWD, c.dev, occ);
     if (per_sm <= 0) return cuda_fail(cudaGetLastError());
-    const int grid = bfly_bwd_grid<LOGD>(T, sms, per_sm);
-    *need = static_cast<size_t>(grid) * 2 * Geo::D * sizeof(float);
-    if (query_only) return WHT_OK;
-    if (*need > 0 && (ws == nullptr || ws_bytes < *need)) return WHT_ERR_WORKSPACE;
-    const float rs = static_cast<float>(1.0 / sqrt(static_cast<double>(Geo::D)));
-    if (grid > 0) {
-        kernel<<<grid, Geo::THREADS, Geo::SMEM_BWD, s>>>(
-            static_cast<const TIO*>(dy), static_cast<const TIO*>(x), static_cast<const TP*>(a),
-            static_cast<TIO*>(dx), static_cast<float*>(ws), static_cast<long long>(T), rs);
-        WHT_CUDA_TRY(cudaGetLastError());
-    }
-    dadb_finalize_kernel<<<(2 * Geo::D + 255) / 256, 256, 0, s>>>(
-        static_cast<const float*>(ws), grid, Geo::D, rs, da, db);
-    WHT_CUDA_TRY(cudaGetLastError());
-    return WHT_OK;
+    const int grid = capped_grid(ceil_div(c.T, Geo::R), c.sms, per_sm);
+    return run_bwd_with_grid(g, c, grid, Geo::D, [&](int n) {
+        kernel<<<n, Geo::THREADS, Geo::SMEM_BWD, c.stream>>>(
+            static_cast<const TIO*>(g.dy), static_cast<const TIO*>(g.x), static_cast<const TP*>(g.a),
+            static_cast<TIO*>(g.dx), static_cast<float*>(g.ws), static_cast<long long>(c.T),
+            inv_sqrt(Geo::D));
+    });
 }
 
 #define WHT_FOR_EACH_LOGD(M) \
     M(3) M(4) M(5) M(6) M(7) M(8) M(9) M(10) M(11) M(12) M(13) M(14) M(15)
 
 template <typename TIO, typename TP>
-int dispatch_bfly_fwd(int logd, const void* x, const void* a, const void* b, void* y, int64_t T,
-                      int dev, int sms, cudaStream_t s) {
+int dispatch_bfly_fwd(int logd, const FwdArgs& f, const Ctx& c) {
     switch (logd) {
-#define M(L) case L: return launch_bfly_fwd<L, TIO, TP>(x, a, b, y, T, dev, sms, s);
+#define M(L) case L: return launch_bfly_fwd<L, TIO, TP>(f, c);
         WHT_FOR_EACH_LOGD(M)
 #undef M
     }
@@ -147,143 +209,172 @@ int dispatch_bfly_fwd(int logd, const void* x, const void* a, const void* b, voi
 }
 
 template <typename TIO, typename TP>
-int dispatch_bfly_bwd(int logd, const void* dy, const void* x, const void* a, void* dx, float* da,
-                      float* db, int64_t T, void* ws, size_t ws_bytes, bool query_only, size_t* need,
-                      int dev, int sms, cudaStream_t s) {
+int dispatch_bfly_bwd(int logd, const BwdArgs& g, const Ctx& c) {
     switch (logd) {
-#define M(L) case L: return launch_bfly_bwd<L, TIO, TP>(dy, x, a, dx, da, db, T, ws, ws_bytes, query_only, need, dev, sms, s);
+#define M(L) case L: return launch_bfly_bwd<L, TIO, TP>(g, c);
         WHT_FOR_EACH_LOGD(M)
 #undef M
     }
     return WHT_ERR_BAD_DIM;
 }
 
-
-// ------------------------------------------------------------------ tensor-core family
+// ------------------------------------------------------------------ tensor-core family, direct loads
 template <int LOGD, int TB, int RG, typename TP>
-int launch_mma_fwd(const void* x, const void* a, const void* b, void* y, int64_t T,
-                   int dev, int sms, cudaStream_t s) {
+int launch_mma_fwd(const FwdArgs& f, const Ctx& c) {
     using Geo = MmaGeo<LOGD, TB, RG>;
     static int occ[kMaxDevices] = {};
     auto kernel = mma_fwd_kernel<LOGD, TB, RG, TP>;
-    const int per_sm = resident_ctas(kernel, Geo::THREADS, Geo::SMEM_FWD, dev, occ);
+    const int per_sm = resident_ctas(kernel, Geo::THREADS, Geo::SMEM_FWD, c.dev, occ);
     if (per_sm <= 0) return cuda_fail(cudaGetLastError());
-    const long long tiles = ceil_div(T, RG);
-    const long long cap = static_cast<long long>(sms) * per_sm;
-    const unsigned grid = static_cast<unsigned>(tiles < cap ? tiles : cap);
-    const float rs = static_cast<float>(1.0 / sqrt(static_cast<double>(Geo::D)));
-    kernel<<<grid, Geo::THREADS, Geo::SMEM_FWD, s>>>(
-        static_cast<const __nv_bfloat16*>(x), static_cast<const TP*>(a), static_cast<const TP*>(b),
-        static_cast<__nv_bfloat16*>(y), static_cast<long long>(T), rs);
+    const int grid = capped_grid(ceil_div(c.T, RG), c.sms, per_sm);
+    kernel<<<grid, Geo::THREADS, Geo::SMEM_FWD, c.stream>>>(
+        static_cast<const __nv_bfloat16*>(f.x), static_cast<const TP*>(f.a), static_cast<const TP*>(f.b),
+        static_cast<__nv_bfloat16*>(f.y), static_cast<long long>(c.T), inv_sqrt(Geo::D));
     WHT_CUDA_TRY(cudaGetLastError());
     return WHT_OK;
 }
 
 template <int LOGD, int TB, int RG, typename TP>
-int launch_mma_bwd(const void* dy, const void* x, const void* a, void* dx, float* da, float* db,
-                   int64_t T, void* ws, size_t ws_bytes, bool query_only, size_t* need,
-                   int dev, int sms, cudaStream_t s) {
+int launch_mma_bwd(const BwdArgs& g, const Ctx& c) {
     using Geo = MmaGeo<LOGD, TB, RG>;
     static int occ[kMaxDevices] = {};
     auto kernel = mma_bwd_kernel<LOGD, TB, RG, TP>;
-    const int per_sm = resident_ctas(kernel, Geo::THREADS, Geo::SMEM_BWD, dev, occ);
+    const int per_sm = resident_ctas(kernel, Geo::THREADS, Geo::SMEM_BWD, c.dev, occ);
     if (per_sm <= 0) return cuda_fail(cudaGetLastError());
-    const long long tiles = ceil_div(T, RG);
-    const long long cap = static_cast<long long>(sms) * per_sm;
-    const int grid = static_cast<int>(tiles < cap ? tiles : cap);
-    *need = static_cast<size_t>(grid) * 2 * Geo::D * sizeof(float);
-    if (query_only) return WHT_OK;
-    if (*need > 0 && (ws == nullptr || ws_bytes < *need)) return WHT_ERR_WORKSPACE;
-    const float rs = static_cast<float>(1.0 / sqrt(static_cast<double>(Geo::D)));
-    if (grid > 0) {
-        kernel<<<grid, Geo::THREADS, Geo::SMEM_BWD, s>>>(
-            static_cast<const __nv_bfloat16*>(dy), static_cast<const __nv_bfloat16*>(x),
-            static_cast<const TP*>(a), static_cast<__nv_bfloat16*>(dx), static_cast<float*>(ws),
-            static_cast<long long>(T), rs);
-        WHT_CUDA_TRY(cudaGetLastError());
-    }
-    dadb_finalize_kernel<<<(2 * Geo::D + 255) / 256, 256, 0, s>>>(
-        static_cast<const float*>(ws), grid, Geo::D, rs, da, db);
+    const int grid = capped_grid(ceil_div(c.T, RG), c.sms, per_sm);
+    return run_bwd_with_grid(g, c, grid, Geo::D, [&](int n) {
+        kernel<<<n, Geo::THREADS, Geo::SMEM_BWD, c.stream>>>(
+            static_cast<const __nv_bfloat16*>(g.dy), static_cast<const __nv_bfloat16*>(g.x),
+            static_cast<const TP*>(g.a), static_cast<__nv_bfloat16*>(g.dx), static_cast<float*>(g.ws),
+            static_cast<long long>(c.T), inv_sqrt(Geo::D));
+    });
+}
+
+// ------------------------------------------------------------------ tensor-core family, streamed rows
+template <int LOGD, int TB, int RG, int S, int MINB, typename TP>
+int launch_mma_fwd_pipe(const FwdArgs& f, const Ctx& c) {
+    using Geo = PipeGeo<LOGD, TB, RG, S, false>;
+    static int occ[kMaxDevices] = {};
+    auto kernel = mma_fwd_pipe_kernel<LOGD, TB, RG, S, MINB, TP>;
+    const int per_sm = resident_ctas(kernel, Geo::THREADS, Geo::SMEM, c.dev, occ);
+    if (per_sm <= 0) return cuda_fail(cudaGetLastError());
+    const int grid = capped_grid(ceil_div(c.T, RG), c.sms, per_sm);
+    kernel<<<grid, Geo::THREADS, Geo::SMEM, c.stream>>>(
+        static_cast<const __nv_bfloat16*>(f.x), static_cast<const TP*>(f.a), static_cast<const TP*>(f.b),
+        static_cast<__nv_bfloat16*>(f.y), static_cast<long long>(c.T), inv_sqrt(Geo::D));
     WHT_CUDA_TRY(cudaGetLastError());
     return WHT_OK;
 }
 
-// Row splits (LOGD, TB, RG) of the tensor-core family.  `wide` spreads a row over
-// more warps (lower latency per row, used for decode and as tuning alternative).
+template <int LOGD, int TB, int RG, int S, int MINB, typename TP>
+int launch_mma_bwd_pipe(const BwdArgs& g, const Ctx& c) {
+    using Geo = PipeGeo<LOGD, TB, RG, S, true>;
+    static int occ[kMaxDevices] = {};
+    auto kernel = mma_bwd_pipe_kernel<LOGD, TB, RG, S, MINB, TP>;
+    const int per_sm = resident_ctas(kernel, Geo::THREADS, Geo::SMEM, c.dev, occ);
+    if (per_sm <= 0) return cuda_fail(cudaGetLastError());
+    const int grid = capped_grid(ceil_div(c.T, RG), c.sms, per_sm);
+    return run_bwd_with_grid(g, c, grid, Geo::D, [&](int n) {
+        kernel<<<n, Geo::THREADS, Geo::SMEM, c.stream>>>(
+            static_cast<const __nv_bfloat16*>(g.dy), static_cast<const __nv_bfloat16*>(g.x),
+            static_cast<const TP*>(g.a), static_cast<__nv_bfloat16*>(g.dx), static_cast<float*>(g.ws),
+            static_cast<long long>(c.T), inv_sqrt(Geo::D));
+    });
+}
+
+// How a row is split for each d: (TB = log2 chunks per thread, RG = rows in flight
+// per CTA, S = ring depth).  `few_rows` picks the direct-load kernels with a row
+// spread over more warps (lowest latency per row: decode and small batches).
 template <typename TP>
-int dispatch_mma_fwd(int logd, bool wide, const void* x, const void* a, const void* b, void* y,
-                     int64_t T, int dev, int sms, cudaStream_t s) {
-    switch (logd) {
-        case 9: return launch_mma_fwd<9, 1, 4, TP>(x, a, b, y, T, dev, sms, s);
-        case 10: return wide ? launch_mma_fwd<10, 1, 2, TP>(x, a, b, y, T, dev, sms, s)
-                             : launch_mma_fwd<10, 2, 4, TP>(x, a, b, y, T, dev, sms, s);
-        case 11: return wide ? launch_mma_fwd<11, 2, 2, TP>(x, a, b, y, T, dev, sms, s)
-                             : launch_mma_fwd<11, 3, 4, TP>(x, a, b, y, T, dev, sms, s);
-        case 12: return wide ? launch_mma_fwd<12, 2, 1, TP>(x, a, b, y, T, dev, sms, s)
-                             : launch_mma_fwd<12, 3, 2, TP>(x, a, b, y, T, dev, sms, s);
-        case 13: return launch_mma_fwd<13, 3, 1, TP>(x, a, b, y, T, dev, sms, s);
+int dispatch_mma_fwd(int logd, bool few_rows, bool streamed, const FwdArgs& f, const Ctx& c) {
+    if (few_rows) {
+        switch (logd) {
+            case 9: return launch_mma_fwd<9, 1, 4, TP>(f, c);
+            case 10: return launch_mma_fwd<10, 1, 2, TP>(f, c);
+            case 11: return launch_mma_fwd<11, 2, 2, TP>(f, c);
+            case 12: return launch_mma_fwd<12, 2, 1, TP>(f, c);
+            case 13: return launch_mma_fwd<13, 3, 1, TP>(f, c);
+        }
+    } else if (!streamed) {
+        switch (logd) {
+            case 9: return launch_mma_fwd<9, 1, 4, TP>(f, c);
+            case 10: return launch_mma_fwd<10, 2, 4, TP>(f, c);
+            case 11: return launch_mma_fwd<11, 3, 4, TP>(f, c);
+            case 12: return launch_mma_fwd<12, 3, 2, TP>(f, c);
+            case 13: return launch_mma_fwd<13, 3, 1, TP>(f, c);
+        }
+    } else {
+        switch (logd) {
+            case 9: return launch_mma_fwd_pipe<9, 1, 8, 4, 2, TP>(f, c);
+            case 10: return launch_mma_fwd_pipe<10, 2, 8, 4, 3, TP>(f, c);
+            case 11: return launch_mma_fwd_pipe<11, 3, 8, 3, 2, TP>(f, c);
+            case 12: return launch_mma_fwd_pipe<12, 3, 2, 3, 2, TP>(f, c);
+            case 13: return launch_mma_fwd_pipe<13, 3, 1, 3, 2, TP>(f, c);
+        }
     }
     return WHT_ERR_BAD_DIM;
 }
 
 template <typename TP>
-int dispatch_mma_bwd(int logd, bool wide, const void* dy, const void* x, const void* a, void* dx,
-                     float* da, float* db, int64_t T, void* ws, size_t ws_bytes, bool query_only,
-                     size_t* need, int dev, int sms, cudaStream_t s) {
-#define WHT_BWD_ARGS dy, x, a, dx, da, db, T, ws, ws_bytes, query_only, need, dev, sms, s
-    switch (logd) {
-        case 9: return launch_mma_bwd<9, 1, 8, TP>(WHT_BWD_ARGS);
-        case 10: return wide ? launch_mma_bwd<10, 1, 4, TP>(WHT_BWD_ARGS) : launch_mma_bwd<10, 2, 8, TP>(WHT_BWD_ARGS);
-        case 11: return wide ? launch_mma_bwd<11, 2, 4, TP>(WHT_BWD_ARGS) : launch_mma_bwd<11, 3, 4, TP>(WHT_BWD_ARGS);
-        case 12: return wide ? launch_mma_bwd<12, 2, 2, TP>(WHT_BWD_ARGS) : launch_mma_bwd<12, 3, 2, TP>(WHT_BWD_ARGS);
-        case 13: return launch_mma_bwd<13, 3, 1, TP>(WHT_BWD_ARGS);
+int dispatch_mma_bwd(int logd, bool streamed, const BwdArgs& g, const Ctx& c) {
+    if (!streamed) {
+        switch (logd) {
+            case 9: return launch_mma_bwd<9, 1, 8, TP>(g, c);
+            case 10: return launch_mma_bwd<10, 2, 8, TP>(g, c);
+            case 11: return launch_mma_bwd<11, 2, 4, TP>(g, c);
+            case 12: return launch_mma_bwd<12, 2, 2, TP>(g, c);
+            case 13: return launch_mma_bwd<13, 3, 1, TP>(g, c);
+        }
+    } else {
+        switch (logd) {
+            case 9: return launch_mma_bwd_pipe<9, 1, 8, 4, 2, TP>(g, c);
+            case 10: return launch_mma_bwd_pipe<10, 2, 8, 3, 2, TP>(g, c);
+            case 11: return launch_mma_bwd_pipe<11, 2, 4, 3, 2, TP>(g, c);
+            case 12: return launch_mma_bwd_pipe<12, 2, 2, 3, 1, TP>(g, c);
+            case 13: return launch_mma_bwd_pipe<13, 3, 1, 2, 1, TP>(g, c);
+        }
     }
-#undef WHT_BWD_ARGS
     return WHT_ERR_BAD_DIM;
 }
 
 bool mma_supported(int logd, int dtype) { return dtype != WHT_F32 && logd >= 9 && logd <= 13; }
 
+// Streaming pays once every row group has several rows to pipeline.
+bool enough_rows_to_stream(int64_t T, int sms) { return T >= static_cast<int64_t>(sms) * 32; }
+
 // ------------------------------------------------------------------ selection
-int run_fwd(const void* x, const void* a, const void* b, void* y, int64_t T, int32_t d, int dtype,
-            cudaStream_t s, bool decode) {
-    int dev = 0, sms = 0;
-    int rc = current_device(&dev, &sms);
+int run_fwd(const FwdArgs& f, int64_t T, int32_t d, int dtype, cudaStream_t s, bool decode) {
+    Ctx c{T, 0, 0, s};
+    int rc = current_device(&c.dev, &c.sms);
     if (rc != WHT_OK) return rc;
     const int logd = log2_of(d);
     if (g_variant != 1 && mma_supported(logd, dtype)) {
-        const bool wide = decode || g_variant == 3;
-        return dtype == WHT_BF16
-                   ? dispatch_mma_fwd<__nv_bfloat16>(logd, wide, x, a, b, y, T, dev, sms, s)
-                   : dispatch_mma_fwd<float>(logd, wide, x, a, b, y, T, dev, sms, s);
+        const bool streamed = g_variant == 3 || (g_variant == 0 && !decode && enough_rows_to_stream(T, c.sms));
+        const bool few_rows = !streamed && (decode || (g_variant == 0 && T < static_cast<int64_t>(c.sms) * 4));
+        return dtype == WHT_BF16 ? dispatch_mma_fwd<__nv_bfloat16>(logd, few_rows, streamed, f, c)
+                                 : dispatch_mma_fwd<float>(logd, few_rows, streamed, f, c);
     }
     switch (dtype) {
-        case WHT_F32: return dispatch_bfly_fwd<float, float>(logd, x, a, b, y, T, dev, sms, s);
-        case WHT_BF16: return dispatch_bfly_fwd<__nv_bfloat16, __nv_bfloat16>(logd, x, a, b, y, T, dev, sms, s);
-        default: return dispatch_bfly_fwd<__nv_bfloat16, float>(logd, x, a, b, y, T, dev, sms, s);
+        case WHT_F32: return dispatch_bfly_fwd<float, float>(logd, f, c);
+        case WHT_BF16: return dispatch_bfly_fwd<__nv_bfloat16, __nv_bfloat16>(logd, f, c);
+        default: return dispatch_bfly_fwd<__nv_bfloat16, float>(logd, f, c);
     }
 }
 
-int run_bwd(const void* dy, const void* x, const void* a, void* dx, float* da, float* db, int64_t T,
-            int32_t d, int dtype, void* ws, size_t ws_bytes, bool query_only, size_t* need,
-            cudaStream_t s) {
-    int dev = 0, sms = 0;
-    int rc = current_device(&dev, &sms);
+int run_bwd(const BwdArgs& g, int64_t T, int32_t d, int dtype, cudaStream_t s) {
+    Ctx c{T, 0, 0, s};
+    int rc = current_device(&c.dev, &c.sms);
     if (rc != WHT_OK) return rc;
     const int logd = log2_of(d);
     if (g_variant != 1 && mma_supported(logd, dtype)) {
-        const bool wide = g_variant != 3;
-        return dtype == WHT_BF16
-                   ? dispatch_mma_bwd<__nv_bfloat16>(logd, wide, dy, x, a, dx, da, db, T, ws, ws_bytes, query_only, need, dev, sms, s)
-                   : dispatch_mma_bwd<float>(logd, wide, dy, x, a, dx, da, db, T, ws, ws_bytes, query_only, need, dev, sms, s);
+        const bool streamed = g_variant == 3 || (g_variant == 0 && enough_rows_to_stream(T, c.sms));
+        return dtype == WHT_BF16 ? dispatch_mma_bwd<__nv_bfloat16>(logd, streamed, g, c)
+                                 : dispatch_mma_bwd<float>(logd, streamed, g, c);
     }
     switch (dtype) {
-        case WHT_F32:
-            return dispatch_bfly_bwd<float, float>(logd, dy, x, a, dx, da, db, T, ws, ws_bytes, query_only, need, dev, sms, s);
-        case WHT_BF16:
-            return dispatch_bfly_bwd<__nv_bfloat16, __nv_bfloat16>(logd, dy, x, a, dx, da, db, T, ws, ws_bytes, query_only, need, dev, sms, s);
-        default:
-            return dispatch_bfly_bwd<__nv_bfloat16, float>(logd, dy, x, a, dx, da, db, T, ws, ws_bytes, query_only, need, dev, sms, s);
+        case WHT_F32: return dispatch_bfly_bwd<float, float>(logd, g, c);
+        case WHT_BF16: return dispatch_bfly_bwd<__nv_bfloat16, __nv_bfloat16>(logd, g, c);
+        default: return dispatch_bfly_bwd<__nv_bfloat16, float>(logd, g, c);
     }
 }
 
@@ -307,6 +398,11 @@ int check_bwd_args(const void* dy, const void* x, const void* a, void* dx, float
     return WHT_OK;
 }
 
+int query_bwd_bytes(int64_t T, int32_t d, int dtype, size_t* need) {
+    BwdArgs q{nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, 0, true, need};
+    return run_bwd(q, T, d, dtype, nullptr);
+}
+
 }  // namespace
 
 extern "C" {
@@ -316,7 +412,7 @@ int wht_affine_fwd(const void* x, const void* a, const void* b, void* y, int64_t
     int rc = check_fwd_args(x, a, b, y, T, d, dtype);
     if (rc != WHT_OK) return rc;
     if (T == 0) return WHT_OK;
-    return run_fwd(x, a, b, y, T, d, dtype, static_cast<cudaStream_t>(stream), false);
+    return run_fwd(FwdArgs{x, a, b, y}, T, d, dtype, static_cast<cudaStream_t>(stream), false);
 }
 
 int wht_affine_fwd_decode(const void* x, const void* a, const void* b, void* y, int64_t T, int32_t d,
@@ -324,15 +420,13 @@ int wht_affine_fwd_decode(const void* x, const void* a, const void* b, void* y, 
     int rc = check_fwd_args(x, a, b, y, T, d, dtype);
     if (rc != WHT_OK) return rc;
     if (T == 0) return WHT_OK;
-    return run_fwd(x, a, b, y, T, d, dtype, static_cast<cudaStream_t>(stream), true);
+    return run_fwd(FwdArgs{x, a, b, y}, T, d, dtype, static_cast<cudaStream_t>(stream), true);
 }
 
 size_t wht_affine_bwd_workspace_bytes(int64_t T, int32_t d, int dtype) {
     if (check_common(T, d, dtype) != WHT_OK) return 0;
     size_t need = 0;
-    if (run_bwd(nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, T, d, dtype, nullptr, 0, true,
-                &need, nullptr) != WHT_OK)
-        return 0;
+    if (query_bwd_bytes(T, d, dtype, &need) != WHT_OK) return 0;
     return need;
 }
 
@@ -343,8 +437,8 @@ int wht_affine_bwd_ws(const void* dy, const void* x, const void* a, void* dx, fl
     if (rc != WHT_OK) return rc;
     if (workspace && !aligned16(workspace)) return WHT_ERR_MISALIGNED;
     size_t need = 0;
-    return run_bwd(dy, x, a, dx, da, db, T, d, dtype, workspace, workspace_bytes, false, &need,
-                   static_cast<cudaStream_t>(stream));
+    BwdArgs g{dy, x, a, dx, da, db, workspace, workspace_bytes, false, &need};
+    return run_bwd(g, T, d, dtype, static_cast<cudaStream_t>(stream));
 }
 
 int wht_affine_bwd(const void* dy, const void* x, const void* a, void* dx, float* da, float* db,
@@ -352,8 +446,7 @@ int wht_affine_bwd(const void* dy, const void* x, const void* a, void* dx, float
     int rc = check_bwd_args(dy, x, a, dx, da, db, T, d, dtype);
     if (rc != WHT_OK) return rc;
     size_t need = 0;
-    rc = run_bwd(nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, T, d, dtype, nullptr, 0, true,
-                 &need, nullptr);
+    rc = query_bwd_bytes(T, d, dtype, &need);
     if (rc != WHT_OK) return rc;
     int dev = 0, sms = 0;
     rc = current_device(&dev, &sms);
@@ -383,8 +476,8 @@ int wht_affine_bwd(const void* dy, const void* x, const void* a, void* dx, float
         ws = st.scratch;
         ws_bytes = st.scratch_bytes;
     }
-    return run_bwd(dy, x, a, dx, da, db, T, d, dtype, ws, ws_bytes, false, &need,
-                   static_cast<cudaStream_t>(stream));
+    BwdArgs g{dy, x, a, dx, da, db, ws, ws_bytes, false, &need};
+    return run_bwd(g, T, d, dtype, static_cast<cudaStream_t>(stream));
 }
 
 int wht_affine_set_variant(int variant) {
@@ -406,13 +499,19 @@ int wht_copy_rows(const void* src, void* dst, int64_t T, int32_t d, int dtype, v
     if (rc != WHT_OK) return rc;
     const long long elem = dtype == WHT_F32 ? 4 : 2;
     const long long n16 = static_cast<long long>(T) * d * elem / 16;
-    const long long want = ceil_div(n16, 256);
-    const long long cap = static_cast<long long>(sms) * 8;
-    copy_rows_kernel<<<static_cast<unsigned>(want < cap ? want : cap), 256, 0,
-                       static_cast<cudaStream_t>(stream)>>>(
+    copy_rows_kernel<<<capped_grid(ceil_div(n16, 256), sms, 8), 256, 0, static_cast<cudaStream_t>(stream)>>>(
         static_cast<const uint4*>(src), static_cast<uint4*>(dst), n16);
     WHT_CUDA_TRY(cudaGetLastError());
     return WHT_OK;
+}
+
+int wht_affine_device_status(void) {
+    unsigned int flag = 0;
+    WHT_CUDA_TRY(cudaMemcpyFromSymbol(&flag, g_wht_device_error, sizeof(flag)));
+    if (flag == 0) return WHT_OK;
+    const unsigned int zero = 0;
+    WHT_CUDA_TRY(cudaMemcpyToSymbol(g_wht_device_error, &zero, sizeof(zero)));
+    return WHT_ERR_DEVICE_WAIT;
 }
 
 int wht_affine_last_cuda_error(void) { return g_last_cuda_error; }
@@ -428,6 +527,8 @@ const char* wht_affine_status_string(int status) {
         case WHT_ERR_WORKSPACE: return "WHT_ERR_WORKSPACE: scratch buffer missing, too small or not allocatable";
         case WHT_ERR_CUDA: return "WHT_ERR_CUDA: a CUDA runtime call failed";
         case WHT_ERR_BAD_VARIANT: return "WHT_ERR_BAD_VARIANT: unknown kernel variant";
+        case WHT_ERR_DEVICE_WAIT:
+            return "WHT_ERR_DEVICE_WAIT: a kernel gave up waiting for an async copy; that launch's results are invalid";
         default: return "unknown wht_status";
     }
 }

@@ -17,7 +17,7 @@ from paper_2603_08343_b200 import workloads as wl
 
 pytestmark = pytest.mark.gpu
 
-VARIANTS = [1, 2]  # 1 = butterfly family, 2 = tensor-core assisted (falls back to 1 where unsupported)
+VARIANTS = [1, 2, 3]  # butterfly; tensor-core assisted with direct loads; with streamed rows (each falls back where unsupported)
 
 
 @pytest.fixture(scope="module")
@@ -27,6 +27,7 @@ def B():
     from paper_2603_08343_b200 import binding
     yield binding
     binding.wht_affine_set_variant(0)
+    binding.wht_affine_device_status()  # raises if any kernel's bounded wait expired during the module
 
 
 def _check_fwd(w, y_gpu, x_cpu, a_cpu, b_cpu, what):
@@ -282,6 +283,16 @@ def test_heavy_tailed_rows(B):
     for variant in VARIANTS:
         w = wl.CONFIGS["large"].with_rows(48)
         _run_case(B, w, variant)
+
+
+def test_streamed_kernels_on_many_rows(B):
+    # enough rows that every row group loops through its ring several times, ragged tail
+    B.wht_affine_set_variant(3)
+    for d, dtype, T in [(512, wl.WHT_BF16, 9001), (1024, wl.WHT_BF16, 20011), (2048, wl.WHT_BF16_PF32, 9973),
+                        (4096, wl.WHT_BF16, 3001), (8192, wl.WHT_BF16_PF32, 1501)]:
+        w = wl.Workload("stream", T, d, dtype, "normal", 300 + d, True, "")
+        _run_case(B, w, 3)
+    B.wht_affine_device_status()
 
 
 def test_copy_rows(B):
