@@ -97,7 +97,8 @@ struct MmaGeo {
     static constexpr int RG = RG_;             // rows in flight per CTA
     static constexpr int GROUP_THREADS = W * 32;
     static constexpr int THREADS = RG * GROUP_THREADS;
-    static constexpr int XCHG_FLOATS = WB > 0 ? 2 * D : 0;  // per row group (double buffer)
+    static constexpr int XCHG_ONE = (W - 1) * NT * 256;     // floats that change owner in one exchange
+    static constexpr int XCHG_FLOATS = 2 * XCHG_ONE;        // per row group (two buffers, used alternately)
     static constexpr int SMEM_FWD = RG * XCHG_FLOATS * 4;
     static constexpr int SMEM_BWD = imax_c(RG * XCHG_FLOATS * 4, RG * D * 4);
 };
@@ -195,30 +196,41 @@ struct MmaXform {
         }
     }
 
-    // Swap the warp bits with the top WB chunk-slot bits through shared memory
-    // (layout A -> B when FROM_A, else B -> A) and finish those stages in registers.
-    template <bool FROM_A>
+    // Swap the warp bits with the top WB chunk-slot bits through shared memory and
+    // finish those stages in registers.  Slot (top, rest) of warp w moves to warp
+    // `top`, slot (w, rest): a transpose of the (warp, top) grid, the same in both
+    // directions (layout A -> B and B -> A); slots with top == w stay where they are
+    // and are not copied.  xbuf holds XCHG_ONE floats.
     static __device__ __forceinline__ void exchange_and_top(F2 (&v)[NT][4], float* xbuf, int w, int lane,
                                                             int barrier_id) {
         if constexpr (Geo::WB > 0) {
+            constexpr int W = Geo::W, NREST = Geo::NREST;
+            // compact position of the block sent from warp `src` to warp `dst` (src != dst)
+            auto block_of = [](int src, int dst, int rest) {
+                return ((src * (W - 1) + dst - (dst > src ? 1 : 0)) * NREST + rest) * 256;
+            };
 #pragma unroll
             for (int idx = 0; idx < NT; ++idx) {
-                const int c = chunk_of<Geo, !FROM_A>(w, idx);
-                float4* p = reinterpret_cast<float4*>(xbuf + c * 256 + lane * 4);
-                p[0] = make_float4(v[idx][0].x, v[idx][0].y, v[idx][1].x, v[idx][1].y);
-                p[32] = make_float4(v[idx][2].x, v[idx][2].y, v[idx][3].x, v[idx][3].y);
+                const int top = idx / NREST, rest = idx % NREST;
+                if (top != w) {
+                    float4* p = reinterpret_cast<float4*>(xbuf + block_of(w, top, rest) + lane * 4);
+                    p[0] = make_float4(v[idx][0].x, v[idx][0].y, v[idx][1].x, v[idx][1].y);
+                    p[32] = make_float4(v[idx][2].x, v[idx][2].y, v[idx][3].x, v[idx][3].y);
+                }
             }
             named_barrier(barrier_id, Geo::GROUP_THREADS);
 #pragma unroll
             for (int idx = 0; idx < NT; ++idx) {
-                const int c = chunk_of<Geo, FROM_A>(w, idx);
-                const float4* p = reinterpret_cast<const float4*>(xbuf + c * 256 + lane * 4);
-                const float4 q0 = p[0], q1 = p[32];
-                v[idx][0] = f2(q0.x, q0.y); v[idx][1] = f2(q0.z, q0.w);
-                v[idx][2] = f2(q1.x, q1.y); v[idx][3] = f2(q1.z, q1.w);
+                const int top = idx / NREST, rest = idx % NREST;
+                if (top != w) {
+                    const float4* p = reinterpret_cast<const float4*>(xbuf + block_of(top, w, rest) + lane * 4);
+                    const float4 q0 = p[0], q1 = p[32];
+                    v[idx][0] = f2(q0.x, q0.y); v[idx][1] = f2(q0.z, q0.w);
+                    v[idx][2] = f2(q1.x, q1.y); v[idx][3] = f2(q1.z, q1.w);
+                }
             }
 #pragma unroll
-            for (int bit = Geo::NREST; bit < NT; bit <<= 1) {
+            for (int bit = NREST; bit < NT; bit <<= 1) {
 #pragma unroll
                 for (int idx = 0; idx < NT; ++idx) {
                     if ((idx & bit) == 0) {
@@ -340,7 +352,7 @@ mma_fwd_kernel(const __nv_bfloat16* x, const TP* __restrict__ a, const TP* __res
         X::pass1_raw(raw, m, hf);
         X::mid_stages(m);
         X::pass2(m, v, hf);
-        X::template exchange_and_top<true>(v, xbuf + parity * Geo::D, w, lane, 1 + rg);
+        X::exchange_and_top(v, xbuf + parity * Geo::XCHG_ONE, w, lane, 1 + rg);
         parity ^= 1;
         uint4* dst = reinterpret_cast<uint4*>(y + row * Geo::D);
 #pragma unroll
@@ -396,7 +408,7 @@ mma_bwd_kernel(const __nv_bfloat16* dy, const __nv_bfloat16* x, const TP* __rest
         X::pass1_raw(raw, m, hf);
         X::mid_stages(m);
         X::pass2(m, v, hf);
-        X::template exchange_and_top<true>(v, xbuf, w, lane, 1 + rg);
+        X::exchange_and_top(v, xbuf, w, lane, 1 + rg);
         // da, db partial sums and g = a (.) dy, all in layout B
 #pragma unroll
         for (int idx = 0; idx < NT; ++idx) {
@@ -411,7 +423,7 @@ mma_bwd_kernel(const __nv_bfloat16* dy, const __nv_bfloat16* x, const TP* __rest
         X::pass1_f32(v, m, hf);
         X::mid_stages(m);
         X::pass2(m, v, hf);
-        X::template exchange_and_top<false>(v, xbuf + Geo::D, w, lane, 1 + rg);
+        X::exchange_and_top(v, xbuf + Geo::XCHG_ONE, w, lane, 1 + rg);
         uint4* dst = reinterpret_cast<uint4*>(dx + row * Geo::D);
 #pragma unroll
         for (int idx = 0; idx < NT; ++idx)

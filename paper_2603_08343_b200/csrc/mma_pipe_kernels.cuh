@@ -172,7 +172,7 @@ mma_fwd_pipe_kernel(const __nv_bfloat16* x, const TP* __restrict__ a, const TP* 
         }
         X::mid_stages(m);
         X::pass2(m, v, hf);
-        X::template exchange_and_top<true>(v, xbuf + parity * Geo::D, w, lane, 1 + rg);
+        X::exchange_and_top(v, xbuf + parity * Geo::XCHG_ONE, w, lane, 1 + rg);
         parity ^= 1;
         if constexpr (Geo::WB > 0) {
             // every warp of the row group has passed the exchange barrier, each after
@@ -260,7 +260,7 @@ mma_bwd_pipe_kernel(const __nv_bfloat16* dy, const __nv_bfloat16* x, const TP* _
         X::pass1_raw(raw, m, hf);
         X::mid_stages(m);
         X::pass2(m, v, hf);
-        X::template exchange_and_top<true>(v, xbuf, w, lane, 1 + rg);
+        X::exchange_and_top(v, xbuf, w, lane, 1 + rg);
         // da, db partial sums and g = a (.) dy, all in layout B
 #pragma unroll
         for (int idx = 0; idx < NT; ++idx) {
@@ -278,7 +278,7 @@ mma_bwd_pipe_kernel(const __nv_bfloat16* dy, const __nv_bfloat16* x, const TP* _
         }
         X::mid_stages(m);
         X::pass2(m, v, hf);
-        X::template exchange_and_top<false>(v, xbuf + Geo::D, w, lane, 1 + rg);
+        X::exchange_and_top(v, xbuf + Geo::XCHG_ONE, w, lane, 1 + rg);
         if constexpr (Geo::WB > 0) {
             if (elected && next_row < T) issue(stage, next_row);
         }

@@ -309,7 +309,7 @@ int dispatch_mma_fwd(int logd, bool few_rows, bool streamed, const FwdArgs& f, c
             case 10: return launch_mma_fwd_pipe<10, 2, 8, 4, 3, TP>(f, c);
             case 11: return launch_mma_fwd_pipe<11, 3, 8, 3, 2, TP>(f, c);
             case 12: return launch_mma_fwd_pipe<12, 3, 2, 3, 2, TP>(f, c);
-            case 13: return launch_mma_fwd_pipe<13, 3, 1, 3, 2, TP>(f, c);
+            case 13: return launch_mma_fwd_pipe<13, 3, 2, 2, 1, TP>(f, c);
         }
     }
     return WHT_ERR_BAD_DIM;
@@ -329,8 +329,8 @@ int dispatch_mma_bwd(int logd, bool streamed, const BwdArgs& g, const Ctx& c) {
         switch (logd) {
             case 9: return launch_mma_bwd_pipe<9, 1, 8, 4, 2, TP>(g, c);
             case 10: return launch_mma_bwd_pipe<10, 2, 8, 3, 2, TP>(g, c);
-            case 11: return launch_mma_bwd_pipe<11, 2, 4, 3, 2, TP>(g, c);
-            case 12: return launch_mma_bwd_pipe<12, 2, 2, 3, 1, TP>(g, c);
+            case 11: return launch_mma_bwd_pipe<11, 2, 4, 2, 2, TP>(g, c);
+            case 12: return launch_mma_bwd_pipe<12, 2, 2, 2, 1, TP>(g, c);
             case 13: return launch_mma_bwd_pipe<13, 3, 1, 2, 1, TP>(g, c);
         }
     }
