@@ -33,6 +33,7 @@ if ROOT not in sys.path:
 import numpy as np
 import torch
 
+from paper_2603_08343_b200 import dp
 from paper_2603_08343_b200 import workloads as wl
 
 METRIC = "wht_affine_tokens_per_s_fwd_bwd"
@@ -313,6 +314,8 @@ def run_ours(args, rank: int, world: int, local_rank: int):
 
     hbm_peak, peak_src = load_peaks()
     w = wl.CONFIGS[args.workload]
+    if args.rows:
+        w = w.with_rows(args.rows)  # a smaller case of the same kernels (profiler captures)
     # every rank draws its own rows (weak scaling): the seed is offset by the rank
     wr = wl.Workload(w.name, w.T, w.d, w.dtype, w.dist, w.seed + 1000 * rank, w.has_bwd, w.note)
     base_rows = min(w.T, 8192) if w.dist != "normal" else w.T
@@ -325,9 +328,8 @@ def run_ours(args, rank: int, world: int, local_rank: int):
     dy = dy_h.cuda().repeat(reps, 1) if w.has_bwd else None
     y = torch.empty_like(x)
     dx = torch.empty_like(x) if w.has_bwd else None
-    da = torch.empty(w.d, dtype=torch.float32, device="cuda")
-    db = torch.empty_like(da)
-    grads = torch.empty(2 * w.d, dtype=torch.float32, device="cuda")
+    bucket = dp.GradBucket(w.d, device="cuda")  # da|db, contiguous: one all-reduce per step
+    da, db = bucket.da, bucket.db
 
     # small working sets are rotated through enough buffers to exceed L2 (126 MB)
     step_bytes = (4 if w.has_bwd else 2) * w.T * w.d * w.io_bytes
@@ -355,10 +357,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
             B.wht_affine_bwd(dys[i], xs[i], a, dxs[i], da, db, w.T, w.d, w.dtype)
             if ev is not None:
                 ev[2].record()
-            if world > 1:
-                grads[:w.d].copy_(da)
-                grads[w.d:].copy_(db)
-                dist.all_reduce(grads)
+            bucket.all_reduce()  # the path's only exchange; nothing to do on one rank
 
     for _ in range(max(args.warmup, 3)):
         step()
@@ -492,6 +491,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--variant", type=int, default=0)
     ap.add_argument("--no-sections", action="store_true")
+    ap.add_argument("--rows", type=int, default=0,
+                    help="override the workload's row count (small cases for profiler captures; "
+                         "not the benchmark configuration)")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))

@@ -138,14 +138,3 @@ def gen_params(w: Workload):
     a = torch.rand(w.d, generator=ga, dtype=torch.float32) + 0.5
     b = torch.randn(w.d, generator=gb, dtype=torch.float32) * 0.1
     return a.to(w.param_torch_dtype), b.to(w.param_torch_dtype)
-
-
-def shard_rows(T: int, world_size: int, rank: int):
-    """Contiguous row range [r0, r1) of rank `rank` when T rows are split over ranks.
-
-    Rows are independent, so data parallelism is a plain partition; the first
-    T % world_size ranks take one extra row.
-    """
-    base, extra = divmod(T, world_size)
-    r0 = rank * base + min(rank, extra)
-    return r0, r0 + base + (1 if rank < extra else 0)

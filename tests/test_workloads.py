@@ -38,8 +38,9 @@ def test_distributions():
 
 
 def test_shard_rows_partition():
+    from paper_2603_08343_b200 import dp
     for T, n in [(10, 3), (65536, 8), (7, 8), (0, 2)]:
-        spans = [wl.shard_rows(T, n, r) for r in range(n)]
+        spans = [dp.shard_rows(T, n, r) for r in range(n)]
         assert spans[0][0] == 0 and spans[-1][1] == T
         assert all(spans[i][1] == spans[i + 1][0] for i in range(n - 1))
         sizes = [b - a for a, b in spans]
