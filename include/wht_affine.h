@@ -107,6 +107,39 @@ int wht_affine_bwd_ws(const void* dy, const void* x, const void* a,
                       int64_t T, int32_t d, int dtype,
                       void* workspace, size_t workspace_bytes, void* stream);
 
+/*
+ * Backward pass for callers that must not allocate.  (The paper has no counterpart:
+ * this entry point exists for the library's users, not for the method.)
+ *
+ * Some callers cannot let a library call cudaMalloc on their behalf: code running
+ * inside a memory-pool or caching-allocator regime where every byte of device
+ * memory is already spoken for, real-time or serving loops where an allocation
+ * (which synchronises the device) would stall other streams, and set-ups that
+ * forbid the call outright once initialisation is over.  wht_affine_bwd allocates
+ * its scratch lazily and wht_affine_bwd_ws makes the caller find the memory; this
+ * variant needs neither.  Its scratch is a fixed array compiled into the library's
+ * device image, WHT_NOALLOC_SCRATCH_BYTES (16 MiB) large, which every GPU that
+ * loads the library holds until the process exits.  Same arguments, semantics and
+ * bit-identical results as wht_affine_bwd.
+ *
+ *   - Never calls cudaMalloc, cudaFree or any allocating routine.
+ *   - A problem whose scratch need, wht_affine_bwd_workspace_bytes(T, d, dtype),
+ *     exceeds WHT_NOALLOC_SCRATCH_BYTES is rejected with WHT_ERR_WORKSPACE and
+ *     nothing is launched (on a 148-SM part every d <= 8192 fits for any T).
+ *   - The first call on each device looks up the array's device address (one
+ *     cudaGetSymbolAddress, no allocation) and caches it; make that first call
+ *     outside any stream capture.
+ *   - All calls on a device share the one array.  The kernels overwrite every
+ *     scratch word they later read, so nothing needs clearing between calls and
+ *     stale contents from an earlier call are harmless; but two of these calls
+ *     that overlap on the GPU (different streams, no ordering) race on it and
+ *     give wrong da/db.  Serialise them, or use wht_affine_bwd_ws.
+ */
+#define WHT_NOALLOC_SCRATCH_BYTES (16u * 1024u * 1024u)
+int wht_affine_bwd_noalloc(const void* dy, const void* x, const void* a,
+                           void* dx, float* da, float* db,
+                           int64_t T, int32_t d, int dtype, void* stream);
+
 /* Scratch bytes wht_affine_bwd_ws needs on the current device (0 on bad arguments). */
 size_t wht_affine_bwd_workspace_bytes(int64_t T, int32_t d, int dtype);
 

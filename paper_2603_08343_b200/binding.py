@@ -18,7 +18,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libwht_affine.so")
 
 EXPORTS = (
-    "wht_affine_fwd", "wht_affine_fwd_decode", "wht_affine_bwd", "wht_affine_bwd_ws",
+    "wht_affine_fwd", "wht_affine_fwd_decode", "wht_affine_bwd", "wht_affine_bwd_ws", "wht_affine_bwd_noalloc",
     "wht_affine_bwd_workspace_bytes", "wht_affine_set_variant", "wht_affine_get_variant",
     "wht_copy_rows", "wht_affine_device_status", "wht_affine_last_cuda_error", "wht_affine_status_string",
     "wht_affine_shutdown",
@@ -43,6 +43,7 @@ def _load() -> ctypes.CDLL:
     lib.wht_affine_fwd.argtypes = [vp, vp, vp, vp, i64, i32, ci, vp]
     lib.wht_affine_fwd_decode.argtypes = [vp, vp, vp, vp, i64, i32, ci, vp]
     lib.wht_affine_bwd.argtypes = [vp, vp, vp, vp, vp, vp, i64, i32, ci, vp]
+    lib.wht_affine_bwd_noalloc.argtypes = [vp, vp, vp, vp, vp, vp, i64, i32, ci, vp]
     lib.wht_affine_bwd_ws.argtypes = [vp, vp, vp, vp, vp, vp, i64, i32, ci, vp, sz, vp]
     lib.wht_affine_bwd_workspace_bytes.argtypes = [i64, i32, ci]
     lib.wht_affine_bwd_workspace_bytes.restype = sz
@@ -114,6 +115,19 @@ def wht_affine_bwd_ws(dy, x, a, dx, da, db, T: int, d: int, dtype: int, workspac
     nbytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
     _check(_lib.wht_affine_bwd_ws(_ptr(dy), _ptr(x), _ptr(a), _ptr(dx), _ptr(da), _ptr(db), T, d, dtype,
                                   _ptr(workspace), nbytes, _stream(stream)), "wht_affine_bwd_ws")
+
+
+def wht_affine_bwd_noalloc(dy, x, a, dx, da, db, T: int, d: int, dtype: int, stream=None) -> None:
+    """Backward pass that never allocates: its scratch is a fixed 16 MiB array inside the library.
+
+    For callers that cannot let a library call cudaMalloc (a pool that owns all device
+    memory, latency-critical loops, allocation banned after start-up).  Same results as
+    wht_affine_bwd; raises WhtError(WHT_ERR_WORKSPACE) when the problem needs more scratch
+    than the array holds.  Calls on one device share the array: do not overlap them.
+    """
+    _require_cuda(dy, x, a, dx, da, db)
+    _check(_lib.wht_affine_bwd_noalloc(_ptr(dy), _ptr(x), _ptr(a), _ptr(dx), _ptr(da), _ptr(db), T, d, dtype,
+                                       _stream(stream)), "wht_affine_bwd_noalloc")
 
 
 def wht_affine_bwd_workspace_bytes(T: int, d: int, dtype: int) -> int:

@@ -398,6 +398,24 @@ int check_bwd_args(const void* dy, const void* x, const void* a, void* dx, float
     return WHT_OK;
 }
 
+// Scratch of wht_affine_bwd_noalloc: part of the device image, so no call ever
+// allocates it.  In host code this name is only a handle for the runtime -- the
+// device address comes from cudaGetSymbolAddress, once per device.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[WHT_NOALLOC_SCRATCH_BYTES];
+void* g_noalloc_scratch_ptr[kMaxDevices] = {};
+
+int noalloc_scratch_for_current_device(int dev, void** out) {
+    std::lock_guard<std::mutex> lock(g_mutex);
+    if (g_noalloc_scratch_ptr[dev] == nullptr) {
+        void* p = nullptr;
+        WHT_CUDA_TRY(cudaGetSymbolAddress(&p, g_noalloc_scratch));  // address on the CURRENT device
+        if (p == nullptr) return WHT_ERR_WORKSPACE;
+        g_noalloc_scratch_ptr[dev] = p;
+    }
+    *out = g_noalloc_scratch_ptr[dev];
+    return WHT_OK;
+}
+
 int query_bwd_bytes(int64_t T, int32_t d, int dtype, size_t* need) {
     BwdArgs q{nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, 0, true, need};
     return run_bwd(q, T, d, dtype, nullptr);
@@ -477,6 +495,24 @@ int wht_affine_bwd(const void* dy, const void* x, const void* a, void* dx, float
         ws_bytes = st.scratch_bytes;
     }
     BwdArgs g{dy, x, a, dx, da, db, ws, ws_bytes, false, &need};
+    return run_bwd(g, T, d, dtype, static_cast<cudaStream_t>(stream));
+}
+
+int wht_affine_bwd_noalloc(const void* dy, const void* x, const void* a, void* dx, float* da, float* db,
+                           int64_t T, int32_t d, int dtype, void* stream) {
+    int rc = check_bwd_args(dy, x, a, dx, da, db, T, d, dtype);
+    if (rc != WHT_OK) return rc;
+    size_t need = 0;
+    rc = query_bwd_bytes(T, d, dtype, &need);
+    if (rc != WHT_OK) return rc;
+    if (need > WHT_NOALLOC_SCRATCH_BYTES) return WHT_ERR_WORKSPACE;  // beyond the built-in array
+    int dev = 0, sms = 0;
+    rc = current_device(&dev, &sms);
+    if (rc != WHT_OK) return rc;
+    void* ws = nullptr;
+    rc = noalloc_scratch_for_current_device(dev, &ws);
+    if (rc != WHT_OK) return rc;
+    BwdArgs g{dy, x, a, dx, da, db, ws, WHT_NOALLOC_SCRATCH_BYTES, false, &need};
     return run_bwd(g, T, d, dtype, static_cast<cudaStream_t>(stream));
 }
 
