@@ -145,13 +145,16 @@ size_t wht_affine_bwd_workspace_bytes(int64_t T, int32_t d, int dtype);
 
 /*
  * Kernel family used by the three compute calls (for A/B measurements):
- *   0 = automatic (default): tensor-core assisted kernels for bf16 rows with
- *       512 <= d <= 8192 (rows streamed through a shared-memory ring when there
- *       are many, loaded directly when there are few), butterfly otherwise;
+ *   0 = automatic (default): for bf16 rows, the tcgen05 kernels when there are many
+ *       rows and 1024 <= d <= 8192 (backward: <= 4096), else the mma.sync kernels
+ *       for 512 <= d <= 8192 (rows streamed through a shared-memory ring when there
+ *       are many, loaded directly when there are few); butterfly otherwise;
  *   1 = butterfly (registers + warp shuffles + shared memory), every d and dtype;
- *   2 = tensor-core assisted with direct row loads;
- *   3 = tensor-core assisted with streamed rows.
- * A variant that does not support the requested (d, dtype) falls back to 1.
+ *   2 = mma.sync tensor-core assisted with direct row loads;
+ *   3 = mma.sync tensor-core assisted with streamed rows;
+ *   4 = tcgen05: rows copied into shared memory as they are and multiplied by H_128
+ *       on the tensor core (accumulators in tensor memory), the rest in registers.
+ * A variant that does not support the requested (d, dtype) falls back (4 -> 3 -> 1).
  * Process-wide; not meant to be changed while calls are in flight.
  */
 int wht_affine_set_variant(int variant);

@@ -1,0 +1,722 @@
+// tcgen05 kernel family for bf16 rows, d = 1024 * PIECES (1024 ... 8192), many rows.
+//
+// H_d = H_2 (x) ... (x) H_2 acts on the index bits independently, so the seven
+// stages on index bits 3..9 are one product with H_128.  A row piece of 1024
+// contiguous bf16 elements is, as it lies in memory, a 128 x 8 matrix
+// B[k][n] = x[k*8 + n]   (k = bits 3..9, n = bits 0..2, n contiguous: 16 bytes per k),
+// which is exactly the canonical un-swizzled "MN-major" shared-memory operand
+// layout of tcgen05.mma (core matrix = 8 k-values x 16 bytes = 128 contiguous
+// bytes; next 8 k-values 128 bytes on; next 8 columns = next piece, 2048 bytes on).
+// So a tile of consecutive rows is copied into shared memory AS IT IS by one bulk
+// async copy and handed to the tensor core without passing through registers:
+//
+//     D[m][n'] = sum_k H_128[m][k] * B[k][n']        (bf16 x +-1, fp32 accumulate in TMEM)
+//
+// with n' = (row in tile, piece, n): N = 128 columns = 16 pieces = 32 KiB of rows.
+// Products with +-1 are exact, so this is fp32 accumulation of the stored values.
+// TMEM lane m (= thread m of the 128-thread epilogue group) then holds, for every
+// row of the tile, the values whose index bits 3..9 equal m: bits 0..2 and the
+// piece bits are all in that thread's registers, so the remaining stages are plain
+// register butterflies with no exchange between threads at all, and the thread
+// ends up with 8 contiguous output elements per piece: one 128-bit store, a warp
+// writes 512 contiguous bytes.
+//
+// Roles in a CTA of 10 warps (one CTA per SM, persistent over tiles):
+//   warp 0, lane 0   producer: cp.async.bulk of each tile into a shared-memory ring
+//   warp 1, lane 0   issues tcgen05.mma (8 instructions of K = 16 per product) and
+//                    tcgen05.commit onto mbarriers
+//   warps 2..9       epilogue: tcgen05.ld, register stages, affine, stores; each warp
+//                    owns TMEM lanes 32*(warp % 4) .. +31 and one half of the columns
+//
+// The backward pass runs two products per tile: D1 = H_128 X (for da) and
+// D2 = H_128 G, where G = (a/sqrt(d)) (.) dy after ITS register stages, written back
+// into the ring slot as bf16 hi + lo (two products into one accumulator; the pair
+// carries 16-17 significant bits, and the accumulation is again fp32).
+//
+// Every wait on an mbarrier is bounded.  A wait that expires raises a CTA-wide abort
+// flag and the device status word; every role then leaves its loop, copies in flight
+// are waited for (bounded), TMEM is freed and the kernel returns: a fault in the
+// pipeline shows up as WHT_ERR_DEVICE_WAIT on the host, never as a hang.
+// No copy uses cluster multicast; every source is this GPU's own memory.
+#pragma once
+#include "mma_pipe_kernels.cuh"
+
+namespace wht {
+
+// ---- tcgen05 / TMEM wrappers ---------------------------------------------------------
+__device__ __forceinline__ void tmem_alloc(uint32_t* slot, uint32_t ncols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(slot)),
+                 "r"(ncols)
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t base, uint32_t ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(base), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() {
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_after() {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+}
+// D(tmem) (+)= A(smem desc) * B(smem desc), bf16 operands, fp32 accumulator
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                          uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// mbarrier arrive once all tcgen05 operations issued so far by this thread are complete
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+// 16 consecutive columns of this thread's TMEM lane
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
+    uint32_t r[16];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr)
+        : "memory");
+#pragma unroll
+    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void tmem_ld8(uint32_t taddr, float* v) {
+    uint32_t r[8];
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+                 : "r"(taddr)
+                 : "memory");
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[i]);
+}
+template <int COLS>
+__device__ __forceinline__ void tmem_ld_cols(uint32_t taddr, float (&v)[COLS]) {
+    if constexpr (COLS % 16 == 0) {
+#pragma unroll
+        for (int c = 0; c < COLS; c += 16) tmem_ld16(taddr + c, v + c);
+    } else {
+#pragma unroll
+        for (int c = 0; c < COLS; c += 8) tmem_ld8(taddr + c, v + c);
+    }
+}
+
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+// make this thread's shared-memory writes visible to the async proxy (tensor core reads)
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+// Bounded wait that also gives up as soon as another role has raised the abort flag.
+__device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag) {
+    for (uint32_t i = 0; i < (1u << 22); ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (i > 16) {
+            if (*abort_flag) return false;
+            __nanosleep(32);
+        }
+    }
+    *abort_flag = 1;
+    atomicExch(&g_wht_device_error, kDeviceErrWaitExpired);
+    return false;
+}
+
+// The same for a whole warp: every lane polls (and so observes the barrier itself), the
+// verdict is made uniform so that the .sync.aligned tcgen05 instructions that follow are
+// reached by all 32 lanes together or not at all.
+__device__ __forceinline__ bool warp_wait_or_abort(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag) {
+    const bool ok = wait_or_abort(bar, parity, abort_flag);
+    return __all_sync(kFullMask, ok);
+}
+
+// Shared-memory matrix descriptor: no swizzle, 128 bytes between core matrices along K,
+// 2048 bytes between core matrices along M/N.  Valid for both operands used here.
+__device__ __forceinline__ uint64_t umma_smem_desc(uint32_t smem_addr) {
+    uint64_t d = static_cast<uint64_t>((smem_addr & 0x3FFFFu) >> 4);
+    d |= static_cast<uint64_t>(128 >> 4) << 16;   // leading-dimension byte offset
+    d |= static_cast<uint64_t>(2048 >> 4) << 32;  // stride-dimension byte offset
+    d |= static_cast<uint64_t>(1) << 46;          // descriptor version of this architecture
+    return d;
+}
+// Instruction descriptor: bf16 x bf16 -> fp32, A K-major, B MN-major, M = 128, N columns.
+__host__ __device__ constexpr uint32_t umma_idesc(int n) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | (static_cast<uint32_t>(n >> 3) << 17) |
+           (static_cast<uint32_t>(128 >> 4) << 24);
+}
+
+template <int LOGD, int NCOL_>
+struct UmmaGeo {
+    static constexpr int D = 1 << LOGD;
+    static constexpr int PIECES = D / 1024;
+    static constexpr int R = 8 * PIECES;             // values of one row held by one thread
+    static constexpr int N = NCOL_;                  // accumulator columns per tile
+    static constexpr int ROWS = N / R;               // rows per tile
+    static constexpr int TILE_BYTES = N * 256;       // = ROWS * D * 2
+    static constexpr int H_BYTES = 128 * 128 * 2;
+    static constexpr int EPI_WARPS = 8;
+    static constexpr int THREADS = 32 * (2 + EPI_WARPS);
+    static constexpr int CPW = N / 2;                // columns per epilogue warp
+    static constexpr int RPW = CPW / R;              // rows per epilogue warp and tile
+    static_assert(PIECES >= 1 && RPW >= 1 && N % 16 == 0 && N <= 256, "unsupported tile");
+};
+
+// H_128 as the A operand (K-major, un-swizzled): element (m, k) at byte
+// (m/8)*2048 + (k/8)*128 + (m%8)*16 + (k%8)*2; +-1 are exact in bf16.
+__device__ __forceinline__ void write_h128(unsigned char* dst, int tid, int nthreads) {
+    for (int c = tid; c < 2048; c += nthreads) {
+        const int m = ((c >> 7) << 3) | (c & 7);
+        const int k0 = ((c >> 3) & 15) << 3;
+        uint32_t w[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const uint32_t lo = (__popc(m & (k0 + 2 * j)) & 1) ? 0xBF80u : 0x3F80u;
+            const uint32_t hi = (__popc(m & (k0 + 2 * j + 1)) & 1) ? 0xBF80u : 0x3F80u;
+            w[j] = lo | (hi << 16);
+        }
+        *reinterpret_cast<uint4*>(dst + c * 16) = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+}
+
+// Stages on the index bits a thread holds: v[piece*8 + n], n = bits 0..2.
+// Bit 0 pairs neighbours inside a register pair (scalar), the rest are packed.
+template <int R>
+__device__ __forceinline__ void thread_stages(float (&v)[R]) {
+#pragma unroll
+    for (int i = 0; i < R; i += 2) {
+        const float lo = v[i], hi = v[i + 1];
+        v[i] = lo + hi;
+        v[i + 1] = lo - hi;
+    }
+#pragma unroll
+    for (int s = 2; s < R; s <<= 1) {
+#pragma unroll
+        for (int i = 0; i < R; i += 2) {
+            if ((i & s) == 0) {
+                F2 lo = f2(v[i], v[i + 1]), hi = f2(v[i + s], v[i + s + 1]);
+                bfly2(lo, hi);
+                v[i] = lo.x; v[i + 1] = lo.y;
+                v[i + s] = hi.x; v[i + s + 1] = hi.y;
+            }
+        }
+    }
+}
+
+// ---- forward ---------------------------------------------------------------------------
+template <int LOGD, int NCOL, int STAGES, typename TP>
+struct UmmaFwdSmem {
+    using Geo = UmmaGeo<LOGD, NCOL>;
+    static constexpr int ACC = 512 / NCOL > 4 ? 4 : 512 / NCOL;          // accumulator buffers in TMEM
+    static constexpr int TMEM_COLS = ACC * NCOL <= 256 ? 256 : 512;
+    static constexpr bool PARAMS_IN_SMEM = Geo::R > 32;
+    static constexpr int OFF_H = 0;
+    static constexpr int OFF_RING = Geo::H_BYTES;
+    static constexpr int OFF_PARAMS = OFF_RING + STAGES * Geo::TILE_BYTES;
+    static constexpr int PARAM_BYTES = PARAMS_IN_SMEM ? 2 * Geo::D * 4 : 0;
+    static constexpr int OFF_BARS = OFF_PARAMS + PARAM_BYTES;
+    static constexpr int NBARS = 2 * STAGES + 2 * ACC;
+    static constexpr int OFF_MISC = OFF_BARS + NBARS * 8;
+    static constexpr int BYTES = OFF_MISC + 16;
+};
+
+// Per-channel vector in shared memory as fp32 for d = 8192, in the order threads read it:
+// float4 number ((piece*2 + half)*128 + m) holds elements piece*1024 + m*8 + half*4 .. +3.
+template <int D, typename TP>
+__device__ __forceinline__ void stage_params_umma(const TP* __restrict__ src, float* dst, float scale, int tid,
+                                                  int nthreads) {
+    for (int i = tid; i < D / 4; i += nthreads) {
+        const int e0 = i * 4, piece = e0 >> 10, m = (e0 & 1023) >> 3, half = (e0 & 7) >> 2;
+        float4 q;
+        if constexpr (sizeof(TP) == 4) {
+            q = __ldg(reinterpret_cast<const float4*>(src) + i);
+        } else {
+            const uint2 r = __ldg(reinterpret_cast<const uint2*>(src) + i);
+            q = make_float4(bf16lo_to_f32(r.x), bf16hi_to_f32(r.x), bf16lo_to_f32(r.y), bf16hi_to_f32(r.y));
+        }
+        reinterpret_cast<float4*>(dst)[(piece * 2 + half) * 128 + m] =
+            make_float4(q.x * scale, q.y * scale, q.z * scale, q.w * scale);
+    }
+}
+
+template <int LOGD, int NCOL, int STAGES, typename TP>
+__global__ void __launch_bounds__(UmmaGeo<LOGD, NCOL>::THREADS, 1)
+umma_fwd_kernel(const __nv_bfloat16* x, const TP* __restrict__ a, const TP* __restrict__ b, __nv_bfloat16* y,
+                long long T, float inv_sqrt_d) {
+    using Geo = UmmaGeo<LOGD, NCOL>;
+    using L = UmmaFwdSmem<LOGD, NCOL, STAGES, TP>;
+    constexpr int ACC = L::ACC;
+    extern __shared__ __align__(1024) unsigned char umma_smem[];
+    unsigned char* const smem_raw = umma_smem;
+    unsigned char* ring = smem_raw + L::OFF_RING;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem_raw + L::OFF_BARS);
+    uint64_t* full = bars;                   // [STAGES] tile landed in the ring
+    uint64_t* empty = bars + STAGES;         // [STAGES] product has consumed the ring slot
+    uint64_t* acc_full = bars + 2 * STAGES;  // [ACC] accumulator written
+    uint64_t* acc_empty = acc_full + ACC;    // [ACC] accumulator read out by all 8 epilogue warps
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem_raw + L::OFF_MISC);
+    volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem_raw + L::OFF_MISC + 4);
+
+    const int tid = threadIdx.x;
+    const int warp = tid >> 5;
+    const int lane = tid & 31;
+    const long long tiles = (T + Geo::ROWS - 1) / Geo::ROWS;
+    const long long my_tiles = blockIdx.x < tiles ? (tiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+
+    if (tid == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(full + s, 1); mbar_init(empty + s, 1); }
+        for (int t = 0; t < ACC; ++t) { mbar_init(acc_full + t, 1); mbar_init(acc_empty + t, Geo::EPI_WARPS); }
+        *abort_flag = 0;
+        fence_mbar_init();
+    }
+    write_h128(smem_raw + L::OFF_H, tid, Geo::THREADS);
+    if constexpr (L::PARAMS_IN_SMEM) {
+        float* pa = reinterpret_cast<float*>(smem_raw + L::OFF_PARAMS);
+        stage_params_umma<Geo::D>(a, pa, inv_sqrt_d, tid, Geo::THREADS);
+        stage_params_umma<Geo::D>(b, pa + Geo::D, 1.0f, tid, Geo::THREADS);
+    }
+    fence_async_smem();  // H_128 was written by ordinary stores and is read by the tensor core
+    if (warp == 1) {
+        tmem_alloc(tmem_slot, L::TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            long long it = 0;
+            for (; it < my_tiles; ++it) {
+                const int s = static_cast<int>(it % STAGES);
+                const uint32_t ph = static_cast<uint32_t>(it / STAGES) & 1u;
+                if (!wait_or_abort(empty + s, ph ^ 1u, abort_flag)) break;
+                const long long tile = blockIdx.x + it * gridDim.x;
+                const long long row0 = tile * Geo::ROWS;
+                const long long rows = T - row0 < Geo::ROWS ? T - row0 : Geo::ROWS;
+                const uint32_t bytes = static_cast<uint32_t>(rows) * Geo::D * 2;
+                mbar_expect_tx(full + s, bytes);
+                bulk_load(ring + s * Geo::TILE_BYTES, x + row0 * Geo::D, bytes, full + s);
+            }
+            if (*abort_flag) {
+                // copies already issued still land in shared memory: wait for them before leaving
+                const long long lo = it > STAGES ? it - STAGES : 0;
+                for (long long j = lo; j < it; ++j)
+                    mbar_wait_bounded(full + (j % STAGES), static_cast<uint32_t>(j / STAGES) & 1u);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            const uint64_t adesc = umma_smem_desc(smem_u32(smem_raw + L::OFF_H));
+            constexpr uint32_t idesc = umma_idesc(Geo::N);
+            for (long long it = 0; it < my_tiles; ++it) {
+                const int s = static_cast<int>(it % STAGES);
+                const uint32_t ph = static_cast<uint32_t>(it / STAGES) & 1u;
+                const int t = static_cast<int>(it % ACC);
+                const uint32_t pt = static_cast<uint32_t>(it / ACC) & 1u;
+                if (!wait_or_abort(full + s, ph, abort_flag)) break;
+                if (!wait_or_abort(acc_empty + t, pt ^ 1u, abort_flag)) break;
+                tc_fence_after();
+                const uint64_t bdesc = umma_smem_desc(smem_u32(ring + s * Geo::TILE_BYTES));
+#pragma unroll
+                for (int k = 0; k < 8; ++k)  // K = 16 per instruction: 256 bytes further in both operands
+                    umma_bf16(tmem_base + t * Geo::N, adesc + k * 16, bdesc + k * 16, idesc, k > 0);
+                umma_commit(acc_full + t);
+                umma_commit(empty + s);
+            }
+        }
+    } else {
+        const int q = warp & 3;            // TMEM lane quarter this warp may access
+        const int ch = (warp - 2) >> 2;    // column half of the tile
+        const int m = q * 32 + lane;       // index bits 3..9 of every element this thread produces
+        const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + ch * Geo::CPW;
+
+        F2 as[L::PARAMS_IN_SMEM ? 1 : Geo::PIECES][4], bs[L::PARAMS_IN_SMEM ? 1 : Geo::PIECES][4];
+        const float* pa = reinterpret_cast<const float*>(smem_raw + L::OFF_PARAMS);
+        if constexpr (!L::PARAMS_IN_SMEM) {
+            const F2 rs2 = f2(inv_sqrt_d, inv_sqrt_d);
+#pragma unroll
+            for (int p = 0; p < Geo::PIECES; ++p) {
+                load_params8(a + p * 1024 + m * 8, as[p]);
+                load_params8(b + p * 1024 + m * 8, bs[p]);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) as[p][j] = mul2(as[p][j], rs2);
+            }
+        }
+
+        for (long long it = 0; it < my_tiles; ++it) {
+            const int t = static_cast<int>(it % ACC);
+            const uint32_t pt = static_cast<uint32_t>(it / ACC) & 1u;
+            if (!warp_wait_or_abort(acc_full + t, pt, abort_flag)) break;
+            tc_fence_after();
+            float u[Geo::CPW];
+            tmem_ld_cols<Geo::CPW>(lane_addr + t * Geo::N, u);
+            tmem_wait_ld();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(acc_empty + t);  // the accumulator is in registers now
+
+            const long long tile = blockIdx.x + it * gridDim.x;
+#pragma unroll
+            for (int rl = 0; rl < Geo::RPW; ++rl) {
+                const long long row = tile * Geo::ROWS + ch * Geo::RPW + rl;
+                float v[Geo::R];
+#pragma unroll
+                for (int i = 0; i < Geo::R; ++i) v[i] = u[rl * Geo::R + i];
+                thread_stages<Geo::R>(v);
+                if (row < T) {
+                    uint4* dst = reinterpret_cast<uint4*>(y + row * Geo::D + m * 8);
+#pragma unroll
+                    for (int p = 0; p < Geo::PIECES; ++p) {
+                        F2 w[4];
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) w[j] = f2(v[p * 8 + 2 * j], v[p * 8 + 2 * j + 1]);
+                        if constexpr (L::PARAMS_IN_SMEM) {
+                            const float4* qa = reinterpret_cast<const float4*>(pa) + (p * 2) * 128 + m;
+                            const float4* qb = reinterpret_cast<const float4*>(pa + Geo::D) + (p * 2) * 128 + m;
+                            const float4 a0 = qa[0], a1 = qa[128], b0 = qb[0], b1 = qb[128];
+                            F2 ap[4] = {f2(a0.x, a0.y), f2(a0.z, a0.w), f2(a1.x, a1.y), f2(a1.z, a1.w)};
+                            F2 bp[4] = {f2(b0.x, b0.y), f2(b0.z, b0.w), f2(b1.x, b1.y), f2(b1.z, b1.w)};
+                            fwd_store_chunk(w, ap, bp, dst + p * 128);
+                        } else {
+                            fwd_store_chunk(w, as[p], bs[p], dst + p * 128);
+                        }
+                    }
+                }
+            }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        __syncwarp();
+        tc_fence_after();
+        tmem_dealloc(tmem_base, L::TMEM_COLS);
+    }
+}
+
+// ---- backward --------------------------------------------------------------------------
+template <int LOGD, int NCOL, int STAGES>
+struct UmmaBwdSmem {
+    using Geo = UmmaGeo<LOGD, NCOL>;
+    static constexpr int STAGE_BYTES = 2 * Geo::TILE_BYTES;  // x tile, then dy tile
+    static constexpr int TMEM_COLS = 4 * NCOL <= 256 ? 256 : 512;  // D1 x2, D2 x2
+    static constexpr int OFF_H = 0;
+    static constexpr int OFF_RING = Geo::H_BYTES;
+    static constexpr int OFF_BARS = OFF_RING + STAGES * STAGE_BYTES;
+    static constexpr int NBARS = 3 * STAGES + 8;
+    static constexpr int OFF_MISC = OFF_BARS + NBARS * 8;
+    static constexpr int BYTES = OFF_MISC + 16;
+    static_assert(STAGES * STAGE_BYTES >= 2 * Geo::D * 4, "the ring is reused to fold da, db");
+};
+
+// partials layout: [gridDim.x][2][D] fp32; slot 0: sum_t dy (.) (x H) WITHOUT the
+// 1/sqrt(d) factor (the second pass applies it), slot 1: sum_t dy.
+template <int LOGD, int NCOL, int STAGES, typename TP>
+__global__ void __launch_bounds__(UmmaGeo<LOGD, NCOL>::THREADS, 1)
+umma_bwd_kernel(const __nv_bfloat16* dy, const __nv_bfloat16* x, const TP* __restrict__ a, __nv_bfloat16* dx,
+                float* __restrict__ partials, long long T, float inv_sqrt_d) {
+    using Geo = UmmaGeo<LOGD, NCOL>;
+    using L = UmmaBwdSmem<LOGD, NCOL, STAGES>;
+    static_assert(Geo::R <= 32, "per-thread accumulators must fit in registers");
+    extern __shared__ __align__(1024) unsigned char umma_smem[];
+    unsigned char* const smem_raw = umma_smem;
+    unsigned char* ring = smem_raw + L::OFF_RING;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem_raw + L::OFF_BARS);
+    uint64_t* full = bars;                      // [STAGES] x and dy tiles landed
+    uint64_t* stage_empty = bars + STAGES;      // [STAGES] second product has consumed the slot
+    uint64_t* g_ready = bars + 2 * STAGES;      // [STAGES] G (hi, lo) written into the slot by the 8 warps
+    uint64_t* d1_full = bars + 3 * STAGES;      // [2]
+    uint64_t* d1_empty = d1_full + 2;           // [2]
+    uint64_t* d2_full = d1_full + 4;            // [2]
+    uint64_t* d2_empty = d1_full + 6;           // [2]
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem_raw + L::OFF_MISC);
+    volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem_raw + L::OFF_MISC + 4);
+
+    const int tid = threadIdx.x;
+    const int warp = tid >> 5;
+    const int lane = tid & 31;
+    const long long tiles = (T + Geo::ROWS - 1) / Geo::ROWS;
+    const long long my_tiles = blockIdx.x < tiles ? (tiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+
+    if (tid == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(full + s, 1);
+            mbar_init(stage_empty + s, 1);
+            mbar_init(g_ready + s, Geo::EPI_WARPS);
+        }
+        for (int t = 0; t < 2; ++t) {
+            mbar_init(d1_full + t, 1);
+            mbar_init(d1_empty + t, Geo::EPI_WARPS);
+            mbar_init(d2_full + t, 1);
+            mbar_init(d2_empty + t, Geo::EPI_WARPS);
+        }
+        *abort_flag = 0;
+        fence_mbar_init();
+    }
+    write_h128(smem_raw + L::OFF_H, tid, Geo::THREADS);
+    fence_async_smem();
+    if (warp == 1) {
+        tmem_alloc(tmem_slot, L::TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    const uint32_t tmem_d1 = tmem_base;
+    const uint32_t tmem_d2 = tmem_base + 2 * Geo::N;
+
+    // per-thread partial column sums (epilogue warps only; declared here so that the fold
+    // after the role loops can see them)
+    F2 da_acc[Geo::PIECES][4], db_acc[Geo::PIECES][4];
+#pragma unroll
+    for (int p = 0; p < Geo::PIECES; ++p) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) { da_acc[p][j] = f2(0.0f, 0.0f); db_acc[p][j] = f2(0.0f, 0.0f); }
+    }
+
+    if (warp == 0) {
+        if (lane == 0) {
+            long long it = 0;
+            for (; it < my_tiles; ++it) {
+                const int s = static_cast<int>(it % STAGES);
+                const uint32_t ph = static_cast<uint32_t>(it / STAGES) & 1u;
+                if (!wait_or_abort(stage_empty + s, ph ^ 1u, abort_flag)) break;
+                const long long tile = blockIdx.x + it * gridDim.x;
+                const long long row0 = tile * Geo::ROWS;
+                const long long rows = T - row0 < Geo::ROWS ? T - row0 : Geo::ROWS;
+                const uint32_t bytes = static_cast<uint32_t>(rows) * Geo::D * 2;
+                mbar_expect_tx(full + s, 2 * bytes);
+                bulk_load(ring + s * L::STAGE_BYTES, x + row0 * Geo::D, bytes, full + s);
+                bulk_load(ring + s * L::STAGE_BYTES + Geo::TILE_BYTES, dy + row0 * Geo::D, bytes, full + s);
+            }
+            if (*abort_flag) {
+                const long long lo = it > STAGES ? it - STAGES : 0;
+                for (long long j = lo; j < it; ++j)
+                    mbar_wait_bounded(full + (j % STAGES), static_cast<uint32_t>(j / STAGES) & 1u);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            const uint64_t adesc = umma_smem_desc(smem_u32(smem_raw + L::OFF_H));
+            constexpr uint32_t idesc = umma_idesc(Geo::N);
+            // first product of tile i: D1 = H_128 X
+            auto step_x = [&](long long i) -> bool {
+                const int s = static_cast<int>(i % STAGES);
+                const uint32_t ph = static_cast<uint32_t>(i / STAGES) & 1u;
+                const int t = static_cast<int>(i & 1);
+                const uint32_t pt = static_cast<uint32_t>(i >> 1) & 1u;
+                if (!wait_or_abort(full + s, ph, abort_flag)) return false;
+                if (!wait_or_abort(d1_empty + t, pt ^ 1u, abort_flag)) return false;
+                tc_fence_after();
+                const uint64_t bdesc = umma_smem_desc(smem_u32(ring + s * L::STAGE_BYTES));
+#pragma unroll
+                for (int k = 0; k < 8; ++k)
+                    umma_bf16(tmem_d1 + t * Geo::N, adesc + k * 16, bdesc + k * 16, idesc, k > 0);
+                umma_commit(d1_full + t);
+                return true;
+            };
+            // second product of tile i: D2 = H_128 G_hi + H_128 G_lo
+            auto step_g = [&](long long i) -> bool {
+                const int s = static_cast<int>(i % STAGES);
+                const uint32_t ph = static_cast<uint32_t>(i / STAGES) & 1u;
+                const int t = static_cast<int>(i & 1);
+                const uint32_t pt = static_cast<uint32_t>(i >> 1) & 1u;
+                if (!wait_or_abort(g_ready + s, ph, abort_flag)) return false;
+                if (!wait_or_abort(d2_empty + t, pt ^ 1u, abort_flag)) return false;
+                tc_fence_after();
+                const uint64_t bhi = umma_smem_desc(smem_u32(ring + s * L::STAGE_BYTES));
+                const uint64_t blo = umma_smem_desc(smem_u32(ring + s * L::STAGE_BYTES + Geo::TILE_BYTES));
+#pragma unroll
+                for (int k = 0; k < 8; ++k)
+                    umma_bf16(tmem_d2 + t * Geo::N, adesc + k * 16, bhi + k * 16, idesc, k > 0);
+#pragma unroll
+                for (int k = 0; k < 8; ++k) umma_bf16(tmem_d2 + t * Geo::N, adesc + k * 16, blo + k * 16, idesc, 1);
+                umma_commit(d2_full + t);
+                umma_commit(stage_empty + s);
+                return true;
+            };
+            bool ok = my_tiles > 0 ? step_x(0) : true;
+            for (long long i = 0; ok && i < my_tiles; ++i) {
+                if (i + 1 < my_tiles) ok = step_x(i + 1);
+                if (ok) ok = step_g(i);
+            }
+        }
+    } else {
+        const int q = warp & 3;
+        const int ch = (warp - 2) >> 2;
+        const int m = q * 32 + lane;
+        const uint32_t lane_off = (static_cast<uint32_t>(q * 32) << 16) + ch * Geo::CPW;
+
+        F2 as[Geo::PIECES][4];
+        {
+            const F2 rs2 = f2(inv_sqrt_d, inv_sqrt_d);
+#pragma unroll
+            for (int p = 0; p < Geo::PIECES; ++p) {
+                load_params8(a + p * 1024 + m * 8, as[p]);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) as[p][j] = mul2(as[p][j], rs2);
+            }
+        }
+
+        // dx rows of tile j: read D2, round, store
+        auto store_dx = [&](long long j) -> bool {
+            const int t = static_cast<int>(j & 1);
+            const uint32_t pt = static_cast<uint32_t>(j >> 1) & 1u;
+            if (!warp_wait_or_abort(d2_full + t, pt, abort_flag)) return false;
+            tc_fence_after();
+            float u[Geo::CPW];
+            tmem_ld_cols<Geo::CPW>(tmem_d2 + lane_off + t * Geo::N, u);
+            tmem_wait_ld();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(d2_empty + t);
+            const long long tile = blockIdx.x + j * gridDim.x;
+#pragma unroll
+            for (int rl = 0; rl < Geo::RPW; ++rl) {
+                const long long row = tile * Geo::ROWS + ch * Geo::RPW + rl;
+                if (row < T) {
+                    uint4* dst = reinterpret_cast<uint4*>(dx + row * Geo::D + m * 8);
+#pragma unroll
+                    for (int p = 0; p < Geo::PIECES; ++p) {
+                        const float* w = u + rl * Geo::R + p * 8;
+                        uint4 o;
+                        o.x = pack_bf16x2(w[0], w[1]);
+                        o.y = pack_bf16x2(w[2], w[3]);
+                        o.z = pack_bf16x2(w[4], w[5]);
+                        o.w = pack_bf16x2(w[6], w[7]);
+                        __stcs(dst + p * 128, o);
+                    }
+                }
+            }
+            return true;
+        };
+
+        bool ok = true;
+        for (long long it = 0; ok && it < my_tiles; ++it) {
+            const int s = static_cast<int>(it % STAGES);
+            const uint32_t ph = static_cast<uint32_t>(it / STAGES) & 1u;
+            const int t = static_cast<int>(it & 1);
+            const uint32_t pt = static_cast<uint32_t>(it >> 1) & 1u;
+            if (!warp_wait_or_abort(d1_full + t, pt, abort_flag)) { ok = false; break; }
+            // the first product ran, so the tile has landed; observing the barrier ourselves
+            // makes the copied dy bytes visible to this thread's ordinary loads
+            if (!warp_wait_or_abort(full + s, ph, abort_flag)) { ok = false; break; }
+            tc_fence_after();
+            float u[Geo::CPW];
+            tmem_ld_cols<Geo::CPW>(tmem_d1 + lane_off + t * Geo::N, u);
+            tmem_wait_ld();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(d1_empty + t);
+
+            unsigned char* slot_x = ring + s * L::STAGE_BYTES;
+            unsigned char* slot_dy = slot_x + Geo::TILE_BYTES;
+            const long long tile = blockIdx.x + it * gridDim.x;
+#pragma unroll
+            for (int rl = 0; rl < Geo::RPW; ++rl) {
+                const int rt = ch * Geo::RPW + rl;  // row inside the tile
+                const bool valid = tile * Geo::ROWS + rt < T;
+                float v[Geo::R];
+#pragma unroll
+                for (int i = 0; i < Geo::R; ++i) v[i] = u[rl * Geo::R + i];
+                thread_stages<Geo::R>(v);  // v = (x H)[piece*1024 + m*8 + n], unnormalised
+                if (!valid) {
+                    // rows past T were never copied: their accumulator columns hold whatever the
+                    // slot held before (possibly NaN), and 0 * NaN would poison the column sums
+#pragma unroll
+                    for (int i = 0; i < Geo::R; ++i) v[i] = 0.0f;
+                }
+                float g[Geo::R];
+#pragma unroll
+                for (int p = 0; p < Geo::PIECES; ++p) {
+                    const int chunk = ((rt * Geo::PIECES + p) * 128 + m) * 16;
+                    uint4 raw = make_uint4(0u, 0u, 0u, 0u);
+                    if (valid) raw = *reinterpret_cast<const uint4*>(slot_dy + chunk);
+                    const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const F2 dyv = unpack_bf16x2(w[j]);
+                        da_acc[p][j] = fma2(dyv, f2(v[p * 8 + 2 * j], v[p * 8 + 2 * j + 1]), da_acc[p][j]);
+                        db_acc[p][j] = add2(db_acc[p][j], dyv);
+                        const F2 gv = mul2(as[p][j], dyv);
+                        g[p * 8 + 2 * j] = gv.x;
+                        g[p * 8 + 2 * j + 1] = gv.y;
+                    }
+                }
+                thread_stages<Geo::R>(g);  // the low and piece stages of the second transform
+#pragma unroll
+                for (int p = 0; p < Geo::PIECES; ++p) {
+                    const int chunk = ((rt * Geo::PIECES + p) * 128 + m) * 16;
+                    uint4 hi, lo;
+                    split_hi_lo(f2(g[p * 8 + 0], g[p * 8 + 1]), hi.x, lo.x);
+                    split_hi_lo(f2(g[p * 8 + 2], g[p * 8 + 3]), hi.y, lo.y);
+                    split_hi_lo(f2(g[p * 8 + 4], g[p * 8 + 5]), hi.z, lo.z);
+                    split_hi_lo(f2(g[p * 8 + 6], g[p * 8 + 7]), hi.w, lo.w);
+                    *reinterpret_cast<uint4*>(slot_x + chunk) = hi;   // the x tile is consumed: D1 is complete
+                    *reinterpret_cast<uint4*>(slot_dy + chunk) = lo;  // this thread alone read this dy chunk
+                }
+            }
+            fence_async_smem();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(g_ready + s);
+            if (it > 0) ok = store_dx(it - 1);
+        }
+        if (ok && my_tiles > 0) ok = store_dx(my_tiles - 1);
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        __syncwarp();
+        tc_fence_after();
+        tmem_dealloc(tmem_base, L::TMEM_COLS);
+    }
+
+    // fold the two column halves (they hold different rows of the same channels) in a fixed
+    // order and publish this CTA's partial sums; the ring is free now
+    float* fold = reinterpret_cast<float*>(ring);
+    if (warp >= 6) {
+        const int m = (warp & 3) * 32 + lane;
+#pragma unroll
+        for (int p = 0; p < Geo::PIECES; ++p) {
+            float4* pd = reinterpret_cast<float4*>(fold) + ((0 * Geo::PIECES + p) * 2) * 128 + m;
+            float4* pb = reinterpret_cast<float4*>(fold) + ((1 * Geo::PIECES + p) * 2) * 128 + m;
+            pd[0] = make_float4(da_acc[p][0].x, da_acc[p][0].y, da_acc[p][1].x, da_acc[p][1].y);
+            pd[128] = make_float4(da_acc[p][2].x, da_acc[p][2].y, da_acc[p][3].x, da_acc[p][3].y);
+            pb[0] = make_float4(db_acc[p][0].x, db_acc[p][0].y, db_acc[p][1].x, db_acc[p][1].y);
+            pb[128] = make_float4(db_acc[p][2].x, db_acc[p][2].y, db_acc[p][3].x, db_acc[p][3].y);
+        }
+    }
+    __syncthreads();
+    if (warp >= 2 && warp < 6) {
+        const int m = (warp & 3) * 32 + lane;
+        float* out = partials + static_cast<size_t>(blockIdx.x) * 2 * Geo::D;
+#pragma unroll
+        for (int p = 0; p < Geo::PIECES; ++p) {
+            const float4* pd = reinterpret_cast<const float4*>(fold) + ((0 * Geo::PIECES + p) * 2) * 128 + m;
+            const float4* pb = reinterpret_cast<const float4*>(fold) + ((1 * Geo::PIECES + p) * 2) * 128 + m;
+            const float4 d0 = pd[0], d1 = pd[128], b0 = pb[0], b1 = pb[128];
+            float4* oa = reinterpret_cast<float4*>(out + p * 1024 + m * 8);
+            float4* ob = reinterpret_cast<float4*>(out + Geo::D + p * 1024 + m * 8);
+            oa[0] = make_float4(da_acc[p][0].x + d0.x, da_acc[p][0].y + d0.y, da_acc[p][1].x + d0.z,
+                                da_acc[p][1].y + d0.w);
+            oa[1] = make_float4(da_acc[p][2].x + d1.x, da_acc[p][2].y + d1.y, da_acc[p][3].x + d1.z,
+                                da_acc[p][3].y + d1.w);
+            ob[0] = make_float4(db_acc[p][0].x + b0.x, db_acc[p][0].y + b0.y, db_acc[p][1].x + b0.z,
+                                db_acc[p][1].y + b0.w);
+            ob[1] = make_float4(db_acc[p][2].x + b1.x, db_acc[p][2].y + b1.y, db_acc[p][3].x + b1.z,
+                                db_acc[p][3].y + b1.w);
+        }
+    }
+}
+
+}  // namespace wht

@@ -10,6 +10,7 @@
 #include "bfly_kernels.cuh"
 #include "mma_kernels.cuh"
 #include "mma_pipe_kernels.cuh"
+#include "umma_kernels.cuh"
 
 namespace {
 
@@ -337,6 +338,78 @@ int dispatch_mma_bwd(int logd, bool streamed, const BwdArgs& g, const Ctx& c) {
     return WHT_ERR_BAD_DIM;
 }
 
+// ------------------------------------------------------------------ tcgen05 family
+// One persistent CTA per SM; a kernel's shared-memory need alone keeps a second CTA off the SM,
+// which the kernel relies on when it allocates tensor memory.
+template <typename Kernel>
+int prepare_umma(Kernel kernel, int smem, int dev, int* cache) {
+    if (cache[dev]) return WHT_OK;
+    WHT_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    cache[dev] = 1;
+    return WHT_OK;
+}
+
+template <int LOGD, int NCOL, int STAGES, typename TP>
+int launch_umma_fwd(const FwdArgs& f, const Ctx& c) {
+    using Geo = UmmaGeo<LOGD, NCOL>;
+    using L = UmmaFwdSmem<LOGD, NCOL, STAGES, TP>;
+    static_assert(L::BYTES > 116 * 1024, "must be alone on its SM");
+    static int ready[kMaxDevices] = {};
+    auto kernel = umma_fwd_kernel<LOGD, NCOL, STAGES, TP>;
+    int rc = prepare_umma(kernel, L::BYTES, c.dev, ready);
+    if (rc != WHT_OK) return rc;
+    const int grid = capped_grid(ceil_div(c.T, Geo::ROWS), c.sms, 1);
+    kernel<<<grid, Geo::THREADS, L::BYTES, c.stream>>>(
+        static_cast<const __nv_bfloat16*>(f.x), static_cast<const TP*>(f.a), static_cast<const TP*>(f.b),
+        static_cast<__nv_bfloat16*>(f.y), static_cast<long long>(c.T), inv_sqrt(Geo::D));
+    WHT_CUDA_TRY(cudaGetLastError());
+    return WHT_OK;
+}
+
+template <int LOGD, int NCOL, int STAGES, typename TP>
+int launch_umma_bwd(const BwdArgs& g, const Ctx& c) {
+    using Geo = UmmaGeo<LOGD, NCOL>;
+    using L = UmmaBwdSmem<LOGD, NCOL, STAGES>;
+    static_assert(L::BYTES > 116 * 1024, "must be alone on its SM");
+    static int ready[kMaxDevices] = {};
+    auto kernel = umma_bwd_kernel<LOGD, NCOL, STAGES, TP>;
+    if (!g.query_only) {
+        int rc = prepare_umma(kernel, L::BYTES, c.dev, ready);
+        if (rc != WHT_OK) return rc;
+    }
+    const int grid = capped_grid(ceil_div(c.T, Geo::ROWS), c.sms, 1);
+    return run_bwd_with_grid(g, c, grid, Geo::D, [&](int n) {
+        kernel<<<n, Geo::THREADS, L::BYTES, c.stream>>>(
+            static_cast<const __nv_bfloat16*>(g.dy), static_cast<const __nv_bfloat16*>(g.x),
+            static_cast<const TP*>(g.a), static_cast<__nv_bfloat16*>(g.dx), static_cast<float*>(g.ws),
+            static_cast<long long>(c.T), inv_sqrt(Geo::D));
+    });
+}
+
+template <typename TP>
+int dispatch_umma_fwd(int logd, const FwdArgs& f, const Ctx& c) {
+    switch (logd) {
+        case 10: return launch_umma_fwd<10, 128, 4, TP>(f, c);
+        case 11: return launch_umma_fwd<11, 128, 4, TP>(f, c);
+        case 12: return launch_umma_fwd<12, 128, 4, TP>(f, c);
+        case 13: return launch_umma_fwd<13, 128, 4, TP>(f, c);
+    }
+    return WHT_ERR_BAD_DIM;
+}
+
+template <typename TP>
+int dispatch_umma_bwd(int logd, const BwdArgs& g, const Ctx& c) {
+    switch (logd) {
+        case 10: return launch_umma_bwd<10, 128, 3, TP>(g, c);
+        case 11: return launch_umma_bwd<11, 128, 3, TP>(g, c);
+        case 12: return launch_umma_bwd<12, 64, 5, TP>(g, c);
+    }
+    return WHT_ERR_BAD_DIM;
+}
+
+bool umma_fwd_supported(int logd, int dtype) { return dtype != WHT_F32 && logd >= 10 && logd <= 13; }
+bool umma_bwd_supported(int logd, int dtype) { return dtype != WHT_F32 && logd >= 10 && logd <= 12; }
+
 bool mma_supported(int logd, int dtype) { return dtype != WHT_F32 && logd >= 9 && logd <= 13; }
 
 // Streaming pays once every row group has several rows to pipeline.
@@ -348,8 +421,12 @@ int run_fwd(const FwdArgs& f, int64_t T, int32_t d, int dtype, cudaStream_t s, b
     int rc = current_device(&c.dev, &c.sms);
     if (rc != WHT_OK) return rc;
     const int logd = log2_of(d);
+    if (umma_fwd_supported(logd, dtype) &&
+        (g_variant == 4 || (g_variant == 0 && !decode && enough_rows_to_stream(T, c.sms)))) {
+        return dtype == WHT_BF16 ? dispatch_umma_fwd<__nv_bfloat16>(logd, f, c) : dispatch_umma_fwd<float>(logd, f, c);
+    }
     if (g_variant != 1 && mma_supported(logd, dtype)) {
-        const bool streamed = g_variant == 3 || (g_variant == 0 && !decode && enough_rows_to_stream(T, c.sms));
+        const bool streamed = g_variant >= 3 || (g_variant == 0 && !decode && enough_rows_to_stream(T, c.sms));
         const bool few_rows = !streamed && (decode || (g_variant == 0 && T < static_cast<int64_t>(c.sms) * 4));
         return dtype == WHT_BF16 ? dispatch_mma_fwd<__nv_bfloat16>(logd, few_rows, streamed, f, c)
                                  : dispatch_mma_fwd<float>(logd, few_rows, streamed, f, c);
@@ -366,8 +443,11 @@ int run_bwd(const BwdArgs& g, int64_t T, int32_t d, int dtype, cudaStream_t s) {
     int rc = current_device(&c.dev, &c.sms);
     if (rc != WHT_OK) return rc;
     const int logd = log2_of(d);
+    if (umma_bwd_supported(logd, dtype) && (g_variant == 4 || (g_variant == 0 && enough_rows_to_stream(T, c.sms)))) {
+        return dtype == WHT_BF16 ? dispatch_umma_bwd<__nv_bfloat16>(logd, g, c) : dispatch_umma_bwd<float>(logd, g, c);
+    }
     if (g_variant != 1 && mma_supported(logd, dtype)) {
-        const bool streamed = g_variant == 3 || (g_variant == 0 && enough_rows_to_stream(T, c.sms));
+        const bool streamed = g_variant >= 3 || (g_variant == 0 && enough_rows_to_stream(T, c.sms));
         return dtype == WHT_BF16 ? dispatch_mma_bwd<__nv_bfloat16>(logd, streamed, g, c)
                                  : dispatch_mma_bwd<float>(logd, streamed, g, c);
     }
@@ -517,7 +597,7 @@ int wht_affine_bwd_noalloc(const void* dy, const void* x, const void* a, void* d
 }
 
 int wht_affine_set_variant(int variant) {
-    if (variant < 0 || variant > 3) return WHT_ERR_BAD_VARIANT;
+    if (variant < 0 || variant > 4) return WHT_ERR_BAD_VARIANT;
     g_variant = variant;
     return WHT_OK;
 }

@@ -17,7 +17,7 @@ from paper_2603_08343_b200 import workloads as wl
 
 pytestmark = pytest.mark.gpu
 
-VARIANTS = [1, 2, 3]  # butterfly; tensor-core assisted with direct loads; with streamed rows (each falls back where unsupported)
+VARIANTS = [1, 2, 3, 4]  # butterfly; mma.sync with direct loads; with streamed rows; tcgen05 (each falls back where unsupported)
 
 
 @pytest.fixture(scope="module")
@@ -292,6 +292,15 @@ def test_streamed_kernels_on_many_rows(B):
                         (4096, wl.WHT_BF16, 3001), (8192, wl.WHT_BF16_PF32, 1501)]:
         w = wl.Workload("stream", T, d, dtype, "normal", 300 + d, True, "")
         _run_case(B, w, 3)
+    B.wht_affine_device_status()
+
+
+def test_tcgen05_kernels_on_many_rows(B):
+    # several tiles per CTA on every SM (the ring and both accumulator sets wrap), ragged last tile
+    for d, dtype, T in [(1024, wl.WHT_BF16, 148 * 16 * 5 + 7), (2048, wl.WHT_BF16_PF32, 148 * 8 * 4 + 3),
+                        (4096, wl.WHT_BF16, 148 * 4 * 3 + 1), (8192, wl.WHT_BF16_PF32, 148 * 2 * 3 + 1)]:
+        w = wl.Workload("tc5", T, d, dtype, "normal", 400 + d, True, "")
+        _run_case(B, w, 4)
     B.wht_affine_device_status()
 
 
