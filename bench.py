@@ -37,6 +37,11 @@ from paper_2603_08343_b200 import dp
 from paper_2603_08343_b200 import workloads as wl
 
 METRIC = "wht_affine_tokens_per_s_fwd_bwd"
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the dominant kernel,
+# from the ncu capture summarised under profiles/; keyed by (workload, rows).  A quarter-size
+# case was captured and scaled by the rows (traffic is proportional to them).  Reset to {} when
+# the kernel changes.
+NCU_TRAFFIC_BYTES = {}
 UNIT = "tokens/s"
 
 
@@ -66,7 +71,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
-                 "-i", str(self.gpu_index), "-lms", "100"],
+                 "-i", str(self.gpu_index), "-lms", "20"],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
@@ -157,7 +162,9 @@ def run_reference(args, rank: int, world: int):
         return
     w = wl.CONFIGS[args.workload]
     rows = {"tiny": 64, "prefill": 2048, "training": 1024, "large": 128}[args.workload]
-    for _ in range(args.warmup):
+    # keep the whole run to about a minute of CPU work whatever K is: the per-row cost is constant
+    rows = max(16, min(rows, (32 * rows) // max(args.steps, 1)))
+    for _ in range(min(args.warmup, 3)):
         oracle_step_seconds(w, min(rows, 64))
     times = [oracle_step_seconds(w, rows) for _ in range(args.steps)]
     total = sum(times)
@@ -369,11 +376,12 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         sampler.start()
         time.sleep(0.3)
     torch.cuda.synchronize()
-    events = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    # timed region: K steps back to back, one event on either side (nothing between the calls,
+    # so that each kernel may start while its predecessor drains)
     t_wall0 = time.time()
     with Timer() as total:
         for k in range(args.steps):
-            step(events[k])
+            step()
     total_ms = total.ms()
     torch.cuda.synchronize()
     t_wall1 = time.time()
@@ -382,26 +390,50 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         tmax = torch.tensor([total_ms], device="cuda")
         dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
         total_ms = float(tmax.item())
-    clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
+    clocks_step = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
 
+    # per-call durations for the roofline figure: K launches of one call back to back between
+    # two events (sustained, launches overlapping as they do inside the step), and, for
+    # comparison, the same calls inside the step sequence with an event after every call
+    # (each event adds a few microseconds of idle front-end time to the call before it)
+    def fwd_only():
+        i = counter["i"] % nbuf
+        counter["i"] += 1
+        B.wht_affine_fwd(xs[i], a, b, ys[i], w.T, w.d, w.dtype)
+
+    def bwd_only():
+        i = counter["i"] % nbuf
+        counter["i"] += 1
+        B.wht_affine_bwd(dys[i], xs[i], a, dxs[i], da, db, w.T, w.d, w.dtype)
+
+    fwd_b2b_ms = time_loop(fwd_only, args.steps, warmup=3)
+    bwd_b2b_ms = time_loop(bwd_only, args.steps, warmup=3) if w.has_bwd else None
+    ev_steps = min(args.steps, 200)
+    events = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(ev_steps)]
+    for k in range(ev_steps):
+        step(events[k])
+    torch.cuda.synchronize()
     fwd_ms = [e[0].elapsed_time(e[1]) for e in events]
     bwd_ms = [e[1].elapsed_time(e[2]) for e in events] if w.has_bwd else []
+    clocks = clocks_step
     ms_per_step = total_ms / args.steps
     value = world * w.T / (ms_per_step * 1e-3)
 
-    # roofline of the dominant kernel: the backward main kernel when there is one
+    # roofline of the dominant call: the backward call when there is one
     if w.has_bwd:
-        dom, dom_ms = "wht_affine_bwd (main kernel + the small finalize pass)", statistics.mean(bwd_ms)
+        dom, dom_ms = "wht_affine_bwd (main kernel + the small second pass)", bwd_b2b_ms
         bytes_per_launch = 3 * w.T * w.d * w.io_bytes
     else:
-        dom, dom_ms = "wht_affine_fwd", statistics.mean(fwd_ms)
+        dom, dom_ms = "wht_affine_fwd", fwd_b2b_ms
         bytes_per_launch = 2 * w.T * w.d * w.io_bytes
     achieved = bytes_per_launch / 1e9 / (dom_ms * 1e-3)
+    traffic = NCU_TRAFFIC_BYTES.get((w.name, w.T))
     roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": hbm_peak, "unit": "GB/s",
-                "frac": achieved / hbm_peak, "peak_source": peak_src, "traffic": None,
+                "frac": achieved / hbm_peak, "peak_source": peak_src, "traffic": traffic,
                 "algorithmic_bytes_per_launch": bytes_per_launch, "avg_launch_ms": dom_ms,
+                "timing": f"{args.steps} launches back to back between two CUDA events",
                 "frac_of_nominal_8000": achieved / 8000.0}
-    fwd_gbps = 2 * w.T * w.d * w.io_bytes / 1e9 / (statistics.mean(fwd_ms) * 1e-3)
+    fwd_gbps = 2 * w.T * w.d * w.io_bytes / 1e9 / (fwd_b2b_ms * 1e-3)
 
     # ---- end to end: pinned host buffers in, results back to the host, every step
     e2e = None
@@ -415,13 +447,17 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         dxp = torch.empty_like(xp).pin_memory()
         dap = torch.empty(w.d, dtype=torch.float32).pin_memory()
         dbp = torch.empty(w.d, dtype=torch.float32).pin_memory()
-        h2d += dyp.numel() * dyp.element_size() + xp.numel() * xp.element_size() + ap.numel() * ap.element_size()
+        h2d += dyp.numel() * dyp.element_size()
         d2h += dxp.numel() * dxp.element_size() + 8 * w.d
 
+    pipe = B.HostPipe(chunk_rows=max(1024, (32 << 20) // (w.d * w.io_bytes)))
+
     def e2e_step():
-        B.forward_host(xp, ap, bp, yp, staging)
+        # x, a, b in -> forward -> y out; dy in -> backward (x still resident) -> dx, da, db out
+        B.forward_host(xp, ap, bp, yp, staging, pipe=pipe)
         if w.has_bwd:
-            B.backward_host(dyp, xp, ap, dxp, dap, dbp, staging)
+            B.backward_host(dyp, xp, ap, dxp, dap, dbp, staging, pipe=pipe, x_resident=True)
+        pipe.join()
 
     e2e_steps = max(2, min(args.steps, 5))
     e2e_ms = time_loop(e2e_step, e2e_steps, warmup=1)
@@ -431,7 +467,8 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         e2e_ms = float(tmax.item())
     e2e = {"value": world * w.T / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
            "d2h_bytes_per_step": int(d2h), "ms_per_step": e2e_ms, "steps": e2e_steps,
-           "api": "binding.forward_host + binding.backward_host (pinned host -> device -> C ABI -> pinned host)"}
+           "api": "binding.forward_host + binding.backward_host with a HostPipe (pinned host -> device -> C ABI -> "
+                  "pinned host; rows move in chunks on two copy streams, x stays resident between the two calls)"}
     del xp, yp, staging
     if w.has_bwd:
         del dyp, dxp
@@ -452,12 +489,14 @@ def run_ours(args, rank: int, world: int, local_rank: int):
                    "step": "wht_affine_fwd + wht_affine_bwd" if w.has_bwd else "wht_affine_fwd",
                    "l2": l2_note, "variant": B.wht_affine_get_variant(),
                    "parallelism": f"dp{world} (rows sharded; all-reduce of da|db only)" if world > 1 else "single GPU"},
-        "fwd": {"ms": statistics.mean(fwd_ms), "GBps": fwd_gbps, "frac_of_measured_peak": fwd_gbps / hbm_peak,
-                "frac_of_nominal_8000": fwd_gbps / 8000.0, "tokens_per_s": w.T / (statistics.mean(fwd_ms) * 1e-3)},
+        "fwd": {"ms": fwd_b2b_ms, "GBps": fwd_gbps, "frac_of_measured_peak": fwd_gbps / hbm_peak,
+                "frac_of_nominal_8000": fwd_gbps / 8000.0, "tokens_per_s": w.T / (fwd_b2b_ms * 1e-3),
+                "ms_in_step_with_events": statistics.mean(fwd_ms)},
         "roofline": roofline, "e2e": e2e, "gpu_launches": launches_per_step * args.steps, "clocks": clocks,
     }
     if w.has_bwd:
-        out["bwd"] = {"ms": dom_ms, "GBps": achieved, "frac_of_measured_peak": achieved / hbm_peak,
+        out["bwd"] = {"ms_in_step_with_events": statistics.mean(bwd_ms),
+                      "ms": dom_ms, "GBps": achieved, "frac_of_measured_peak": achieved / hbm_peak,
                       "frac_of_nominal_8000": achieved / 8000.0, "tokens_per_s": w.T / (dom_ms * 1e-3)}
 
     # ---- CPU baseline: the oracle as it stands, on a bounded sample of the same workload
@@ -485,8 +524,8 @@ def run_ours(args, rank: int, world: int, local_rank: int):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--workload", default="training", choices=["tiny", "prefill", "training", "large"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--variant", type=int, default=0)

@@ -189,31 +189,104 @@ def backward(dy, x, a, stream=None):
     return dx, da, db
 
 
-def forward_host(x_host, a_host, b_host, y_host, staging, stream=None):
+class HostPipe:
+    """Two copy streams for the host <-> device legs of a step.
+
+    Rows are independent, so the forward pass runs chunk by chunk: chunk i is transformed
+    while chunk i+1 is still arriving and chunk i-1 is already on its way back, and the
+    copies of the two directions (y going out, dy coming in) share the link.  `join()`
+    makes the current stream wait for everything queued on the copy streams.
+    """
+
+    def __init__(self, chunk_rows: int = 8192):
+        self.chunk_rows = int(chunk_rows)
+        self.s_in = torch.cuda.Stream()
+        self.s_out = torch.cuda.Stream()
+
+    def chunks(self, T: int):
+        return [(r, min(T, r + self.chunk_rows)) for r in range(0, T, self.chunk_rows)]
+
+    def join(self):
+        cur = torch.cuda.current_stream()
+        cur.wait_stream(self.s_in)
+        cur.wait_stream(self.s_out)
+
+
+def forward_host(x_host, a_host, b_host, y_host, staging, stream=None, pipe: HostPipe | None = None):
     """End-to-end forward from pinned host memory: copy in, transform, copy out.
 
-    `staging` is a dict of preallocated device tensors {"x", "a", "b", "y"}.
-    All copies are asynchronous on the current stream.
+    `staging` is a dict of preallocated device tensors {"x", "a", "b", "y"}.  Without `pipe`
+    all copies are asynchronous on the current stream; with a HostPipe the rows move in chunks
+    on its copy streams and the caller ends the step with pipe.join().
     """
-    staging["x"].copy_(x_host, non_blocking=True)
-    staging["a"].copy_(a_host, non_blocking=True)
-    staging["b"].copy_(b_host, non_blocking=True)
-    forward(staging["x"], staging["a"], staging["b"], out=staging["y"], stream=stream)
-    y_host.copy_(staging["y"], non_blocking=True)
+    if pipe is None:
+        staging["x"].copy_(x_host, non_blocking=True)
+        staging["a"].copy_(a_host, non_blocking=True)
+        staging["b"].copy_(b_host, non_blocking=True)
+        forward(staging["x"], staging["a"], staging["b"], out=staging["y"], stream=stream)
+        y_host.copy_(staging["y"], non_blocking=True)
+        return y_host
+    cur = torch.cuda.current_stream() if stream is None else stream
+    xs, ys, a, b = staging["x"], staging["y"], staging["a"], staging["b"]
+    d = xs.shape[-1]
+    code = dtype_code(xs, a)
+    pipe.s_in.wait_stream(cur)   # the staging buffers may still be in use by earlier work
+    pipe.s_out.wait_stream(cur)
+    with torch.cuda.stream(pipe.s_in):
+        a.copy_(a_host, non_blocking=True)
+        b.copy_(b_host, non_blocking=True)
+    for r0, r1 in pipe.chunks(xs.shape[0]):
+        with torch.cuda.stream(pipe.s_in):
+            xs[r0:r1].copy_(x_host[r0:r1], non_blocking=True)
+            arrived = torch.cuda.Event()
+            arrived.record(pipe.s_in)
+        cur.wait_event(arrived)
+        wht_affine_fwd(xs[r0:r1], a, b, ys[r0:r1], r1 - r0, d, code, cur)
+        done = torch.cuda.Event()
+        done.record(cur)
+        pipe.s_out.wait_event(done)
+        with torch.cuda.stream(pipe.s_out):
+            y_host[r0:r1].copy_(ys[r0:r1], non_blocking=True)
     return y_host
 
 
-def backward_host(dy_host, x_host, a_host, dx_host, da_host, db_host, staging, stream=None):
+def backward_host(dy_host, x_host, a_host, dx_host, da_host, db_host, staging, stream=None,
+                  pipe: HostPipe | None = None, x_resident: bool = False):
     """End-to-end backward from pinned host memory; `staging` holds device tensors
-    {"dy", "x", "a", "dx", "da", "db"}."""
+    {"dy", "x", "a", "dx", "da", "db"}.  `x_resident` skips the copy of x and a when the forward
+    call of the same step has just put them on the device (as in training)."""
     st = staging
-    st["dy"].copy_(dy_host, non_blocking=True)
-    st["x"].copy_(x_host, non_blocking=True)
-    st["a"].copy_(a_host, non_blocking=True)
     d = st["x"].shape[-1]
     T = st["x"].numel() // d
-    wht_affine_bwd(st["dy"], st["x"], st["a"], st["dx"], st["da"], st["db"], T, d,
-                   dtype_code(st["x"], st["a"]), stream)
-    dx_host.copy_(st["dx"], non_blocking=True)
-    da_host.copy_(st["da"], non_blocking=True)
-    db_host.copy_(st["db"], non_blocking=True)
+    code = dtype_code(st["x"], st["a"])
+    if pipe is None:
+        st["dy"].copy_(dy_host, non_blocking=True)
+        if not x_resident:
+            st["x"].copy_(x_host, non_blocking=True)
+            st["a"].copy_(a_host, non_blocking=True)
+        wht_affine_bwd(st["dy"], st["x"], st["a"], st["dx"], st["da"], st["db"], T, d, code, stream)
+        dx_host.copy_(st["dx"], non_blocking=True)
+        da_host.copy_(st["da"], non_blocking=True)
+        db_host.copy_(st["db"], non_blocking=True)
+        return
+    cur = torch.cuda.current_stream() if stream is None else stream
+    # dy comes in on the copy stream (sharing the link with the forward's y going out); the
+    # column sums need every row, so the kernel runs once, after the last chunk has arrived
+    with torch.cuda.stream(pipe.s_in):
+        if not x_resident:
+            st["x"].copy_(x_host, non_blocking=True)
+            st["a"].copy_(a_host, non_blocking=True)
+        for r0, r1 in pipe.chunks(T):
+            st["dy"][r0:r1].copy_(dy_host[r0:r1], non_blocking=True)
+        arrived = torch.cuda.Event()
+        arrived.record(pipe.s_in)
+    cur.wait_event(arrived)
+    wht_affine_bwd(st["dy"], st["x"], st["a"], st["dx"], st["da"], st["db"], T, d, code, cur)
+    done = torch.cuda.Event()
+    done.record(cur)
+    pipe.s_out.wait_event(done)
+    with torch.cuda.stream(pipe.s_out):
+        for r0, r1 in pipe.chunks(T):
+            dx_host[r0:r1].copy_(st["dx"][r0:r1], non_blocking=True)
+        da_host.copy_(st["da"], non_blocking=True)
+        db_host.copy_(st["db"], non_blocking=True)

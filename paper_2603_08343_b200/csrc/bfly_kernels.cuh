@@ -286,6 +286,8 @@ bfly_bwd_kernel(const TIO* dy, const TIO* x, const TP* __restrict__ a, TIO* dx,
 __global__ void __launch_bounds__(256)
 dadb_finalize_kernel(const float* __restrict__ partials, int nparts, int d, float inv_sqrt_d,
                      float* __restrict__ da, float* __restrict__ db) {
+    grid_dependency_wait();  // the partials come from the kernel launched just before
+    grid_launch_dependents();
     const int j = blockIdx.x * blockDim.x + threadIdx.x;
     if (j >= 2 * d) return;
     const int which = j / d;

@@ -339,6 +339,8 @@ mma_fwd_kernel(const __nv_bfloat16* x, const TP* __restrict__ a, const TP* __res
     uint32_t hf[4];
     make_h16_fragment(hf, lane);
     const F2 rs2 = f2(inv_sqrt_d, inv_sqrt_d);
+    grid_dependency_wait();
+    grid_launch_dependents();
 
     int parity = 0;
     const long long stride = static_cast<long long>(gridDim.x) * RG;

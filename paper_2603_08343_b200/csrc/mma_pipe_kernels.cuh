@@ -298,6 +298,8 @@ __global__ void __launch_bounds__(1024)
 dadb_finalize32_kernel(const float* __restrict__ partials, int nparts, int d, float inv_sqrt_d,
                        float* __restrict__ da, float* __restrict__ db) {
     __shared__ float red[32][33];
+    grid_dependency_wait();  // the partials come from the kernel launched just before
+    grid_launch_dependents();
     const int cx = threadIdx.x & 31;
     const int sl = threadIdx.x >> 5;
     const int j = blockIdx.x * 32 + cx;  // column in [0, 2d): da columns then db columns

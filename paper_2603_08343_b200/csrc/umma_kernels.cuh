@@ -114,14 +114,32 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
 // make this thread's shared-memory writes visible to the async proxy (tensor core reads)
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
-// Bounded wait that also gives up as soon as another role has raised the abort flag.
+// try_wait that lets the hardware park the thread for up to `ns` nanoseconds (it is woken as
+// soon as the phase completes), so a waiting warp does not burn issue slots polling.
+__device__ __forceinline__ bool mbar_try_wait_for(uint64_t* bar, uint32_t parity, uint32_t ns) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity), "r"(ns)
+        : "memory");
+    return ok != 0;
+}
+
+// Bounded wait (at least a few tenths of a second in all) that also gives up as soon as
+// another role has raised the abort flag.
 __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag) {
-    for (uint32_t i = 0; i < (1u << 22); ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+    for (uint32_t i = 0; i < (1u << 16); ++i) {
+        if (mbar_try_wait_for(bar, parity, 20000u)) return true;
+        if (*abort_flag) return false;
+    }
+    for (uint32_t i = 0; i < (1u << 20); ++i) {  // in case the hint is not honoured
         if (mbar_try_wait(bar, parity)) return true;
-        if (i > 16) {
-            if (*abort_flag) return false;
-            __nanosleep(32);
-        }
+        if (*abort_flag) return false;
+        __nanosleep(256);
     }
     *abort_flag = 1;
     atomicExch(&g_wht_device_error, kDeviceErrWaitExpired);
@@ -275,11 +293,6 @@ umma_fwd_kernel(const __nv_bfloat16* x, const TP* __restrict__ a, const TP* __re
         fence_mbar_init();
     }
     write_h128(smem_raw + L::OFF_H, tid, Geo::THREADS);
-    if constexpr (L::PARAMS_IN_SMEM) {
-        float* pa = reinterpret_cast<float*>(smem_raw + L::OFF_PARAMS);
-        stage_params_umma<Geo::D>(a, pa, inv_sqrt_d, tid, Geo::THREADS);
-        stage_params_umma<Geo::D>(b, pa + Geo::D, 1.0f, tid, Geo::THREADS);
-    }
     fence_async_smem();  // H_128 was written by ordinary stores and is read by the tensor core
     if (warp == 1) {
         tmem_alloc(tmem_slot, L::TMEM_COLS);
@@ -289,6 +302,15 @@ umma_fwd_kernel(const __nv_bfloat16* x, const TP* __restrict__ a, const TP* __re
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    // everything above touched only this CTA's own shared and tensor memory
+    grid_dependency_wait();
+    grid_launch_dependents();
+    if constexpr (L::PARAMS_IN_SMEM) {
+        float* pa = reinterpret_cast<float*>(smem_raw + L::OFF_PARAMS);
+        stage_params_umma<Geo::D>(a, pa, inv_sqrt_d, tid, Geo::THREADS);
+        stage_params_umma<Geo::D>(b, pa + Geo::D, 1.0f, tid, Geo::THREADS);
+        __syncthreads();
+    }
 
     if (warp == 0) {
         if (lane == 0) {
@@ -425,7 +447,17 @@ umma_bwd_kernel(const __nv_bfloat16* dy, const __nv_bfloat16* x, const TP* __res
                 float* __restrict__ partials, long long T, float inv_sqrt_d) {
     using Geo = UmmaGeo<LOGD, NCOL>;
     using L = UmmaBwdSmem<LOGD, NCOL, STAGES>;
-    static_assert(Geo::R <= 32, "per-thread accumulators must fit in registers");
+    // How the two groups of four epilogue warps share a tile.  Up to 32 values per row and
+    // thread (d <= 4096) each group takes half of the rows.  Beyond that the per-thread
+    // accumulators for all channels would not fit in registers, so each group takes ALL rows
+    // but only the channels whose top index bit equals its group number: the stage on that
+    // bit is applied first, straight on the accumulator columns (each thread reads both
+    // halves from TMEM and keeps lo + hi or lo - hi), and for dx last, in the same way.
+    constexpr bool SPLIT = Geo::R > 32;
+    constexpr int RE = SPLIT ? Geo::R / 2 : Geo::R;      // values per row a thread works on
+    constexpr int PE = RE / 8;                           // pieces per row a thread works on
+    constexpr int NROW = SPLIT ? Geo::ROWS : Geo::RPW;   // rows per tile a thread works on
+    static_assert(RE <= 32, "per-thread accumulators must fit in registers");
     extern __shared__ __align__(1024) unsigned char umma_smem[];
     unsigned char* const smem_raw = umma_smem;
     unsigned char* ring = smem_raw + L::OFF_RING;
@@ -471,14 +503,17 @@ umma_bwd_kernel(const __nv_bfloat16* dy, const __nv_bfloat16* x, const TP* __res
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    // everything above touched only this CTA's own shared and tensor memory
+    grid_dependency_wait();
+    grid_launch_dependents();
     const uint32_t tmem_d1 = tmem_base;
     const uint32_t tmem_d2 = tmem_base + 2 * Geo::N;
 
     // per-thread partial column sums (epilogue warps only; declared here so that the fold
     // after the role loops can see them)
-    F2 da_acc[Geo::PIECES][4], db_acc[Geo::PIECES][4];
+    F2 da_acc[PE][4], db_acc[PE][4];
 #pragma unroll
-    for (int p = 0; p < Geo::PIECES; ++p) {
+    for (int p = 0; p < PE; ++p) {
 #pragma unroll
         for (int j = 0; j < 4; ++j) { da_acc[p][j] = f2(0.0f, 0.0f); db_acc[p][j] = f2(0.0f, 0.0f); }
     }
@@ -554,45 +589,80 @@ umma_bwd_kernel(const __nv_bfloat16* dy, const __nv_bfloat16* x, const TP* __res
         const int q = warp & 3;
         const int ch = (warp - 2) >> 2;
         const int m = q * 32 + lane;
-        const uint32_t lane_off = (static_cast<uint32_t>(q * 32) << 16) + ch * Geo::CPW;
+        const int piece0 = SPLIT ? ch * PE : 0;  // first piece of the channels this thread owns
+        const F2 top_sign = ch ? f2(-1.0f, -1.0f) : f2(1.0f, 1.0f);  // split: lo + hi or lo - hi
+        // TMEM address of this thread's lane; the non-split groups start at their half of the columns
+        const uint32_t lane_off = (static_cast<uint32_t>(q * 32) << 16) + (SPLIT ? 0 : ch * Geo::CPW);
 
-        F2 as[Geo::PIECES][4];
+        F2 as[PE][4];
         {
             const F2 rs2 = f2(inv_sqrt_d, inv_sqrt_d);
 #pragma unroll
-            for (int p = 0; p < Geo::PIECES; ++p) {
-                load_params8(a + p * 1024 + m * 8, as[p]);
+            for (int p = 0; p < PE; ++p) {
+                load_params8(a + (piece0 + p) * 1024 + m * 8, as[p]);
 #pragma unroll
                 for (int j = 0; j < 4; ++j) as[p][j] = mul2(as[p][j], rs2);
             }
         }
 
-        // dx rows of tile j: read D2, round, store
+        // RE values of row r of this thread's share, from accumulator `acc`: the columns as they
+        // are, or (split) the top-bit stage lo +- hi of the two column halves of the row
+        auto row_values = [&](uint32_t acc, int r, float (&v)[RE], const float* preloaded) {
+            if constexpr (SPLIT) {
+                float lo[RE], hi[RE];
+                tmem_ld_cols<RE>(acc + lane_off + r * Geo::R, lo);
+                tmem_ld_cols<RE>(acc + lane_off + r * Geo::R + RE, hi);
+                tmem_wait_ld();
+#pragma unroll
+                for (int i = 0; i < RE; i += 2) {
+                    const F2 l = f2(lo[i], lo[i + 1]), h = f2(hi[i], hi[i + 1]);
+                    const F2 o = fma2(h, top_sign, l);
+                    v[i] = o.x;
+                    v[i + 1] = o.y;
+                }
+            } else {
+#pragma unroll
+                for (int i = 0; i < RE; ++i) v[i] = preloaded[r * RE + i];
+            }
+        };
+
+        // dx rows of tile j: read D2, (split: top-bit stage,) round, store
         auto store_dx = [&](long long j) -> bool {
             const int t = static_cast<int>(j & 1);
             const uint32_t pt = static_cast<uint32_t>(j >> 1) & 1u;
             if (!warp_wait_or_abort(d2_full + t, pt, abort_flag)) return false;
             tc_fence_after();
-            float u[Geo::CPW];
-            tmem_ld_cols<Geo::CPW>(tmem_d2 + lane_off + t * Geo::N, u);
-            tmem_wait_ld();
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(d2_empty + t);
+            const uint32_t acc = tmem_d2 + t * Geo::N;
+            float u[SPLIT ? 1 : Geo::CPW];
+            if constexpr (!SPLIT) {
+                tmem_ld_cols<Geo::CPW>(acc + lane_off, u);
+                tmem_wait_ld();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(d2_empty + t);
+            }
             const long long tile = blockIdx.x + j * gridDim.x;
 #pragma unroll
-            for (int rl = 0; rl < Geo::RPW; ++rl) {
-                const long long row = tile * Geo::ROWS + ch * Geo::RPW + rl;
+            for (int r = 0; r < NROW; ++r) {
+                const long long row = tile * Geo::ROWS + (SPLIT ? r : ch * Geo::RPW + r);
+                float w[RE];
+                row_values(acc, r, w, u);
+                if constexpr (SPLIT) {
+                    if (r == NROW - 1) {
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(d2_empty + t);
+                    }
+                }
                 if (row < T) {
-                    uint4* dst = reinterpret_cast<uint4*>(dx + row * Geo::D + m * 8);
+                    uint4* dst = reinterpret_cast<uint4*>(dx + row * Geo::D + piece0 * 1024 + m * 8);
 #pragma unroll
-                    for (int p = 0; p < Geo::PIECES; ++p) {
-                        const float* w = u + rl * Geo::R + p * 8;
+                    for (int p = 0; p < PE; ++p) {
                         uint4 o;
-                        o.x = pack_bf16x2(w[0], w[1]);
-                        o.y = pack_bf16x2(w[2], w[3]);
-                        o.z = pack_bf16x2(w[4], w[5]);
-                        o.w = pack_bf16x2(w[6], w[7]);
+                        o.x = pack_bf16x2(w[p * 8 + 0], w[p * 8 + 1]);
+                        o.y = pack_bf16x2(w[p * 8 + 2], w[p * 8 + 3]);
+                        o.z = pack_bf16x2(w[p * 8 + 4], w[p * 8 + 5]);
+                        o.w = pack_bf16x2(w[p * 8 + 6], w[p * 8 + 7]);
                         __stcs(dst + p * 128, o);
                     }
                 }
@@ -611,34 +681,43 @@ umma_bwd_kernel(const __nv_bfloat16* dy, const __nv_bfloat16* x, const TP* __res
             // makes the copied dy bytes visible to this thread's ordinary loads
             if (!warp_wait_or_abort(full + s, ph, abort_flag)) { ok = false; break; }
             tc_fence_after();
-            float u[Geo::CPW];
-            tmem_ld_cols<Geo::CPW>(tmem_d1 + lane_off + t * Geo::N, u);
-            tmem_wait_ld();
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(d1_empty + t);
+            const uint32_t acc = tmem_d1 + t * Geo::N;
+            float u[SPLIT ? 1 : Geo::CPW];
+            if constexpr (!SPLIT) {
+                tmem_ld_cols<Geo::CPW>(acc + lane_off, u);
+                tmem_wait_ld();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(d1_empty + t);
+            }
 
             unsigned char* slot_x = ring + s * L::STAGE_BYTES;
             unsigned char* slot_dy = slot_x + Geo::TILE_BYTES;
             const long long tile = blockIdx.x + it * gridDim.x;
 #pragma unroll
-            for (int rl = 0; rl < Geo::RPW; ++rl) {
-                const int rt = ch * Geo::RPW + rl;  // row inside the tile
+            for (int r = 0; r < NROW; ++r) {
+                const int rt = SPLIT ? r : ch * Geo::RPW + r;  // row inside the tile
                 const bool valid = tile * Geo::ROWS + rt < T;
-                float v[Geo::R];
-#pragma unroll
-                for (int i = 0; i < Geo::R; ++i) v[i] = u[rl * Geo::R + i];
-                thread_stages<Geo::R>(v);  // v = (x H)[piece*1024 + m*8 + n], unnormalised
+                float v[RE];
+                row_values(acc, r, v, u);
+                if constexpr (SPLIT) {
+                    if (r == NROW - 1) {
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(d1_empty + t);
+                    }
+                }
+                thread_stages<RE>(v);  // v = (x H) at this thread's channels, unnormalised
                 if (!valid) {
                     // rows past T were never copied: their accumulator columns hold whatever the
                     // slot held before (possibly NaN), and 0 * NaN would poison the column sums
 #pragma unroll
-                    for (int i = 0; i < Geo::R; ++i) v[i] = 0.0f;
+                    for (int i = 0; i < RE; ++i) v[i] = 0.0f;
                 }
-                float g[Geo::R];
+                float g[RE];
 #pragma unroll
-                for (int p = 0; p < Geo::PIECES; ++p) {
-                    const int chunk = ((rt * Geo::PIECES + p) * 128 + m) * 16;
+                for (int p = 0; p < PE; ++p) {
+                    const int chunk = ((rt * Geo::PIECES + piece0 + p) * 128 + m) * 16;
                     uint4 raw = make_uint4(0u, 0u, 0u, 0u);
                     if (valid) raw = *reinterpret_cast<const uint4*>(slot_dy + chunk);
                     const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
@@ -652,10 +731,10 @@ umma_bwd_kernel(const __nv_bfloat16* dy, const __nv_bfloat16* x, const TP* __res
                         g[p * 8 + 2 * j + 1] = gv.y;
                     }
                 }
-                thread_stages<Geo::R>(g);  // the low and piece stages of the second transform
+                thread_stages<RE>(g);  // the register stages of the second transform
 #pragma unroll
-                for (int p = 0; p < Geo::PIECES; ++p) {
-                    const int chunk = ((rt * Geo::PIECES + p) * 128 + m) * 16;
+                for (int p = 0; p < PE; ++p) {
+                    const int chunk = ((rt * Geo::PIECES + piece0 + p) * 128 + m) * 16;
                     uint4 hi, lo;
                     split_hi_lo(f2(g[p * 8 + 0], g[p * 8 + 1]), hi.x, lo.x);
                     split_hi_lo(f2(g[p * 8 + 2], g[p * 8 + 3]), hi.y, lo.y);
@@ -681,40 +760,57 @@ umma_bwd_kernel(const __nv_bfloat16* dy, const __nv_bfloat16* x, const TP* __res
         tmem_dealloc(tmem_base, L::TMEM_COLS);
     }
 
-    // fold the two column halves (they hold different rows of the same channels) in a fixed
-    // order and publish this CTA's partial sums; the ring is free now
-    float* fold = reinterpret_cast<float*>(ring);
-    if (warp >= 6) {
-        const int m = (warp & 3) * 32 + lane;
+    float* out = partials + static_cast<size_t>(blockIdx.x) * 2 * Geo::D;
+    if constexpr (SPLIT) {
+        // every (channel, thread) pair is unique: publish straight from registers
+        if (warp >= 2) {
+            const int m = (warp & 3) * 32 + lane;
+            const int piece0 = ((warp - 2) >> 2) * PE;
 #pragma unroll
-        for (int p = 0; p < Geo::PIECES; ++p) {
-            float4* pd = reinterpret_cast<float4*>(fold) + ((0 * Geo::PIECES + p) * 2) * 128 + m;
-            float4* pb = reinterpret_cast<float4*>(fold) + ((1 * Geo::PIECES + p) * 2) * 128 + m;
-            pd[0] = make_float4(da_acc[p][0].x, da_acc[p][0].y, da_acc[p][1].x, da_acc[p][1].y);
-            pd[128] = make_float4(da_acc[p][2].x, da_acc[p][2].y, da_acc[p][3].x, da_acc[p][3].y);
-            pb[0] = make_float4(db_acc[p][0].x, db_acc[p][0].y, db_acc[p][1].x, db_acc[p][1].y);
-            pb[128] = make_float4(db_acc[p][2].x, db_acc[p][2].y, db_acc[p][3].x, db_acc[p][3].y);
+            for (int p = 0; p < PE; ++p) {
+                float4* oa = reinterpret_cast<float4*>(out + (piece0 + p) * 1024 + m * 8);
+                float4* ob = reinterpret_cast<float4*>(out + Geo::D + (piece0 + p) * 1024 + m * 8);
+                oa[0] = make_float4(da_acc[p][0].x, da_acc[p][0].y, da_acc[p][1].x, da_acc[p][1].y);
+                oa[1] = make_float4(da_acc[p][2].x, da_acc[p][2].y, da_acc[p][3].x, da_acc[p][3].y);
+                ob[0] = make_float4(db_acc[p][0].x, db_acc[p][0].y, db_acc[p][1].x, db_acc[p][1].y);
+                ob[1] = make_float4(db_acc[p][2].x, db_acc[p][2].y, db_acc[p][3].x, db_acc[p][3].y);
+            }
         }
-    }
-    __syncthreads();
-    if (warp >= 2 && warp < 6) {
-        const int m = (warp & 3) * 32 + lane;
-        float* out = partials + static_cast<size_t>(blockIdx.x) * 2 * Geo::D;
+    } else {
+        // fold the two row halves (different rows of the same channels) in a fixed order and
+        // publish this CTA's partial sums; the ring is free now
+        float* fold = reinterpret_cast<float*>(ring);
+        if (warp >= 6) {
+            const int m = (warp & 3) * 32 + lane;
 #pragma unroll
-        for (int p = 0; p < Geo::PIECES; ++p) {
-            const float4* pd = reinterpret_cast<const float4*>(fold) + ((0 * Geo::PIECES + p) * 2) * 128 + m;
-            const float4* pb = reinterpret_cast<const float4*>(fold) + ((1 * Geo::PIECES + p) * 2) * 128 + m;
-            const float4 d0 = pd[0], d1 = pd[128], b0 = pb[0], b1 = pb[128];
-            float4* oa = reinterpret_cast<float4*>(out + p * 1024 + m * 8);
-            float4* ob = reinterpret_cast<float4*>(out + Geo::D + p * 1024 + m * 8);
-            oa[0] = make_float4(da_acc[p][0].x + d0.x, da_acc[p][0].y + d0.y, da_acc[p][1].x + d0.z,
-                                da_acc[p][1].y + d0.w);
-            oa[1] = make_float4(da_acc[p][2].x + d1.x, da_acc[p][2].y + d1.y, da_acc[p][3].x + d1.z,
-                                da_acc[p][3].y + d1.w);
-            ob[0] = make_float4(db_acc[p][0].x + b0.x, db_acc[p][0].y + b0.y, db_acc[p][1].x + b0.z,
-                                db_acc[p][1].y + b0.w);
-            ob[1] = make_float4(db_acc[p][2].x + b1.x, db_acc[p][2].y + b1.y, db_acc[p][3].x + b1.z,
-                                db_acc[p][3].y + b1.w);
+            for (int p = 0; p < PE; ++p) {
+                float4* pd = reinterpret_cast<float4*>(fold) + ((0 * PE + p) * 2) * 128 + m;
+                float4* pb = reinterpret_cast<float4*>(fold) + ((1 * PE + p) * 2) * 128 + m;
+                pd[0] = make_float4(da_acc[p][0].x, da_acc[p][0].y, da_acc[p][1].x, da_acc[p][1].y);
+                pd[128] = make_float4(da_acc[p][2].x, da_acc[p][2].y, da_acc[p][3].x, da_acc[p][3].y);
+                pb[0] = make_float4(db_acc[p][0].x, db_acc[p][0].y, db_acc[p][1].x, db_acc[p][1].y);
+                pb[128] = make_float4(db_acc[p][2].x, db_acc[p][2].y, db_acc[p][3].x, db_acc[p][3].y);
+            }
+        }
+        __syncthreads();
+        if (warp >= 2 && warp < 6) {
+            const int m = (warp & 3) * 32 + lane;
+#pragma unroll
+            for (int p = 0; p < PE; ++p) {
+                const float4* pd = reinterpret_cast<const float4*>(fold) + ((0 * PE + p) * 2) * 128 + m;
+                const float4* pb = reinterpret_cast<const float4*>(fold) + ((1 * PE + p) * 2) * 128 + m;
+                const float4 d0 = pd[0], d1 = pd[128], b0 = pb[0], b1 = pb[128];
+                float4* oa = reinterpret_cast<float4*>(out + p * 1024 + m * 8);
+                float4* ob = reinterpret_cast<float4*>(out + Geo::D + p * 1024 + m * 8);
+                oa[0] = make_float4(da_acc[p][0].x + d0.x, da_acc[p][0].y + d0.y, da_acc[p][1].x + d0.z,
+                                    da_acc[p][1].y + d0.w);
+                oa[1] = make_float4(da_acc[p][2].x + d1.x, da_acc[p][2].y + d1.y, da_acc[p][3].x + d1.z,
+                                    da_acc[p][3].y + d1.w);
+                ob[0] = make_float4(db_acc[p][0].x + b0.x, db_acc[p][0].y + b0.y, db_acc[p][1].x + b0.z,
+                                    db_acc[p][1].y + b0.w);
+                ob[1] = make_float4(db_acc[p][2].x + b1.x, db_acc[p][2].y + b1.y, db_acc[p][3].x + b1.z,
+                                    db_acc[p][3].y + b1.w);
+            }
         }
     }
 }

@@ -104,6 +104,24 @@ int resident_ctas(Kernel kernel, int threads, size_t smem, int dev, int* cache) 
     return cache[dev];
 }
 
+// Launch with the programmatic-stream-serialization attribute: the kernel may be scheduled
+// while its predecessor in the stream drains.  Only for kernels that call
+// grid_dependency_wait() before they touch global memory.
+template <typename... KArgs, typename... Args>
+void launch_overlapped(void (*kernel)(KArgs...), int grid, int block, size_t smem, cudaStream_t s, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(grid));
+    cfg.blockDim = dim3(static_cast<unsigned>(block));
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);  // errors are read by the caller (cudaGetLastError)
+}
+
 float inv_sqrt(int d) { return static_cast<float>(1.0 / sqrt(static_cast<double>(d))); }
 
 // Everything a launcher needs besides the tensors.
@@ -136,11 +154,11 @@ struct BwdArgs {
 
 int launch_finalize(const BwdArgs& g, int nparts, int d, cudaStream_t s) {
     if (d >= 32) {
-        dadb_finalize32_kernel<<<2 * d / 32, 1024, 0, s>>>(static_cast<const float*>(g.ws), nparts, d,
-                                                          inv_sqrt(d), g.da, g.db);
+        launch_overlapped(dadb_finalize32_kernel, 2 * d / 32, 1024, 0, s, static_cast<const float*>(g.ws), nparts, d,
+                          inv_sqrt(d), g.da, g.db);
     } else {
-        dadb_finalize_kernel<<<(2 * d + 255) / 256, 256, 0, s>>>(static_cast<const float*>(g.ws), nparts, d,
-                                                                inv_sqrt(d), g.da, g.db);
+        launch_overlapped(dadb_finalize_kernel, (2 * d + 255) / 256, 256, 0, s, static_cast<const float*>(g.ws),
+                          nparts, d, inv_sqrt(d), g.da, g.db);
     }
     WHT_CUDA_TRY(cudaGetLastError());
     return WHT_OK;
@@ -228,9 +246,9 @@ int launch_mma_fwd(const FwdArgs& f, const Ctx& c) {
     const int per_sm = resident_ctas(kernel, Geo::THREADS, Geo::SMEM_FWD, c.dev, occ);
     if (per_sm <= 0) return cuda_fail(cudaGetLastError());
     const int grid = capped_grid(ceil_div(c.T, RG), c.sms, per_sm);
-    kernel<<<grid, Geo::THREADS, Geo::SMEM_FWD, c.stream>>>(
-        static_cast<const __nv_bfloat16*>(f.x), static_cast<const TP*>(f.a), static_cast<const TP*>(f.b),
-        static_cast<__nv_bfloat16*>(f.y), static_cast<long long>(c.T), inv_sqrt(Geo::D));
+    launch_overlapped(kernel, grid, Geo::THREADS, Geo::SMEM_FWD, c.stream,
+                      static_cast<const __nv_bfloat16*>(f.x), static_cast<const TP*>(f.a), static_cast<const TP*>(f.b),
+                      static_cast<__nv_bfloat16*>(f.y), static_cast<long long>(c.T), inv_sqrt(Geo::D));
     WHT_CUDA_TRY(cudaGetLastError());
     return WHT_OK;
 }
@@ -359,9 +377,9 @@ int launch_umma_fwd(const FwdArgs& f, const Ctx& c) {
     int rc = prepare_umma(kernel, L::BYTES, c.dev, ready);
     if (rc != WHT_OK) return rc;
     const int grid = capped_grid(ceil_div(c.T, Geo::ROWS), c.sms, 1);
-    kernel<<<grid, Geo::THREADS, L::BYTES, c.stream>>>(
-        static_cast<const __nv_bfloat16*>(f.x), static_cast<const TP*>(f.a), static_cast<const TP*>(f.b),
-        static_cast<__nv_bfloat16*>(f.y), static_cast<long long>(c.T), inv_sqrt(Geo::D));
+    launch_overlapped(kernel, grid, Geo::THREADS, L::BYTES, c.stream,
+                      static_cast<const __nv_bfloat16*>(f.x), static_cast<const TP*>(f.a), static_cast<const TP*>(f.b),
+                      static_cast<__nv_bfloat16*>(f.y), static_cast<long long>(c.T), inv_sqrt(Geo::D));
     WHT_CUDA_TRY(cudaGetLastError());
     return WHT_OK;
 }
@@ -379,10 +397,10 @@ int launch_umma_bwd(const BwdArgs& g, const Ctx& c) {
     }
     const int grid = capped_grid(ceil_div(c.T, Geo::ROWS), c.sms, 1);
     return run_bwd_with_grid(g, c, grid, Geo::D, [&](int n) {
-        kernel<<<n, Geo::THREADS, L::BYTES, c.stream>>>(
-            static_cast<const __nv_bfloat16*>(g.dy), static_cast<const __nv_bfloat16*>(g.x),
-            static_cast<const TP*>(g.a), static_cast<__nv_bfloat16*>(g.dx), static_cast<float*>(g.ws),
-            static_cast<long long>(c.T), inv_sqrt(Geo::D));
+        launch_overlapped(kernel, n, Geo::THREADS, L::BYTES, c.stream,
+                          static_cast<const __nv_bfloat16*>(g.dy), static_cast<const __nv_bfloat16*>(g.x),
+                          static_cast<const TP*>(g.a), static_cast<__nv_bfloat16*>(g.dx), static_cast<float*>(g.ws),
+                          static_cast<long long>(c.T), inv_sqrt(Geo::D));
     });
 }
 
@@ -403,12 +421,13 @@ int dispatch_umma_bwd(int logd, const BwdArgs& g, const Ctx& c) {
         case 10: return launch_umma_bwd<10, 128, 3, TP>(g, c);
         case 11: return launch_umma_bwd<11, 128, 3, TP>(g, c);
         case 12: return launch_umma_bwd<12, 64, 5, TP>(g, c);
+        case 13: return launch_umma_bwd<13, 128, 3, TP>(g, c);
     }
     return WHT_ERR_BAD_DIM;
 }
 
 bool umma_fwd_supported(int logd, int dtype) { return dtype != WHT_F32 && logd >= 10 && logd <= 13; }
-bool umma_bwd_supported(int logd, int dtype) { return dtype != WHT_F32 && logd >= 10 && logd <= 12; }
+bool umma_bwd_supported(int logd, int dtype) { return dtype != WHT_F32 && logd >= 10 && logd <= 13; }
 
 bool mma_supported(int logd, int dtype) { return dtype != WHT_F32 && logd >= 9 && logd <= 13; }
 

@@ -61,6 +61,19 @@ __device__ __forceinline__ void bfly8(float (&v)[8]) {
     }
 }
 
+// ---- programmatic dependent launch ------------------------------------------------
+// A kernel launched with the "programmatic stream serialization" attribute may be
+// scheduled while the kernel before it in the stream is still running: its CTAs
+// take SMs as they become free and run their set-up.  grid_dependency_wait() then
+// blocks until that earlier kernel has completed and its writes are visible; no
+// global memory may be read or written before it.  grid_launch_dependents() lets
+// the kernel AFTER this one start in the same way.  Both are no-ops in a kernel
+// launched without the attribute / followed by a kernel launched without it.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_launch_dependents() {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
 constexpr __host__ __device__ int ilog2_c(int v) { return v <= 1 ? 0 : 1 + ilog2_c(v >> 1); }
 constexpr __host__ __device__ int imin_c(int a, int b) { return a < b ? a : b; }
 constexpr __host__ __device__ int imax_c(int a, int b) { return a > b ? a : b; }
