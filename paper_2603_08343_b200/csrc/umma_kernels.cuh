@@ -626,9 +626,18 @@ umma_bwd_kernel(const __nv_bfloat16* dy, const __nv_bfloat16* x, const TP* __res
             }
         };
 
+        __nv_bfloat16* const dx_thr = dx + piece0 * 1024 + m * 8;  // this thread's 8 columns of piece0
+        const int ntiles = static_cast<int>(my_tiles);
+        // valid rows of this CTA's j-th tile (the last tile of the problem may be ragged)
+        auto rows_in_tile = [&](int j, long long& row0) -> int {
+            row0 = (static_cast<long long>(blockIdx.x) + static_cast<long long>(j) * gridDim.x) * Geo::ROWS;
+            const long long left = T - row0;
+            return left < Geo::ROWS ? static_cast<int>(left) : Geo::ROWS;
+        };
+
         // dx rows of tile j: read D2, (split: top-bit stage,) round, store
-        auto store_dx = [&](long long j) -> bool {
-            const int t = static_cast<int>(j & 1);
+        auto store_dx = [&](int j) -> bool {
+            const int t = j & 1;
             const uint32_t pt = static_cast<uint32_t>(j >> 1) & 1u;
             if (!warp_wait_or_abort(d2_full + t, pt, abort_flag)) return false;
             tc_fence_after();
@@ -641,21 +650,15 @@ umma_bwd_kernel(const __nv_bfloat16* dy, const __nv_bfloat16* x, const TP* __res
                 __syncwarp();
                 if (lane == 0) mbar_arrive(d2_empty + t);
             }
-            const long long tile = blockIdx.x + j * gridDim.x;
+            long long row0;
+            const int nvalid = rows_in_tile(j, row0);
+            uint4* const dst0 = reinterpret_cast<uint4*>(dx_thr + row0 * Geo::D);
 #pragma unroll
             for (int r = 0; r < NROW; ++r) {
-                const long long row = tile * Geo::ROWS + (SPLIT ? r : ch * Geo::RPW + r);
-                float w[RE];
-                row_values(acc, r, w, u);
-                if constexpr (SPLIT) {
-                    if (r == NROW - 1) {
-                        tc_fence_before();
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(d2_empty + t);
-                    }
-                }
-                if (row < T) {
-                    uint4* dst = reinterpret_cast<uint4*>(dx + row * Geo::D + piece0 * 1024 + m * 8);
+                const int rt = SPLIT ? r : ch * Geo::RPW + r;  // row inside the tile
+                if (rt < nvalid) {                              // uniform over the warp
+                    float w[RE];
+                    row_values(acc, r, w, u);
 #pragma unroll
                     for (int p = 0; p < PE; ++p) {
                         uint4 o;
@@ -663,18 +666,23 @@ umma_bwd_kernel(const __nv_bfloat16* dy, const __nv_bfloat16* x, const TP* __res
                         o.y = pack_bf16x2(w[p * 8 + 2], w[p * 8 + 3]);
                         o.z = pack_bf16x2(w[p * 8 + 4], w[p * 8 + 5]);
                         o.w = pack_bf16x2(w[p * 8 + 6], w[p * 8 + 7]);
-                        __stcs(dst + p * 128, o);
+                        __stcs(dst0 + rt * (Geo::D / 8) + p * 128, o);
                     }
                 }
+            }
+            if constexpr (SPLIT) {
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(d2_empty + t);
             }
             return true;
         };
 
         bool ok = true;
-        for (long long it = 0; ok && it < my_tiles; ++it) {
-            const int s = static_cast<int>(it % STAGES);
+        for (int it = 0; ok && it < ntiles; ++it) {
+            const int s = it % STAGES;
             const uint32_t ph = static_cast<uint32_t>(it / STAGES) & 1u;
-            const int t = static_cast<int>(it & 1);
+            const int t = it & 1;
             const uint32_t pt = static_cast<uint32_t>(it >> 1) & 1u;
             if (!warp_wait_or_abort(d1_full + t, pt, abort_flag)) { ok = false; break; }
             // the first product ran, so the tile has landed; observing the barrier ourselves
@@ -691,65 +699,61 @@ umma_bwd_kernel(const __nv_bfloat16* dy, const __nv_bfloat16* x, const TP* __res
                 if (lane == 0) mbar_arrive(d1_empty + t);
             }
 
-            unsigned char* slot_x = ring + s * L::STAGE_BYTES;
-            unsigned char* slot_dy = slot_x + Geo::TILE_BYTES;
-            const long long tile = blockIdx.x + it * gridDim.x;
+            // this thread's 16-byte chunk of piece0 of row 0 of the tile, in the x and dy slots
+            unsigned char* const cx = ring + s * L::STAGE_BYTES + (piece0 * 128 + m) * 16;
+            unsigned char* const cdy = cx + Geo::TILE_BYTES;
+            long long row0;
+            const int nvalid = rows_in_tile(it, row0);
 #pragma unroll
             for (int r = 0; r < NROW; ++r) {
                 const int rt = SPLIT ? r : ch * Geo::RPW + r;  // row inside the tile
-                const bool valid = tile * Geo::ROWS + rt < T;
-                float v[RE];
-                row_values(acc, r, v, u);
-                if constexpr (SPLIT) {
-                    if (r == NROW - 1) {
-                        tc_fence_before();
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(d1_empty + t);
+                // Rows past T were never copied: their accumulator columns and slot bytes hold
+                // whatever was there before.  They are skipped altogether (uniformly over the
+                // warp); the second product then reads stale columns for them, which nobody stores.
+                if (rt < nvalid) {
+                    float v[RE];
+                    row_values(acc, r, v, u);
+                    thread_stages<RE>(v);  // v = (x H) at this thread's channels, unnormalised
+                    float g[RE];
+#pragma unroll
+                    for (int p = 0; p < PE; ++p) {
+                        const uint4 raw = *reinterpret_cast<const uint4*>(cdy + (rt * Geo::PIECES + p) * 2048);
+                        const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const F2 dyv = unpack_bf16x2(w[j]);
+                            da_acc[p][j] = fma2(dyv, f2(v[p * 8 + 2 * j], v[p * 8 + 2 * j + 1]), da_acc[p][j]);
+                            db_acc[p][j] = add2(db_acc[p][j], dyv);
+                            const F2 gv = mul2(as[p][j], dyv);
+                            g[p * 8 + 2 * j] = gv.x;
+                            g[p * 8 + 2 * j + 1] = gv.y;
+                        }
+                    }
+                    thread_stages<RE>(g);  // the register stages of the second transform
+#pragma unroll
+                    for (int p = 0; p < PE; ++p) {
+                        uint4 hi, lo;
+                        split_hi_lo(f2(g[p * 8 + 0], g[p * 8 + 1]), hi.x, lo.x);
+                        split_hi_lo(f2(g[p * 8 + 2], g[p * 8 + 3]), hi.y, lo.y);
+                        split_hi_lo(f2(g[p * 8 + 4], g[p * 8 + 5]), hi.z, lo.z);
+                        split_hi_lo(f2(g[p * 8 + 6], g[p * 8 + 7]), hi.w, lo.w);
+                        // the x tile is consumed (D1 is complete); this thread alone read this dy chunk
+                        *reinterpret_cast<uint4*>(cx + (rt * Geo::PIECES + p) * 2048) = hi;
+                        *reinterpret_cast<uint4*>(cdy + (rt * Geo::PIECES + p) * 2048) = lo;
                     }
                 }
-                thread_stages<RE>(v);  // v = (x H) at this thread's channels, unnormalised
-                if (!valid) {
-                    // rows past T were never copied: their accumulator columns hold whatever the
-                    // slot held before (possibly NaN), and 0 * NaN would poison the column sums
-#pragma unroll
-                    for (int i = 0; i < RE; ++i) v[i] = 0.0f;
-                }
-                float g[RE];
-#pragma unroll
-                for (int p = 0; p < PE; ++p) {
-                    const int chunk = ((rt * Geo::PIECES + piece0 + p) * 128 + m) * 16;
-                    uint4 raw = make_uint4(0u, 0u, 0u, 0u);
-                    if (valid) raw = *reinterpret_cast<const uint4*>(slot_dy + chunk);
-                    const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const F2 dyv = unpack_bf16x2(w[j]);
-                        da_acc[p][j] = fma2(dyv, f2(v[p * 8 + 2 * j], v[p * 8 + 2 * j + 1]), da_acc[p][j]);
-                        db_acc[p][j] = add2(db_acc[p][j], dyv);
-                        const F2 gv = mul2(as[p][j], dyv);
-                        g[p * 8 + 2 * j] = gv.x;
-                        g[p * 8 + 2 * j + 1] = gv.y;
-                    }
-                }
-                thread_stages<RE>(g);  // the register stages of the second transform
-#pragma unroll
-                for (int p = 0; p < PE; ++p) {
-                    const int chunk = ((rt * Geo::PIECES + piece0 + p) * 128 + m) * 16;
-                    uint4 hi, lo;
-                    split_hi_lo(f2(g[p * 8 + 0], g[p * 8 + 1]), hi.x, lo.x);
-                    split_hi_lo(f2(g[p * 8 + 2], g[p * 8 + 3]), hi.y, lo.y);
-                    split_hi_lo(f2(g[p * 8 + 4], g[p * 8 + 5]), hi.z, lo.z);
-                    split_hi_lo(f2(g[p * 8 + 6], g[p * 8 + 7]), hi.w, lo.w);
-                    *reinterpret_cast<uint4*>(slot_x + chunk) = hi;   // the x tile is consumed: D1 is complete
-                    *reinterpret_cast<uint4*>(slot_dy + chunk) = lo;  // this thread alone read this dy chunk
-                }
+            }
+            if constexpr (SPLIT) {
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(d1_empty + t);
             }
             fence_async_smem();
             __syncwarp();
             if (lane == 0) mbar_arrive(g_ready + s);
             if (it > 0) ok = store_dx(it - 1);
         }
-        if (ok && my_tiles > 0) ok = store_dx(my_tiles - 1);
+        if (ok && ntiles > 0) ok = store_dx(ntiles - 1);
     }
 
     tc_fence_before();
