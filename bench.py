@@ -38,10 +38,9 @@ from paper_2603_08343_b200 import workloads as wl
 
 METRIC = "wht_affine_tokens_per_s_fwd_bwd"
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the dominant kernel,
-# from the ncu capture summarised under profiles/; keyed by (workload, rows).  A quarter-size
-# case was captured and scaled by the rows (traffic is proportional to them).  Reset to {} when
-# the kernel changes.
-NCU_TRAFFIC_BYTES = {}
+# from the one-pass ncu capture at full size quoted in profiles/umma_bwd_training_d2048.txt;
+# keyed by (workload, rows).  Reset to {} when the kernel changes.
+NCU_TRAFFIC_BYTES = {("training", 65536): 536976384 + 224866048}  # umma_bwd_kernel<11,128,3>, full size
 UNIT = "tokens/s"
 
 
