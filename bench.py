@@ -268,6 +268,38 @@ def section_decode(B):
     return out
 
 
+def section_paper_shapes(B, hbm_peak):
+    """The paper's own inference shapes (its prefill table: batch 1024 x 64 tokens = 65536 rows; its
+    decode table: batch 2048, one row per sequence and step) at its two power-of-two model widths."""
+    out = {}
+    for d in (1024, 2048):
+        w = wl.Workload("paper", 1024 * 64, d, wl.WHT_BF16, "normal", 10 + d, False, "")
+        a, b = (t.cuda() for t in wl.gen_params(w))
+        x = wl.gen_full(w.with_rows(8192), "x").cuda().repeat(8, 1)
+        y = torch.empty_like(x)
+        ms = time_loop(lambda: B.wht_affine_fwd(x, a, b, y, w.T, w.d, w.dtype), 50, warmup=5)
+        gb = 2 * w.T * w.d * 2 / 1e9
+        entry = {"prefill_T": w.T, "prefill_fwd_us": 1e3 * ms, "prefill_fwd_GBps": gb / (ms * 1e-3),
+                 "prefill_frac_of_measured_peak": gb / (ms * 1e-3) / hbm_peak,
+                 "prefill_tokens_per_s": w.T / (ms * 1e-3)}
+        xd = x[:2048].contiguous()
+        yd = torch.empty_like(xd)
+        s = torch.cuda.Stream()
+        with torch.cuda.stream(s):
+            for _ in range(3):
+                B.wht_affine_fwd_decode(xd, a, b, yd, 2048, d, w.dtype)
+            torch.cuda.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=s):
+                for _ in range(50):
+                    B.wht_affine_fwd_decode(xd, a, b, yd, 2048, d, w.dtype)
+            entry["decode_T"] = 2048
+            entry["decode_graph_replay_us_per_call"] = 1e3 * time_loop(g.replay, 40, warmup=3) / 50
+        out[f"d{d}"] = entry
+        del x, y
+    return out
+
+
 def section_fwd_bwd(B, name, hbm_peak, iters):
     """Forward and backward timed separately on a workload larger than L2."""
     w = wl.CONFIGS[name]
@@ -285,6 +317,7 @@ def section_fwd_bwd(B, name, hbm_peak, iters):
     f_ms = time_loop(lambda: B.wht_affine_fwd(x, a, b, y, w.T, w.d, w.dtype), iters)
     b_ms = time_loop(lambda: B.wht_affine_bwd(dy, x, a, y, da, db, w.T, w.d, w.dtype), iters)
     c_ms = time_loop(lambda: B.wht_copy_rows(x, y, w.T, w.d, w.dtype), iters)
+    r_ms = time_loop(lambda: B.wht_affine_fwd_residual(x, a, b, dy, y, w.T, w.d, w.dtype), iters)
     fb = 2 * w.T * w.d * w.io_bytes / 1e9
     bb = 3 * w.T * w.d * w.io_bytes / 1e9
     res = {"T": w.T, "d": w.d, "rows_drawn": base_rows, "rows_tiled": reps,
@@ -292,7 +325,10 @@ def section_fwd_bwd(B, name, hbm_peak, iters):
            "fwd_frac_of_8000": fb / (f_ms * 1e-3) / 8000.0, "fwd_tokens_per_s": w.T / (f_ms * 1e-3),
            "bwd_us": 1e3 * b_ms, "bwd_GBps": bb / (b_ms * 1e-3), "bwd_frac_of_measured_peak": bb / (b_ms * 1e-3) / hbm_peak,
            "bwd_frac_of_8000": bb / (b_ms * 1e-3) / 8000.0, "bwd_tokens_per_s": w.T / (b_ms * 1e-3),
-           "copy_rows_GBps": fb / (c_ms * 1e-3)}
+           "copy_rows_GBps": fb / (c_ms * 1e-3),
+           # forward fused with the residual add: reads x and the residual stream, writes y (3 row tensors)
+           "fwd_residual_us": 1e3 * r_ms, "fwd_residual_GBps": bb / (r_ms * 1e-3),
+           "fwd_residual_frac_of_measured_peak": bb / (r_ms * 1e-3) / hbm_peak}
     # the dense projection this path replaces, as context: cuBLAS bf16 [T x d] x [d x d]
     if w.dtype != wl.WHT_F32:
         wmat = torch.randn(w.d, w.d, device="cuda", dtype=torch.bfloat16)
@@ -514,6 +550,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         sections["decode"] = section_decode(B)
         sections["training"] = section_fwd_bwd(B, "training", hbm_peak, 20)
         sections["large"] = section_fwd_bwd(B, "large", hbm_peak, 5)
+        sections["paper_shapes"] = section_paper_shapes(B, hbm_peak)
         out["sections"] = sections
     print(json.dumps(out))
     if world > 1:

@@ -66,6 +66,18 @@ int wht_affine_fwd(const void* x, const void* a, const void* b, void* y,
                    int64_t T, int32_t d, int dtype, void* stream);
 
 /*
+ * Forward pass fused with the residual connection that follows the attention block
+ * (the paper's Sec. 3 motivation: the projection's output feeds that connection):
+ *     y[t, :] = resid[t, :] + a (.) (x[t, :] H_d)/sqrt(d) + b
+ * resid [T x d] has the layout and storage type of x.  The sum is taken in fp32 and
+ * rounded once at the store.  y may alias resid or x exactly.  One kernel: reads x and
+ * resid once, writes y once (no separate add pass over HBM).  Its backward is that of
+ * wht_affine_fwd plus the identity for resid (d resid = dy), so wht_affine_bwd serves.
+ */
+int wht_affine_fwd_residual(const void* x, const void* a, const void* b, const void* resid, void* y,
+                            int64_t T, int32_t d, int dtype, void* stream);
+
+/*
  * Forward pass tuned for a handful of rows (the decode regime of the paper's
  * inference benchmark: one new token per sequence).  Same arguments, semantics
  * and results as wht_affine_fwd; any T is legal, T <= 256 is what it is shaped

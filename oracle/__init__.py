@@ -7,6 +7,7 @@ from .wht_oracle import (  # noqa: F401
     sylvester_hadamard,
     widen_bf16_bits,
     wht_affine_fwd,
+    wht_affine_fwd_residual,
     wht_affine_bwd,
     wht_normalised,
     da_db_columns,

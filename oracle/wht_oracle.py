@@ -21,7 +21,8 @@ What the paper fixes, and where:
 
 Pins (tests/test_oracle_pins.py): the printed H_4, scipy's Sylvester matrix,
 the Kronecker recursion, H H^T = d I in integers, norm preservation, involution,
-impulse and constant rows, brute force at d <= 16, the Fig. 2 butterfly with its
+impulse and constant rows, brute force at d <= 16 (also with a residual row added),
+the Fig. 2 butterfly with its
 d*log2(d) operation count, central finite differences and the adjoint identity
 for the gradients.  No function here is "parity unpinned".
 """
@@ -84,6 +85,12 @@ def wht_affine_fwd(x: np.ndarray, a: np.ndarray, b: np.ndarray) -> np.ndarray:
     b = np.asarray(b, dtype=np.float64)
     z = wht_normalised(x)
     return a[None, :] * z + b[None, :]
+
+
+def wht_affine_fwd_residual(x: np.ndarray, a: np.ndarray, b: np.ndarray, resid: np.ndarray) -> np.ndarray:
+    """out[t, j] = resid[t, j] + a[j] * z[t, j] + b[j]: Eq. 1 followed by the residual
+    connection of the attention block that the projection's output feeds (Sec. 3)."""
+    return np.asarray(resid, dtype=np.float64) + wht_affine_fwd(x, a, b)
 
 
 def wht_affine_bwd(dy: np.ndarray, x: np.ndarray, a: np.ndarray):

@@ -18,7 +18,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libwht_affine.so")
 
 EXPORTS = (
-    "wht_affine_fwd", "wht_affine_fwd_decode", "wht_affine_bwd", "wht_affine_bwd_ws", "wht_affine_bwd_noalloc",
+    "wht_affine_fwd", "wht_affine_fwd_residual", "wht_affine_fwd_decode", "wht_affine_bwd", "wht_affine_bwd_ws", "wht_affine_bwd_noalloc",
     "wht_affine_bwd_workspace_bytes", "wht_affine_set_variant", "wht_affine_get_variant",
     "wht_copy_rows", "wht_affine_device_status", "wht_affine_last_cuda_error", "wht_affine_status_string",
     "wht_affine_shutdown",
@@ -41,6 +41,7 @@ def _load() -> ctypes.CDLL:
     lib = ctypes.CDLL(LIB_PATH)
     vp, i64, i32, ci, sz = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32, ctypes.c_int, ctypes.c_size_t
     lib.wht_affine_fwd.argtypes = [vp, vp, vp, vp, i64, i32, ci, vp]
+    lib.wht_affine_fwd_residual.argtypes = [vp, vp, vp, vp, vp, i64, i32, ci, vp]
     lib.wht_affine_fwd_decode.argtypes = [vp, vp, vp, vp, i64, i32, ci, vp]
     lib.wht_affine_bwd.argtypes = [vp, vp, vp, vp, vp, vp, i64, i32, ci, vp]
     lib.wht_affine_bwd_noalloc.argtypes = [vp, vp, vp, vp, vp, vp, i64, i32, ci, vp]
@@ -96,6 +97,13 @@ def wht_affine_fwd(x, a, b, y, T: int, d: int, dtype: int, stream=None) -> None:
     _require_cuda(x, a, b, y)
     _check(_lib.wht_affine_fwd(_ptr(x), _ptr(a), _ptr(b), _ptr(y), T, d, dtype, _stream(stream)),
            "wht_affine_fwd")
+
+
+def wht_affine_fwd_residual(x, a, b, resid, y, T: int, d: int, dtype: int, stream=None) -> None:
+    """y = resid + a (.) (x H)/sqrt(d) + b in one kernel (resid has the layout and type of x)."""
+    _require_cuda(x, a, b, resid, y)
+    _check(_lib.wht_affine_fwd_residual(_ptr(x), _ptr(a), _ptr(b), _ptr(resid), _ptr(y), T, d, dtype,
+                                        _stream(stream)), "wht_affine_fwd_residual")
 
 
 def wht_affine_fwd_decode(x, a, b, y, T: int, d: int, dtype: int, stream=None) -> None:
@@ -168,11 +176,14 @@ def dtype_code(x: torch.Tensor, a: torch.Tensor) -> int:
     raise ValueError(f"unsupported storage types x={x.dtype}, a={a.dtype}")
 
 
-def forward(x, a, b, out=None, decode: bool = False, stream=None):
-    """y = a (.) (x H)/sqrt(d) + b for x[..., d]; returns `out` (allocated if None)."""
+def forward(x, a, b, out=None, decode: bool = False, stream=None, resid=None):
+    """y = [resid +] a (.) (x H)/sqrt(d) + b for x[..., d]; returns `out` (allocated if None)."""
     d = x.shape[-1]
     T = x.numel() // d if d else 0
     y = torch.empty_like(x) if out is None else out
+    if resid is not None:
+        wht_affine_fwd_residual(x, a, b, resid, y, T, d, dtype_code(x, a), stream)
+        return y
     fn = wht_affine_fwd_decode if decode else wht_affine_fwd
     fn(x, a, b, y, T, d, dtype_code(x, a), stream)
     return y

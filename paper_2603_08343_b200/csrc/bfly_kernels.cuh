@@ -158,7 +158,7 @@ __device__ __forceinline__ void store8_stream(__nv_bfloat16* p, const float (&v)
 // ---- forward: y = a (.) (x H)/sqrt(d) + b ------------------------------------
 template <int LOGD, typename TIO, typename TP>
 __global__ void __launch_bounds__(BflyGeo<LOGD>::THREADS)
-bfly_fwd_kernel(const TIO* x, const TP* __restrict__ a, const TP* __restrict__ b, TIO* y,
+bfly_fwd_kernel(const TIO* x, const TP* __restrict__ a, const TP* __restrict__ b, const TIO* resid, TIO* y,
                 long long T, float inv_sqrt_d) {
     using Geo = BflyGeo<LOGD>;
     extern __shared__ __align__(16) float smem[];
@@ -195,6 +195,12 @@ bfly_fwd_kernel(const TIO* x, const TP* __restrict__ a, const TP* __restrict__ b
             for (int c = 0; c < Geo::C; ++c) {
 #pragma unroll
                 for (int e = 0; e < 8; ++e) v[c][e] = fmaf(v[c][e], as[c][e], bs[c][e]);
+                if (resid != nullptr) {  // fused residual: summed in fp32, rounded once at the store
+                    float r[8];
+                    load8_stream(resid + row * Geo::D + (c * Geo::G + t) * 8, r);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) v[c][e] += r[e];
+                }
                 store8_stream(y + row * Geo::D + (c * Geo::G + t) * 8, v[c]);
             }
         }

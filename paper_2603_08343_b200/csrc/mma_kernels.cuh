@@ -270,6 +270,17 @@ __device__ __forceinline__ void fwd_store_chunk(const F2 (&v)[4], const F2 (&as)
     o.w = pack_bf16x2(fma2(v[3], as[3], bs[3]));
     __stcs(dst, o);
 }
+// y chunk = r + (as (.) v + b) with r the 8 stored residual values `res`: the sum is taken in
+// fp32 and rounded to bf16 once
+__device__ __forceinline__ void fwd_store_chunk_res(const F2 (&v)[4], const F2 (&as)[4], const F2 (&bs)[4],
+                                                    const uint4& res, uint4* dst) {
+    uint4 o;
+    o.x = pack_bf16x2(add2(fma2(v[0], as[0], bs[0]), unpack_bf16x2(res.x)));
+    o.y = pack_bf16x2(add2(fma2(v[1], as[1], bs[1]), unpack_bf16x2(res.y)));
+    o.z = pack_bf16x2(add2(fma2(v[2], as[2], bs[2]), unpack_bf16x2(res.z)));
+    o.w = pack_bf16x2(add2(fma2(v[3], as[3], bs[3]), unpack_bf16x2(res.w)));
+    __stcs(dst, o);
+}
 
 // backward, between the two transforms, one chunk: da += dy (.) u, db += dy, v <- as (.) dy
 __device__ __forceinline__ void bwd_mid_chunk(F2 (&v)[4], const uint4& rawdy, const F2 (&as)[4],
@@ -326,7 +337,7 @@ __device__ __forceinline__ void bwd_publish_partials(const F2 (&da_acc)[Geo::NT]
 template <int LOGD, int TB, int RG, typename TP>
 __global__ void __launch_bounds__(MmaGeo<LOGD, TB, RG>::THREADS)
 mma_fwd_kernel(const __nv_bfloat16* x, const TP* __restrict__ a, const TP* __restrict__ b,
-               __nv_bfloat16* y, long long T, float inv_sqrt_d) {
+               const __nv_bfloat16* resid, __nv_bfloat16* y, long long T, float inv_sqrt_d) {
     using Geo = MmaGeo<LOGD, TB, RG>;
     using X = MmaXform<Geo>;
     constexpr int NT = Geo::NT;
@@ -365,7 +376,12 @@ mma_fwd_kernel(const __nv_bfloat16* x, const TP* __restrict__ a, const TP* __res
             load_params8(b + (c * 32 + lane) * 8, bs);
 #pragma unroll
             for (int j = 0; j < 4; ++j) as[j] = mul2(as[j], rs2);
-            fwd_store_chunk(v[idx], as, bs, dst + c * 32 + lane);
+            if (resid != nullptr) {
+                const uint4 r = __ldcs(reinterpret_cast<const uint4*>(resid + row * Geo::D) + c * 32 + lane);
+                fwd_store_chunk_res(v[idx], as, bs, r, dst + c * 32 + lane);
+            } else {
+                fwd_store_chunk(v[idx], as, bs, dst + c * 32 + lane);
+            }
         }
     }
 }

@@ -110,7 +110,7 @@ __device__ __forceinline__ void read_staged8(const float* base, int c, int lane,
 template <int LOGD, int TB, int RG, int S, int MINB, typename TP>
 __global__ void __launch_bounds__(MmaGeo<LOGD, TB, RG>::THREADS, MINB)
 mma_fwd_pipe_kernel(const __nv_bfloat16* x, const TP* __restrict__ a, const TP* __restrict__ b,
-                    __nv_bfloat16* y, long long T, float inv_sqrt_d) {
+                    const __nv_bfloat16* resid, __nv_bfloat16* y, long long T, float inv_sqrt_d) {
     using Geo = PipeGeo<LOGD, TB, RG, S, false>;
     using X = MmaXform<Geo>;
     constexpr int NT = Geo::NT;
@@ -186,7 +186,12 @@ mma_fwd_pipe_kernel(const __nv_bfloat16* x, const TP* __restrict__ a, const TP* 
             F2 as[4], bs[4];
             read_staged8(pa, c, lane, as);
             read_staged8(pb, c, lane, bs);
-            fwd_store_chunk(v[idx], as, bs, dst + c * 32 + lane);
+            if (resid != nullptr) {
+                const uint4 r = __ldcs(reinterpret_cast<const uint4*>(resid + row * Geo::D) + c * 32 + lane);
+                fwd_store_chunk_res(v[idx], as, bs, r, dst + c * 32 + lane);
+            } else {
+                fwd_store_chunk(v[idx], as, bs, dst + c * 32 + lane);
+            }
         }
         if (++stage == S) { stage = 0; phase ^= 1; }
     }

@@ -262,10 +262,12 @@ __device__ __forceinline__ void stage_params_umma(const TP* __restrict__ src, fl
     }
 }
 
-template <int LOGD, int NCOL, int STAGES, typename TP>
+// RES: y = resid + (a (.) (x H)/sqrt(d) + b), the residual read in the store layout (each thread
+// its own 16-byte chunks, fetched before the accumulator is waited for).
+template <int LOGD, int NCOL, int STAGES, typename TP, bool RES>
 __global__ void __launch_bounds__(UmmaGeo<LOGD, NCOL>::THREADS, 1)
-umma_fwd_kernel(const __nv_bfloat16* x, const TP* __restrict__ a, const TP* __restrict__ b, __nv_bfloat16* y,
-                long long T, float inv_sqrt_d) {
+umma_fwd_kernel(const __nv_bfloat16* x, const TP* __restrict__ a, const TP* __restrict__ b,
+                const __nv_bfloat16* resid, __nv_bfloat16* y, long long T, float inv_sqrt_d) {
     using Geo = UmmaGeo<LOGD, NCOL>;
     using L = UmmaFwdSmem<LOGD, NCOL, STAGES, TP>;
     constexpr int ACC = L::ACC;
@@ -375,6 +377,21 @@ umma_fwd_kernel(const __nv_bfloat16* x, const TP* __restrict__ a, const TP* __re
         for (long long it = 0; it < my_tiles; ++it) {
             const int t = static_cast<int>(it % ACC);
             const uint32_t pt = static_cast<uint32_t>(it / ACC) & 1u;
+            uint4 res[RES ? Geo::RPW * Geo::PIECES : 1];
+            if constexpr (RES) {
+                const long long tile_r = blockIdx.x + it * gridDim.x;
+#pragma unroll
+                for (int rl = 0; rl < Geo::RPW; ++rl) {
+                    const long long row = tile_r * Geo::ROWS + ch * Geo::RPW + rl;
+#pragma unroll
+                    for (int p = 0; p < Geo::PIECES; ++p) {
+                        res[rl * Geo::PIECES + p] = make_uint4(0u, 0u, 0u, 0u);
+                        if (row < T)
+                            res[rl * Geo::PIECES + p] =
+                                __ldcs(reinterpret_cast<const uint4*>(resid + row * Geo::D + m * 8) + p * 128);
+                    }
+                }
+            }
             if (!warp_wait_or_abort(acc_full + t, pt, abort_flag)) break;
             tc_fence_after();
             float u[Geo::CPW];
@@ -405,9 +422,11 @@ umma_fwd_kernel(const __nv_bfloat16* x, const TP* __restrict__ a, const TP* __re
                             const float4 a0 = qa[0], a1 = qa[128], b0 = qb[0], b1 = qb[128];
                             F2 ap[4] = {f2(a0.x, a0.y), f2(a0.z, a0.w), f2(a1.x, a1.y), f2(a1.z, a1.w)};
                             F2 bp[4] = {f2(b0.x, b0.y), f2(b0.z, b0.w), f2(b1.x, b1.y), f2(b1.z, b1.w)};
-                            fwd_store_chunk(w, ap, bp, dst + p * 128);
+                            if constexpr (RES) fwd_store_chunk_res(w, ap, bp, res[rl * Geo::PIECES + p], dst + p * 128);
+                            else fwd_store_chunk(w, ap, bp, dst + p * 128);
                         } else {
-                            fwd_store_chunk(w, as[p], bs[p], dst + p * 128);
+                            if constexpr (RES) fwd_store_chunk_res(w, as[p], bs[p], res[rl * Geo::PIECES + p], dst + p * 128);
+                            else fwd_store_chunk(w, as[p], bs[p], dst + p * 128);
                         }
                     }
                 }

@@ -137,6 +137,7 @@ struct FwdArgs {
     const void* a;
     const void* b;
     void* y;
+    const void* resid = nullptr;  // fused residual input (layout and type of x), or none
 };
 
 struct BwdArgs {
@@ -193,7 +194,7 @@ int launch_bfly_fwd(const FwdArgs& f, const Ctx& c) {
     const int grid = capped_grid(ceil_div(c.T, Geo::R), c.sms, per_sm);
     kernel<<<grid, Geo::THREADS, Geo::SMEM_FWD, c.stream>>>(
         static_cast<const TIO*>(f.x), static_cast<const TP*>(f.a), static_cast<const TP*>(f.b),
-        static_cast<TIO*>(f.y), static_cast<long long>(c.T), inv_sqrt(Geo::D));
+        static_cast<const TIO*>(f.resid), static_cast<TIO*>(f.y), static_cast<long long>(c.T), inv_sqrt(Geo::D));
     WHT_CUDA_TRY(cudaGetLastError());
     return WHT_OK;
 }
@@ -248,7 +249,8 @@ int launch_mma_fwd(const FwdArgs& f, const Ctx& c) {
     const int grid = capped_grid(ceil_div(c.T, RG), c.sms, per_sm);
     launch_overlapped(kernel, grid, Geo::THREADS, Geo::SMEM_FWD, c.stream,
                       static_cast<const __nv_bfloat16*>(f.x), static_cast<const TP*>(f.a), static_cast<const TP*>(f.b),
-                      static_cast<__nv_bfloat16*>(f.y), static_cast<long long>(c.T), inv_sqrt(Geo::D));
+                      static_cast<const __nv_bfloat16*>(f.resid), static_cast<__nv_bfloat16*>(f.y),
+                      static_cast<long long>(c.T), inv_sqrt(Geo::D));
     WHT_CUDA_TRY(cudaGetLastError());
     return WHT_OK;
 }
@@ -280,7 +282,8 @@ int launch_mma_fwd_pipe(const FwdArgs& f, const Ctx& c) {
     const int grid = capped_grid(ceil_div(c.T, RG), c.sms, per_sm);
     kernel<<<grid, Geo::THREADS, Geo::SMEM, c.stream>>>(
         static_cast<const __nv_bfloat16*>(f.x), static_cast<const TP*>(f.a), static_cast<const TP*>(f.b),
-        static_cast<__nv_bfloat16*>(f.y), static_cast<long long>(c.T), inv_sqrt(Geo::D));
+        static_cast<const __nv_bfloat16*>(f.resid), static_cast<__nv_bfloat16*>(f.y), static_cast<long long>(c.T),
+        inv_sqrt(Geo::D));
     WHT_CUDA_TRY(cudaGetLastError());
     return WHT_OK;
 }
@@ -367,21 +370,28 @@ int prepare_umma(Kernel kernel, int smem, int dev, int* cache) {
     return WHT_OK;
 }
 
-template <int LOGD, int NCOL, int STAGES, typename TP>
-int launch_umma_fwd(const FwdArgs& f, const Ctx& c) {
+template <int LOGD, int NCOL, int STAGES, typename TP, bool RES>
+int launch_umma_fwd_impl(const FwdArgs& f, const Ctx& c) {
     using Geo = UmmaGeo<LOGD, NCOL>;
     using L = UmmaFwdSmem<LOGD, NCOL, STAGES, TP>;
     static_assert(L::BYTES > 116 * 1024, "must be alone on its SM");
     static int ready[kMaxDevices] = {};
-    auto kernel = umma_fwd_kernel<LOGD, NCOL, STAGES, TP>;
+    auto kernel = umma_fwd_kernel<LOGD, NCOL, STAGES, TP, RES>;
     int rc = prepare_umma(kernel, L::BYTES, c.dev, ready);
     if (rc != WHT_OK) return rc;
     const int grid = capped_grid(ceil_div(c.T, Geo::ROWS), c.sms, 1);
     launch_overlapped(kernel, grid, Geo::THREADS, L::BYTES, c.stream,
                       static_cast<const __nv_bfloat16*>(f.x), static_cast<const TP*>(f.a), static_cast<const TP*>(f.b),
-                      static_cast<__nv_bfloat16*>(f.y), static_cast<long long>(c.T), inv_sqrt(Geo::D));
+                      static_cast<const __nv_bfloat16*>(f.resid), static_cast<__nv_bfloat16*>(f.y),
+                      static_cast<long long>(c.T), inv_sqrt(Geo::D));
     WHT_CUDA_TRY(cudaGetLastError());
     return WHT_OK;
+}
+
+template <int LOGD, int NCOL, int STAGES, typename TP>
+int launch_umma_fwd(const FwdArgs& f, const Ctx& c) {
+    return f.resid ? launch_umma_fwd_impl<LOGD, NCOL, STAGES, TP, true>(f, c)
+                   : launch_umma_fwd_impl<LOGD, NCOL, STAGES, TP, false>(f, c);
 }
 
 template <int LOGD, int NCOL, int STAGES, typename TP>
@@ -538,6 +548,18 @@ int wht_affine_fwd_decode(const void* x, const void* a, const void* b, void* y, 
     if (rc != WHT_OK) return rc;
     if (T == 0) return WHT_OK;
     return run_fwd(FwdArgs{x, a, b, y}, T, d, dtype, static_cast<cudaStream_t>(stream), true);
+}
+
+int wht_affine_fwd_residual(const void* x, const void* a, const void* b, const void* resid, void* y, int64_t T,
+                            int32_t d, int dtype, void* stream) {
+    int rc = check_fwd_args(x, a, b, y, T, d, dtype);
+    if (rc != WHT_OK) return rc;
+    if (T > 0 && !resid) return WHT_ERR_NULL;
+    if (!aligned16(resid)) return WHT_ERR_MISALIGNED;
+    if (T == 0) return WHT_OK;
+    FwdArgs f{x, a, b, y};
+    f.resid = resid;
+    return run_fwd(f, T, d, dtype, static_cast<cudaStream_t>(stream), false);
 }
 
 size_t wht_affine_bwd_workspace_bytes(int64_t T, int32_t d, int dtype) {

@@ -46,6 +46,8 @@ def test_argument_errors_need_no_gpu(lib):
     assert lib.wht_affine_fwd(None, p, p, p, 4, 256, 0, s) == -1
     assert lib.wht_affine_fwd(p, p, p, off, 4, 256, 0, s) == -5
     assert lib.wht_affine_fwd_decode(p, None, p, p, 4, 256, 1, s) == -1
+    assert lib.wht_affine_fwd_residual(p, p, p, None, p, 4, 256, 1, s) == -1
+    assert lib.wht_affine_fwd_residual(p, p, p, off, p, 4, 256, 1, s) == -5
     assert lib.wht_affine_bwd(p, p, p, p, None, p, 4, 256, 2, s) == -1
     assert lib.wht_affine_bwd(p, off, p, p, p, p, 4, 256, 2, s) == -5
     assert lib.wht_affine_bwd_ws(p, p, p, p, p, p, 4, 100, 2, p, 64, s) == -2

@@ -123,6 +123,26 @@ def test_brute_force_small(d):
         assert y[t, j] == pytest.approx(a[j] * acc / math.sqrt(d) + b[j], abs=1e-13)
 
 
+@pytest.mark.parametrize("d", [2, 8, 16])
+def test_residual_form_brute_force_and_special_cases(d):
+    # out = resid + a (.) z + b: pure-Python sum from the popcount sign rule, then the cases that
+    # reduce to something known (x = 0 -> resid + b exactly; resid = 0 -> the plain forward).
+    rng = np.random.default_rng(300 + d)
+    x = rng.integers(-3, 4, size=(2, d)).astype(np.float64)
+    r = rng.integers(-5, 6, size=(2, d)).astype(np.float64)
+    a = rng.integers(1, 4, size=d).astype(np.float64)
+    b = rng.integers(-2, 3, size=d).astype(np.float64)
+    out = oracle.wht_affine_fwd_residual(x, a, b, r)
+    for t, j in itertools.product(range(2), range(d)):
+        acc = sum(int(x[t, i]) * (-1) ** bin(i & j).count("1") for i in range(d))
+        assert out[t, j] == pytest.approx(r[t, j] + a[j] * acc / math.sqrt(d) + b[j], abs=1e-13)
+    np.testing.assert_array_equal(oracle.wht_affine_fwd_residual(np.zeros((2, d)), a, b, r), r + b)
+    np.testing.assert_array_equal(oracle.wht_affine_fwd_residual(x, a, b, np.zeros((2, d))),
+                                  oracle.wht_affine_fwd(x, a, b))
+    # a dropped or doubled residual term is caught by the first loop; a sign error too
+    assert not np.allclose(oracle.wht_affine_fwd(x, a, b) - r, out)
+
+
 # ---------------------------------------------------------------- Fig. 2 butterfly
 
 def test_butterfly_pairs_of_figure():

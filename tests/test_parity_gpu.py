@@ -304,6 +304,83 @@ def test_tcgen05_kernels_on_many_rows(B):
     B.wht_affine_device_status()
 
 
+def test_back_to_back_calls_see_each_others_results(B):
+    # The kernels are launched so that a call may be scheduled while its predecessor in the stream
+    # still drains; each must nevertheless read what the predecessor wrote.  A chain of calls that
+    # feed one another must give the same bits with and without a synchronisation after every call.
+    B.wht_affine_set_variant(0)
+    for d, dtype, T in [(2048, wl.WHT_BF16_PF32, 148 * 8 * 3 + 5), (1024, wl.WHT_BF16, 148 * 16 * 2 + 3),
+                        (4096, wl.WHT_BF16, 64)]:
+        w = wl.Workload("chain", T, d, dtype, "normal", 500 + d, True, "")
+        x0 = wl.gen_full(w, "x").cuda()
+        dy = wl.gen_full(w, "dy").cuda()
+        a, b = (t.cuda() for t in wl.gen_params(w))
+
+        def chain(sync):
+            bufs = [x0.clone(), torch.empty_like(x0)]
+            da = torch.empty(d, dtype=torch.float32, device="cuda")
+            db = torch.empty_like(da)
+            dx = torch.empty_like(x0)
+            for k in range(6):
+                B.wht_affine_fwd(bufs[k % 2], a, b, bufs[(k + 1) % 2], T, d, dtype)
+                if sync:
+                    torch.cuda.synchronize()
+            # the backward reads the row tensor the last forward has just written, twice in a row
+            for _ in range(2):
+                B.wht_affine_bwd(dy, bufs[0], a, dx, da, db, T, d, dtype)
+                if sync:
+                    torch.cuda.synchronize()
+            torch.cuda.synchronize()
+            return bufs[0].clone(), dx, da, db
+
+        got, ref = chain(False), chain(True)
+        assert all(torch.equal(g, r) for g, r in zip(got, ref)), f"d={d}: chained calls differ"
+        assert torch.isfinite(got[0].float()).all()
+    B.wht_affine_device_status()
+
+
+# ------------------------------------------------------------------ fused residual forward
+
+@pytest.mark.parametrize("variant", VARIANTS)
+@pytest.mark.parametrize("d,dtype,T", [(256, wl.WHT_F32, 64), (64, wl.WHT_BF16, 1031), (1024, wl.WHT_BF16, 257),
+                                       (2048, wl.WHT_BF16_PF32, 300), (4096, wl.WHT_BF16, 37),
+                                       (8192, wl.WHT_BF16_PF32, 21), (16384, wl.WHT_F32, 5)])
+def test_fwd_residual(B, d, dtype, T, variant):
+    B.wht_affine_set_variant(variant)
+    w = wl.Workload("res", T, d, dtype, "normal", 600 + d, True, "")
+    x, r = wl.gen_full(w, "x"), wl.gen_full(w, "dy")  # the second seeded tensor serves as the residual stream
+    a, b = wl.gen_params(w)
+    xd, rd, ad, bd = x.cuda(), r.cuda(), a.cuda(), b.cuda()
+    y = B.forward(xd, ad, bd, resid=rd)
+    torch.cuda.synchronize()
+    ref = oracle.wht_affine_fwd_residual(to_f64(x), to_f64(a), to_f64(b), to_f64(r))
+    if dtype == wl.WHT_F32:
+        # the transform's error scales with ||x||, the final add with |resid|: one rounding of the sum
+        err = np.max(np.abs(to_f64(y.cpu()) - ref), axis=1)
+        assert np.all(err <= 1e-5 * (np.linalg.norm(to_f64(x), axis=1) + np.max(np.abs(to_f64(r)), axis=1)))
+    else:
+        assert_rows_bf16(to_f64(y.cpu()), ref, f"residual d={d} v{variant}")
+    # in place over the residual stream (out == resid), as a model would call it
+    r2 = rd.clone()
+    B.forward(xd, ad, bd, out=r2, resid=r2)
+    assert torch.equal(r2, y)
+
+
+def test_fwd_residual_many_rows(B):
+    # the tcgen05 kernels' residual path over several tiles per CTA with a ragged tail
+    B.wht_affine_set_variant(0)
+    for d, dtype, T in [(1024, wl.WHT_BF16, 148 * 16 * 3 + 5), (2048, wl.WHT_BF16_PF32, 148 * 8 * 2 + 3),
+                        (8192, wl.WHT_BF16_PF32, 148 * 2 * 2 + 1)]:
+        w = wl.Workload("res", T, d, dtype, "normal", 700 + d, True, "")
+        x, r = wl.gen_full(w, "x"), wl.gen_full(w, "dy")
+        a, b = wl.gen_params(w)
+        y = B.forward(x.cuda(), a.cuda(), b.cuda(), resid=r.cuda())
+        torch.cuda.synchronize()
+        ref = oracle.wht_affine_fwd_residual(to_f64(x), to_f64(a), to_f64(b), to_f64(r))
+        assert_rows_bf16(to_f64(y.cpu()), ref, f"residual many rows d={d}")
+    B.wht_affine_device_status()
+
+
 def test_copy_rows(B):
     src = torch.arange(3 * 1024, dtype=torch.float32, device="cuda").view(3, 1024)
     dst = torch.zeros_like(src)
