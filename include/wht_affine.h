@@ -157,8 +157,9 @@ size_t wht_affine_bwd_workspace_bytes(int64_t T, int32_t d, int dtype);
 
 /*
  * Kernel family used by the three compute calls (for A/B measurements):
- *   0 = automatic (default): for bf16 rows, the tcgen05 kernels when there are many
- *       rows and 1024 <= d <= 8192 (backward: <= 4096), else the mma.sync kernels
+ *   0 = automatic (default): for bf16 rows, the tcgen05 kernels when 1024 <= d <= 8192
+ *       and there is enough work for their 32 KiB tiles (forward: T*d >= 4 Mi elements,
+ *       8 Mi at d = 8192; backward: T*d >= 256 Ki), else the mma.sync kernels
  *       for 512 <= d <= 8192 (rows streamed through a shared-memory ring when there
  *       are many, loaded directly when there are few); butterfly otherwise;
  *   1 = butterfly (registers + warp shuffles + shared memory), every d and dtype;

@@ -441,6 +441,13 @@ bool umma_bwd_supported(int logd, int dtype) { return dtype != WHT_F32 && logd >
 
 bool mma_supported(int logd, int dtype) { return dtype != WHT_F32 && logd >= 9 && logd <= 13; }
 
+// The persistent tcgen05 kernels win once there are a few hundred 32 KiB tiles (measured
+// cross-over against the direct-load kernels, CUDA-graph replay, d = 1024 ... 8192).
+bool enough_work_for_tiles(int64_t T, int32_t d) {
+    const int64_t elems = T * static_cast<int64_t>(d);
+    return elems >= (d >= 8192 ? (8ll << 20) : (4ll << 20));
+}
+
 // Streaming pays once every row group has several rows to pipeline.
 bool enough_rows_to_stream(int64_t T, int sms) { return T >= static_cast<int64_t>(sms) * 32; }
 
@@ -451,7 +458,7 @@ int run_fwd(const FwdArgs& f, int64_t T, int32_t d, int dtype, cudaStream_t s, b
     if (rc != WHT_OK) return rc;
     const int logd = log2_of(d);
     if (umma_fwd_supported(logd, dtype) &&
-        (g_variant == 4 || (g_variant == 0 && !decode && enough_rows_to_stream(T, c.sms)))) {
+        (g_variant == 4 || (g_variant == 0 && enough_work_for_tiles(T, d)))) {
         return dtype == WHT_BF16 ? dispatch_umma_fwd<__nv_bfloat16>(logd, f, c) : dispatch_umma_fwd<float>(logd, f, c);
     }
     if (g_variant != 1 && mma_supported(logd, dtype)) {
@@ -472,7 +479,10 @@ int run_bwd(const BwdArgs& g, int64_t T, int32_t d, int dtype, cudaStream_t s) {
     int rc = current_device(&c.dev, &c.sms);
     if (rc != WHT_OK) return rc;
     const int logd = log2_of(d);
-    if (umma_bwd_supported(logd, dtype) && (g_variant == 4 || (g_variant == 0 && enough_rows_to_stream(T, c.sms)))) {
+    // the backward is the heavier kernel: the tcgen05 form was never slower than the others from a
+    // few hundred rows on
+    if (umma_bwd_supported(logd, dtype) &&
+        (g_variant == 4 || (g_variant == 0 && T * static_cast<int64_t>(d) >= (1ll << 18)))) {
         return dtype == WHT_BF16 ? dispatch_umma_bwd<__nv_bfloat16>(logd, g, c) : dispatch_umma_bwd<float>(logd, g, c);
     }
     if (g_variant != 1 && mma_supported(logd, dtype)) {
