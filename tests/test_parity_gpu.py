@@ -381,6 +381,39 @@ def test_fwd_residual_many_rows(B):
     B.wht_affine_device_status()
 
 
+def test_host_pipeline_matches_direct_calls(B):
+    # end-to-end helpers: pinned host -> device -> C ABI -> pinned host, rows moving in chunks on two
+    # copy streams; same results as the plain device-resident calls
+    B.wht_affine_set_variant(0)
+    w = wl.CONFIGS["training"].with_rows(5000)
+    x, dy = wl.gen_full(w, "x"), wl.gen_full(w, "dy")
+    a, b = wl.gen_params(w)
+    xd, dyd, ad, bd = x.cuda(), dy.cuda(), a.cuda(), b.cuda()
+    y_ref = B.forward(xd, ad, bd)
+    dx_ref, da_ref, db_ref = B.backward(dyd, xd, ad)
+    torch.cuda.synchronize()
+    st = {"x": torch.empty_like(xd), "a": torch.empty_like(ad), "b": torch.empty_like(bd), "y": torch.empty_like(xd),
+          "dy": torch.empty_like(xd), "dx": torch.empty_like(xd), "da": torch.empty_like(da_ref),
+          "db": torch.empty_like(db_ref)}
+    xp, dyp, ap, bp = x.pin_memory(), dy.pin_memory(), a.pin_memory(), b.pin_memory()
+    for pipe in (None, B.HostPipe(chunk_rows=1024)):
+        yp, dxp = torch.empty_like(xp).pin_memory(), torch.empty_like(xp).pin_memory()
+        dap, dbp = torch.empty(w.d).pin_memory(), torch.empty(w.d).pin_memory()
+        B.forward_host(xp, ap, bp, yp, st, pipe=pipe)
+        B.backward_host(dyp, xp, ap, dxp, dap, dbp, st, pipe=pipe, x_resident=True)
+        if pipe is not None:
+            pipe.join()
+        torch.cuda.synchronize()
+        if pipe is None:
+            assert torch.equal(yp, y_ref.cpu())
+        else:
+            # a 1024-row chunk is below the tcgen05 cross-over: another kernel family, another
+            # summation order, the same rounding target
+            assert_rows_bf16(to_f64(yp), to_f64(y_ref.cpu()), "chunked forward")
+        assert torch.equal(dxp, dx_ref.cpu())
+        assert torch.equal(dap, da_ref.cpu()) and torch.equal(dbp, db_ref.cpu())
+
+
 def test_copy_rows(B):
     src = torch.arange(3 * 1024, dtype=torch.float32, device="cuda").view(3, 1024)
     dst = torch.zeros_like(src)
