@@ -473,6 +473,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
     # ---- end to end: pinned host buffers in, results back to the host, every step
     e2e = None
     staging = {"x": x, "a": a, "b": b, "y": y, "dy": dy, "dx": dx, "da": da, "db": db}
+    e2e_launches = None
     xp, ap, bp = x_h.repeat(reps, 1).pin_memory(), a_h.pin_memory(), b_h.pin_memory()
     yp = torch.empty_like(xp).pin_memory()
     h2d = xp.numel() * xp.element_size() + 2 * ap.numel() * ap.element_size()

@@ -152,6 +152,16 @@ int wht_affine_bwd_noalloc(const void* dy, const void* x, const void* a,
                            void* dx, float* da, float* db,
                            int64_t T, int32_t d, int dtype, void* stream);
 
+/*
+ * Sums the parameter gradients of n backward calls (row chunks of one batch, or micro-batches
+ * whose gradients accumulate): da[j] = sum_p parts[p][0][j], db[j] = sum_p parts[p][1][j].
+ * da and db of Eq. 1's backward are sums over rows, so the gradients of disjoint row sets add.
+ *   parts [n x 2 x d] fp32 in: for each call its da (d values) then its db (d values);
+ *   da [d], db [d] fp32 out (overwritten; zeros when n == 0).
+ * The order of summation is fixed, so the result is bit-reproducible.  One small kernel.
+ */
+int wht_affine_reduce_grads(const float* parts, int32_t n, int32_t d, float* da, float* db, void* stream);
+
 /* Scratch bytes wht_affine_bwd_ws needs on the current device (0 on bad arguments). */
 size_t wht_affine_bwd_workspace_bytes(int64_t T, int32_t d, int dtype);
 

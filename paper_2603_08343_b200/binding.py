@@ -18,7 +18,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libwht_affine.so")
 
 EXPORTS = (
-    "wht_affine_fwd", "wht_affine_fwd_residual", "wht_affine_fwd_decode", "wht_affine_bwd", "wht_affine_bwd_ws", "wht_affine_bwd_noalloc",
+    "wht_affine_fwd", "wht_affine_fwd_residual", "wht_affine_fwd_decode", "wht_affine_bwd", "wht_affine_bwd_ws", "wht_affine_bwd_noalloc", "wht_affine_reduce_grads",
     "wht_affine_bwd_workspace_bytes", "wht_affine_set_variant", "wht_affine_get_variant",
     "wht_copy_rows", "wht_affine_device_status", "wht_affine_last_cuda_error", "wht_affine_status_string",
     "wht_affine_shutdown",
@@ -46,6 +46,7 @@ def _load() -> ctypes.CDLL:
     lib.wht_affine_bwd.argtypes = [vp, vp, vp, vp, vp, vp, i64, i32, ci, vp]
     lib.wht_affine_bwd_noalloc.argtypes = [vp, vp, vp, vp, vp, vp, i64, i32, ci, vp]
     lib.wht_affine_bwd_ws.argtypes = [vp, vp, vp, vp, vp, vp, i64, i32, ci, vp, sz, vp]
+    lib.wht_affine_reduce_grads.argtypes = [vp, i32, i32, vp, vp, vp]
     lib.wht_affine_bwd_workspace_bytes.argtypes = [i64, i32, ci]
     lib.wht_affine_bwd_workspace_bytes.restype = sz
     lib.wht_affine_set_variant.argtypes = [ci]
@@ -136,6 +137,13 @@ def wht_affine_bwd_noalloc(dy, x, a, dx, da, db, T: int, d: int, dtype: int, str
     _require_cuda(dy, x, a, dx, da, db)
     _check(_lib.wht_affine_bwd_noalloc(_ptr(dy), _ptr(x), _ptr(a), _ptr(dx), _ptr(da), _ptr(db), T, d, dtype,
                                        _stream(stream)), "wht_affine_bwd_noalloc")
+
+
+def wht_affine_reduce_grads(parts, n: int, d: int, da, db, stream=None) -> None:
+    """da, db = sums over the n (da_p | db_p) pairs stored contiguously in `parts` [n, 2, d] fp32."""
+    _require_cuda(parts, da, db)
+    _check(_lib.wht_affine_reduce_grads(_ptr(parts), n, d, _ptr(da), _ptr(db), _stream(stream)),
+           "wht_affine_reduce_grads")
 
 
 def wht_affine_bwd_workspace_bytes(T: int, d: int, dtype: int) -> int:
@@ -281,23 +289,35 @@ def backward_host(dy_host, x_host, a_host, dx_host, da_host, db_host, staging, s
         db_host.copy_(st["db"], non_blocking=True)
         return
     cur = torch.cuda.current_stream() if stream is None else stream
-    # dy comes in on the copy stream (sharing the link with the forward's y going out); the
-    # column sums need every row, so the kernel runs once, after the last chunk has arrived
-    with torch.cuda.stream(pipe.s_in):
-        if not x_resident:
+    # dy comes in chunk by chunk on the copy stream (sharing the link with the forward's y going
+    # out); each chunk is transformed as it lands and its dx leaves on the other copy stream, so the
+    # two directions of the link stay busy together.  da, db are sums over rows: every chunk writes
+    # its own pair, one small kernel adds them in a fixed order.
+    chunks = pipe.chunks(T)
+    parts = st.get("grad_parts")
+    if parts is None or parts.shape[0] < len(chunks):
+        parts = st["grad_parts"] = torch.empty(len(chunks), 2, d, dtype=torch.float32, device=st["x"].device)
+    if not x_resident:
+        with torch.cuda.stream(pipe.s_in):
             st["x"].copy_(x_host, non_blocking=True)
             st["a"].copy_(a_host, non_blocking=True)
-        for r0, r1 in pipe.chunks(T):
+    for i, (r0, r1) in enumerate(chunks):
+        with torch.cuda.stream(pipe.s_in):
             st["dy"][r0:r1].copy_(dy_host[r0:r1], non_blocking=True)
-        arrived = torch.cuda.Event()
-        arrived.record(pipe.s_in)
-    cur.wait_event(arrived)
-    wht_affine_bwd(st["dy"], st["x"], st["a"], st["dx"], st["da"], st["db"], T, d, code, cur)
+            arrived = torch.cuda.Event()
+            arrived.record(pipe.s_in)
+        cur.wait_event(arrived)
+        wht_affine_bwd(st["dy"][r0:r1], st["x"][r0:r1], st["a"], st["dx"][r0:r1], parts[i, 0], parts[i, 1],
+                       r1 - r0, d, code, cur)
+        done = torch.cuda.Event()
+        done.record(cur)
+        pipe.s_out.wait_event(done)
+        with torch.cuda.stream(pipe.s_out):
+            dx_host[r0:r1].copy_(st["dx"][r0:r1], non_blocking=True)
+    wht_affine_reduce_grads(parts, len(chunks), d, st["da"], st["db"], cur)
     done = torch.cuda.Event()
     done.record(cur)
     pipe.s_out.wait_event(done)
     with torch.cuda.stream(pipe.s_out):
-        for r0, r1 in pipe.chunks(T):
-            dx_host[r0:r1].copy_(st["dx"][r0:r1], non_blocking=True)
         da_host.copy_(st["da"], non_blocking=True)
         db_host.copy_(st["db"], non_blocking=True)

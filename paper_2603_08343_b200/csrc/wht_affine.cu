@@ -647,6 +647,24 @@ int wht_affine_bwd_noalloc(const void* dy, const void* x, const void* a, void* d
     return run_bwd(g, T, d, dtype, static_cast<cudaStream_t>(stream));
 }
 
+int wht_affine_reduce_grads(const float* parts, int32_t n, int32_t d, float* da, float* db, void* stream) {
+    if (!is_pow2(d) || d < 8 || d > 32768) return WHT_ERR_BAD_DIM;
+    if (n < 0) return WHT_ERR_BAD_T;
+    if (!da || !db || (n > 0 && !parts)) return WHT_ERR_NULL;
+    if (!aligned16(parts) || !aligned16(da) || !aligned16(db)) return WHT_ERR_MISALIGNED;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    // the second pass of the backward with a unit scale: partial p, slot 0 = da_p, slot 1 = db_p
+    if (d >= 32) {
+        launch_overlapped(dadb_finalize32_kernel, 2 * d / 32, 1024, 0, s, parts, static_cast<int>(n),
+                          static_cast<int>(d), 1.0f, da, db);
+    } else {
+        launch_overlapped(dadb_finalize_kernel, (2 * d + 255) / 256, 256, 0, s, parts, static_cast<int>(n),
+                          static_cast<int>(d), 1.0f, da, db);
+    }
+    WHT_CUDA_TRY(cudaGetLastError());
+    return WHT_OK;
+}
+
 int wht_affine_set_variant(int variant) {
     if (variant < 0 || variant > 4) return WHT_ERR_BAD_VARIANT;
     g_variant = variant;

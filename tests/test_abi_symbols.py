@@ -52,6 +52,8 @@ def test_argument_errors_need_no_gpu(lib):
     assert lib.wht_affine_bwd(p, off, p, p, p, p, 4, 256, 2, s) == -5
     assert lib.wht_affine_bwd_ws(p, p, p, p, p, p, 4, 100, 2, p, 64, s) == -2
     assert lib.wht_copy_rows(None, p, 4, 256, 1, s) == -1
+    assert lib.wht_affine_reduce_grads(p, 3, 100, p, p, s) == -2
+    assert lib.wht_affine_reduce_grads(None, 3, 256, p, p, s) == -1
     assert lib.wht_affine_set_variant(9) == -8 and lib.wht_affine_set_variant(5) == -8
     assert lib.wht_affine_set_variant(0) == 0 and lib.wht_affine_get_variant() == 0
     assert lib.wht_affine_fwd(p, p, p, p, 0, 256, 0, s) == 0           # T == 0: nothing to do

@@ -410,8 +410,40 @@ def test_host_pipeline_matches_direct_calls(B):
             # a 1024-row chunk is below the tcgen05 cross-over: another kernel family, another
             # summation order, the same rounding target
             assert_rows_bf16(to_f64(yp), to_f64(y_ref.cpu()), "chunked forward")
-        assert torch.equal(dxp, dx_ref.cpu())
-        assert torch.equal(dap, da_ref.cpu()) and torch.equal(dbp, db_ref.cpu())
+        if pipe is None:
+            assert torch.equal(dxp, dx_ref.cpu())
+            assert torch.equal(dap, da_ref.cpu()) and torch.equal(dbp, db_ref.cpu())
+        else:
+            assert_rows_bf16(to_f64(dxp), to_f64(dx_ref.cpu()), "chunked backward dx")
+            assert_grad_vec(to_f64(dap), to_f64(da_ref.cpu()), "chunked backward da")
+            assert_grad_vec(to_f64(dbp), to_f64(db_ref.cpu()), "chunked backward db")
+
+
+def test_reduce_grads(B):
+    # gradients of disjoint row sets add: chunked backward + wht_affine_reduce_grads == one backward
+    B.wht_affine_set_variant(0)
+    w = wl.CONFIGS["training"].with_rows(3001)
+    x, dy = wl.gen_full(w, "x").cuda(), wl.gen_full(w, "dy").cuda()
+    a = wl.gen_params(w)[0].cuda()
+    bounds = [0, 7, 1500, 1501, 3001]
+    parts = torch.full((len(bounds) - 1, 2, w.d), float("nan"), device="cuda")
+    dx = torch.empty_like(x)
+    for i in range(len(bounds) - 1):
+        r0, r1 = bounds[i], bounds[i + 1]
+        B.wht_affine_bwd(dy[r0:r1], x[r0:r1], a, dx[r0:r1], parts[i, 0], parts[i, 1], r1 - r0, w.d, w.dtype)
+    da, db = torch.empty(w.d, device="cuda"), torch.empty(w.d, device="cuda")
+    B.wht_affine_reduce_grads(parts, parts.shape[0], w.d, da, db)
+    da2, db2 = torch.empty_like(da), torch.empty_like(db)
+    B.wht_affine_reduce_grads(parts, parts.shape[0], w.d, da2, db2)
+    torch.cuda.synchronize()
+    assert torch.equal(da, da2) and torch.equal(db, db2)
+    _, da_ref, db_ref = oracle.wht_affine_bwd(to_f64(dy.cpu()), to_f64(x.cpu()), to_f64(a.cpu()))
+    assert_grad_vec(to_f64(da.cpu()), da_ref, "reduced da")
+    assert_grad_vec(to_f64(db.cpu()), db_ref, "reduced db")
+    np.testing.assert_allclose(to_f64(da.cpu()), parts[:, 0].double().sum(0).cpu().numpy(), rtol=1e-6, atol=1e-4)
+    B.wht_affine_reduce_grads(parts, 0, w.d, da, db)
+    torch.cuda.synchronize()
+    assert torch.count_nonzero(da) == 0 and torch.count_nonzero(db) == 0
 
 
 def test_copy_rows(B):
