@@ -316,6 +316,7 @@ umma_fwd_kernel(const __nv_bfloat16* x, const TP* __restrict__ a, const TP* __re
 
     if (warp == 0) {
         if (lane == 0) {
+            const uint64_t stream_policy = l2_policy_evict_first();
             long long it = 0;
             for (; it < my_tiles; ++it) {
                 const int s = static_cast<int>(it % STAGES);
@@ -326,7 +327,7 @@ umma_fwd_kernel(const __nv_bfloat16* x, const TP* __restrict__ a, const TP* __re
                 const long long rows = T - row0 < Geo::ROWS ? T - row0 : Geo::ROWS;
                 const uint32_t bytes = static_cast<uint32_t>(rows) * Geo::D * 2;
                 mbar_expect_tx(full + s, bytes);
-                bulk_load(ring + s * Geo::TILE_BYTES, x + row0 * Geo::D, bytes, full + s);
+                bulk_load_stream(ring + s * Geo::TILE_BYTES, x + row0 * Geo::D, bytes, full + s, stream_policy);
             }
             if (*abort_flag) {
                 // copies already issued still land in shared memory: wait for them before leaving
@@ -539,6 +540,7 @@ umma_bwd_kernel(const __nv_bfloat16* dy, const __nv_bfloat16* x, const TP* __res
 
     if (warp == 0) {
         if (lane == 0) {
+            const uint64_t stream_policy = l2_policy_evict_first();
             long long it = 0;
             for (; it < my_tiles; ++it) {
                 const int s = static_cast<int>(it % STAGES);
@@ -549,8 +551,9 @@ umma_bwd_kernel(const __nv_bfloat16* dy, const __nv_bfloat16* x, const TP* __res
                 const long long rows = T - row0 < Geo::ROWS ? T - row0 : Geo::ROWS;
                 const uint32_t bytes = static_cast<uint32_t>(rows) * Geo::D * 2;
                 mbar_expect_tx(full + s, 2 * bytes);
-                bulk_load(ring + s * L::STAGE_BYTES, x + row0 * Geo::D, bytes, full + s);
-                bulk_load(ring + s * L::STAGE_BYTES + Geo::TILE_BYTES, dy + row0 * Geo::D, bytes, full + s);
+                bulk_load_stream(ring + s * L::STAGE_BYTES, x + row0 * Geo::D, bytes, full + s, stream_policy);
+                bulk_load_stream(ring + s * L::STAGE_BYTES + Geo::TILE_BYTES, dy + row0 * Geo::D, bytes, full + s,
+                                 stream_policy);
             }
             if (*abort_flag) {
                 const long long lo = it > STAGES ? it - STAGES : 0;
