@@ -55,7 +55,7 @@ typedef enum {
     WHT_ERR_WORKSPACE = -6,   /* workspace missing, too small, or allocation failed  */
     WHT_ERR_CUDA = -7,        /* a CUDA runtime call failed; see wht_affine_last_cuda_error */
     WHT_ERR_BAD_VARIANT = -8, /* unknown kernel variant id                           */
-    WHT_ERR_DEVICE_WAIT = -9  /* a kernel's bounded wait for an async copy expired   */
+    WHT_ERR_DEVICE_WAIT = -9  /* a kernel's bounded wait (copy, product, hand-over) expired */
 } wht_status;
 
 /*
@@ -191,8 +191,9 @@ int wht_affine_get_variant(void);
 int wht_copy_rows(const void* src, void* dst, int64_t T, int32_t d, int dtype, void* stream);
 
 /*
- * The streamed kernels wait for their async copies with a bound; a wait that
- * expires does not hang or trap, it sets a flag on the device and the launch's
+ * The kernels that stream rows through shared memory (the tcgen05 family and the
+ * streamed mma.sync family) wait for their async copies, tensor-core products and
+ * hand-overs between warps with a bound; a wait that expires does not hang or trap, it sets a flag on the device and the launch's
  * results are invalid.  This call synchronises with the current device's work
  * (it copies the flag back), returns WHT_ERR_DEVICE_WAIT if the flag was set
  * since the last query and clears it, else WHT_OK.  Never expected in normal
