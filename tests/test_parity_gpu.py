@@ -446,6 +446,49 @@ def test_reduce_grads(B):
     assert torch.count_nonzero(da) == 0 and torch.count_nonzero(db) == 0
 
 
+def _round_to_bf16_bits(v64: np.ndarray) -> np.ndarray:
+    """fp64 -> nearest-even bfloat16 bit patterns, done on the integer representation of fp32."""
+    f32 = v64.astype(np.float32)
+    # where the fp32 rounding of the fp64 value is itself a tie-breaker it could double-round; such
+    # values have measure ~2^-29 and do not move the statistics below
+    u = f32.view(np.uint32).astype(np.uint64)
+    u = u + 0x7FFF + ((u >> 16) & 1)
+    return (u >> 16).astype(np.uint16)
+
+
+@pytest.mark.parametrize("variant", [0, 3, 4])
+def test_outputs_are_the_correctly_rounded_values_almost_everywhere(B, variant):
+    # fp32 accumulation then ONE rounding: the stored bf16 must be the nearest bf16 of the exact
+    # result except where the fp32 error (~1e-7 relative to the row scale) straddles a rounding
+    # boundary (bf16 spacing ~4e-3 relative): a fraction of order 1e-3.  An intermediate kept in
+    # bf16 anywhere on the path would push the fraction to tens of per cent.
+    B.wht_affine_set_variant(variant)
+    w = wl.CONFIGS["training"].with_rows(2400)
+    x, dy = wl.gen_full(w, "x"), wl.gen_full(w, "dy")
+    a, b = wl.gen_params(w)
+    xd, dyd, ad, bd = x.cuda(), dy.cuda(), a.cuda(), b.cuda()
+    y = B.forward(xd, ad, bd)
+    dx, _, _ = B.backward(dyd, xd, ad)
+    torch.cuda.synchronize()
+    ref_y = oracle.wht_affine_fwd(to_f64(x), to_f64(a), to_f64(b))
+    ref_dx, _, _ = oracle.wht_affine_bwd(to_f64(dy), to_f64(x), to_f64(a))
+    # (tensor, reference, name, allowed fraction not nearest, absolute slack relative to the row maximum:
+    #  fp32 accumulation for y; for dx the bf16 hi + lo operand split adds 2^-17 of the operand scale)
+    # the mma.sync family splits an fp32 operand into bf16 hi + lo in the forward too
+    y_slack = 4e-5 if variant == 3 else 2e-6
+    for got, ref, what, bound, slack in ((y, ref_y, "y", 5e-3, y_slack), (dx, ref_dx, "dx", 2e-2, 4e-5)):
+        bits = got.cpu().view(torch.int16).numpy().view(np.uint16)
+        want = _round_to_bf16_bits(ref)
+        frac = float(np.mean(bits != want))
+        assert frac <= bound, f"{what} v{variant}: {frac:.2e} of the outputs are not the nearest bf16"
+        # every output within half a bf16 step of the exact value plus the arithmetic's own error
+        half_step = np.exp2(np.floor(np.log2(np.maximum(np.abs(ref), 1e-300))) - 8)
+        err = np.abs(to_f64(got.cpu()) - ref)
+        allowed = half_step * (1 + 1e-6) + slack * np.max(np.abs(ref), axis=1, keepdims=True)
+        worst = float(np.max(err / allowed))
+        assert worst <= 1.0, f"{what} v{variant}: an output is {worst:.2f}x beyond half a bf16 step + {slack:g}*max|row|"
+
+
 def test_copy_rows(B):
     src = torch.arange(3 * 1024, dtype=torch.float32, device="cuda").view(3, 1024)
     dst = torch.zeros_like(src)
