@@ -153,6 +153,28 @@ int wht_affine_bwd_noalloc(const void* dy, const void* x, const void* a,
                            int64_t T, int32_t d, int dtype, void* stream);
 
 /*
+ * Grouped (block-diagonal) form for model widths that are not a power of two, d = groups * block
+ * with block a power of two in [8, 32768] (d = 768 = 3 * 256 and 1536 = 3 * 512 in the paper's model
+ * table):
+ *     y[t, g*block + j] = a[g*block + j] * ( x[t, g*block : (g+1)*block] H_block )[j] / sqrt(block)
+ *                         + b[g*block + j]
+ * i.e. Eq. 1 with H replaced by diag(H_block, ..., H_block); still orthonormal, mixes channels
+ * within a group only.  The paper does not say what its implementation does at those widths, so this
+ * is an explicit alternative of this library, not a claim about the paper's choice; groups = 1 is
+ * exactly wht_affine_fwd / wht_affine_bwd.  Same layouts, storage types, aliasing and error rules as
+ * the plain calls; rows are still contiguous [T x d].  One launch per group of the butterfly
+ * kernels on strided views (this form is not tuned).  The backward takes caller-owned scratch of at
+ * least wht_affine_bwd_grouped_workspace_bytes(T, d, block, dtype) bytes and never allocates.
+ */
+int wht_affine_fwd_grouped(const void* x, const void* a, const void* b, void* y,
+                           int64_t T, int32_t d, int32_t block, int dtype, void* stream);
+int wht_affine_bwd_grouped(const void* dy, const void* x, const void* a,
+                           void* dx, float* da, float* db,
+                           int64_t T, int32_t d, int32_t block, int dtype,
+                           void* workspace, size_t workspace_bytes, void* stream);
+size_t wht_affine_bwd_grouped_workspace_bytes(int64_t T, int32_t d, int32_t block, int dtype);
+
+/*
  * Sums the parameter gradients of n backward calls (row chunks of one batch, or micro-batches
  * whose gradients accumulate): da[j] = sum_p parts[p][0][j], db[j] = sum_p parts[p][1][j].
  * da and db of Eq. 1's backward are sums over rows, so the gradients of disjoint row sets add.

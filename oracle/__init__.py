@@ -9,6 +9,9 @@ from .wht_oracle import (  # noqa: F401
     wht_affine_fwd,
     wht_affine_fwd_residual,
     wht_affine_bwd,
+    grouped_hadamard,
+    wht_affine_fwd_grouped,
+    wht_affine_bwd_grouped,
     wht_normalised,
     da_db_columns,
     fwht_butterfly,

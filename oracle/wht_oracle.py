@@ -115,6 +115,35 @@ def wht_affine_bwd(dy: np.ndarray, x: np.ndarray, a: np.ndarray):
     return dx, da, db
 
 
+def grouped_hadamard(d: int, block: int) -> np.ndarray:
+    """Unnormalised block-diagonal matrix diag(H_block, ..., H_block) of order d = groups * block."""
+    _log2_exact(block)
+    if d < block or d % block:
+        raise ValueError(f"d={d} is not a multiple of block={block}")
+    return np.kron(np.eye(d // block), sylvester_hadamard(block))
+
+
+def wht_affine_fwd_grouped(x: np.ndarray, a: np.ndarray, b: np.ndarray, block: int) -> np.ndarray:
+    """Eq. 1 with H replaced by diag(H_block, ...)/sqrt(block): a reading offered for widths that are
+    not a power of two (the paper's d = 768, 1536), about which the paper itself is silent."""
+    x = np.asarray(x, dtype=np.float64)
+    G = grouped_hadamard(x.shape[-1], block)
+    z = (x @ G) / math.sqrt(float(block))
+    return np.asarray(a, dtype=np.float64)[None, :] * z + np.asarray(b, dtype=np.float64)[None, :]
+
+
+def wht_affine_bwd_grouped(dy: np.ndarray, x: np.ndarray, a: np.ndarray, block: int):
+    """Gradients of the grouped form (chain rule, G symmetric): (dx, da, db)."""
+    dy = np.asarray(dy, dtype=np.float64)
+    x = np.asarray(x, dtype=np.float64)
+    a = np.asarray(a, dtype=np.float64)
+    G = grouped_hadamard(x.shape[-1], block)
+    root = math.sqrt(float(block))
+    z = (x @ G) / root
+    dx = ((a[None, :] * dy) @ G.T) / root
+    return dx, np.sum(dy * z, axis=0), np.sum(dy, axis=0)
+
+
 def da_db_columns(dy: np.ndarray, x: np.ndarray, cols: np.ndarray):
     """da[j], db[j] for the listed columns j only, over ALL rows.
 

@@ -19,6 +19,7 @@ LIB_PATH = os.path.join(_HERE, "libwht_affine.so")
 
 EXPORTS = (
     "wht_affine_fwd", "wht_affine_fwd_residual", "wht_affine_fwd_decode", "wht_affine_bwd", "wht_affine_bwd_ws", "wht_affine_bwd_noalloc", "wht_affine_reduce_grads",
+    "wht_affine_fwd_grouped", "wht_affine_bwd_grouped", "wht_affine_bwd_grouped_workspace_bytes",
     "wht_affine_bwd_workspace_bytes", "wht_affine_set_variant", "wht_affine_get_variant",
     "wht_copy_rows", "wht_affine_device_status", "wht_affine_last_cuda_error", "wht_affine_status_string",
     "wht_affine_shutdown",
@@ -47,6 +48,10 @@ def _load() -> ctypes.CDLL:
     lib.wht_affine_bwd_noalloc.argtypes = [vp, vp, vp, vp, vp, vp, i64, i32, ci, vp]
     lib.wht_affine_bwd_ws.argtypes = [vp, vp, vp, vp, vp, vp, i64, i32, ci, vp, sz, vp]
     lib.wht_affine_reduce_grads.argtypes = [vp, i32, i32, vp, vp, vp]
+    lib.wht_affine_fwd_grouped.argtypes = [vp, vp, vp, vp, i64, i32, i32, ci, vp]
+    lib.wht_affine_bwd_grouped.argtypes = [vp, vp, vp, vp, vp, vp, i64, i32, i32, ci, vp, sz, vp]
+    lib.wht_affine_bwd_grouped_workspace_bytes.argtypes = [i64, i32, i32, ci]
+    lib.wht_affine_bwd_grouped_workspace_bytes.restype = sz
     lib.wht_affine_bwd_workspace_bytes.argtypes = [i64, i32, ci]
     lib.wht_affine_bwd_workspace_bytes.restype = sz
     lib.wht_affine_set_variant.argtypes = [ci]
@@ -144,6 +149,25 @@ def wht_affine_reduce_grads(parts, n: int, d: int, da, db, stream=None) -> None:
     _require_cuda(parts, da, db)
     _check(_lib.wht_affine_reduce_grads(_ptr(parts), n, d, _ptr(da), _ptr(db), _stream(stream)),
            "wht_affine_reduce_grads")
+
+
+def wht_affine_fwd_grouped(x, a, b, y, T: int, d: int, block: int, dtype: int, stream=None) -> None:
+    """Block-diagonal form: every group of `block` channels is transformed on its own (d = groups*block)."""
+    _require_cuda(x, a, b, y)
+    _check(_lib.wht_affine_fwd_grouped(_ptr(x), _ptr(a), _ptr(b), _ptr(y), T, d, block, dtype, _stream(stream)),
+           "wht_affine_fwd_grouped")
+
+
+def wht_affine_bwd_grouped(dy, x, a, dx, da, db, T: int, d: int, block: int, dtype: int, workspace,
+                           stream=None) -> None:
+    _require_cuda(dy, x, a, dx, da, db, workspace)
+    nbytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(_lib.wht_affine_bwd_grouped(_ptr(dy), _ptr(x), _ptr(a), _ptr(dx), _ptr(da), _ptr(db), T, d, block, dtype,
+                                       _ptr(workspace), nbytes, _stream(stream)), "wht_affine_bwd_grouped")
+
+
+def wht_affine_bwd_grouped_workspace_bytes(T: int, d: int, block: int, dtype: int) -> int:
+    return int(_lib.wht_affine_bwd_grouped_workspace_bytes(T, d, block, dtype))
 
 
 def wht_affine_bwd_workspace_bytes(T: int, d: int, dtype: int) -> int:

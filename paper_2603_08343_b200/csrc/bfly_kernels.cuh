@@ -159,7 +159,7 @@ __device__ __forceinline__ void store8_stream(__nv_bfloat16* p, const float (&v)
 template <int LOGD, typename TIO, typename TP>
 __global__ void __launch_bounds__(BflyGeo<LOGD>::THREADS)
 bfly_fwd_kernel(const TIO* x, const TP* __restrict__ a, const TP* __restrict__ b, const TIO* resid, TIO* y,
-                long long T, float inv_sqrt_d) {
+                long long T, long long ld, float inv_sqrt_d) {  // ld: elements between consecutive rows (>= D)
     using Geo = BflyGeo<LOGD>;
     extern __shared__ __align__(16) float smem[];
     const int rg = threadIdx.x / Geo::G;  // row group inside the CTA
@@ -183,7 +183,7 @@ bfly_fwd_kernel(const TIO* x, const TP* __restrict__ a, const TP* __restrict__ b
 #pragma unroll
         for (int c = 0; c < Geo::C; ++c) {
             if (valid) {
-                load8_stream(x + row * Geo::D + (c * Geo::G + t) * 8, v[c]);
+                load8_stream(x + row * ld + (c * Geo::G + t) * 8, v[c]);
             } else {
 #pragma unroll
                 for (int e = 0; e < 8; ++e) v[c][e] = 0.0f;
@@ -197,11 +197,11 @@ bfly_fwd_kernel(const TIO* x, const TP* __restrict__ a, const TP* __restrict__ b
                 for (int e = 0; e < 8; ++e) v[c][e] = fmaf(v[c][e], as[c][e], bs[c][e]);
                 if (resid != nullptr) {  // fused residual: summed in fp32, rounded once at the store
                     float r[8];
-                    load8_stream(resid + row * Geo::D + (c * Geo::G + t) * 8, r);
+                    load8_stream(resid + row * ld + (c * Geo::G + t) * 8, r);
 #pragma unroll
                     for (int e = 0; e < 8; ++e) v[c][e] += r[e];
                 }
-                store8_stream(y + row * Geo::D + (c * Geo::G + t) * 8, v[c]);
+                store8_stream(y + row * ld + (c * Geo::G + t) * 8, v[c]);
             }
         }
     }
@@ -213,7 +213,7 @@ bfly_fwd_kernel(const TIO* x, const TP* __restrict__ a, const TP* __restrict__ b
 template <int LOGD, typename TIO, typename TP>
 __global__ void __launch_bounds__(BflyGeo<LOGD>::THREADS)
 bfly_bwd_kernel(const TIO* dy, const TIO* x, const TP* __restrict__ a, TIO* dx,
-                float* __restrict__ partials, long long T, float inv_sqrt_d) {
+                float* __restrict__ partials, long long T, long long ld, float inv_sqrt_d) {
     using Geo = BflyGeo<LOGD>;
     extern __shared__ __align__(16) float smem[];
     const int rg = threadIdx.x / Geo::G;
@@ -235,8 +235,8 @@ bfly_bwd_kernel(const TIO* dy, const TIO* x, const TP* __restrict__ a, TIO* dx,
 #pragma unroll
         for (int c = 0; c < Geo::C; ++c) {
             if (valid) {
-                load8_stream(x + row * Geo::D + (c * Geo::G + t) * 8, v[c]);
-                load8_stream(dy + row * Geo::D + (c * Geo::G + t) * 8, w[c]);
+                load8_stream(x + row * ld + (c * Geo::G + t) * 8, v[c]);
+                load8_stream(dy + row * ld + (c * Geo::G + t) * 8, w[c]);
             } else {
 #pragma unroll
                 for (int e = 0; e < 8; ++e) { v[c][e] = 0.0f; w[c][e] = 0.0f; }
@@ -261,7 +261,7 @@ bfly_bwd_kernel(const TIO* dy, const TIO* x, const TP* __restrict__ a, TIO* dx,
             for (int c = 0; c < Geo::C; ++c) {
 #pragma unroll
                 for (int e = 0; e < 8; ++e) v[c][e] *= inv_sqrt_d;
-                store8_stream(dx + row * Geo::D + (c * Geo::G + t) * 8, v[c]);
+                store8_stream(dx + row * ld + (c * Geo::G + t) * 8, v[c]);
             }
         }
     }

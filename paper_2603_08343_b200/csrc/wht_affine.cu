@@ -130,6 +130,7 @@ struct Ctx {
     int dev;
     int sms;
     cudaStream_t stream;
+    int64_t ld = 0;  // elements between consecutive rows; 0 = contiguous rows (ld == d)
 };
 
 struct FwdArgs {
@@ -194,7 +195,8 @@ int launch_bfly_fwd(const FwdArgs& f, const Ctx& c) {
     const int grid = capped_grid(ceil_div(c.T, Geo::R), c.sms, per_sm);
     kernel<<<grid, Geo::THREADS, Geo::SMEM_FWD, c.stream>>>(
         static_cast<const TIO*>(f.x), static_cast<const TP*>(f.a), static_cast<const TP*>(f.b),
-        static_cast<const TIO*>(f.resid), static_cast<TIO*>(f.y), static_cast<long long>(c.T), inv_sqrt(Geo::D));
+        static_cast<const TIO*>(f.resid), static_cast<TIO*>(f.y), static_cast<long long>(c.T),
+        static_cast<long long>(c.ld ? c.ld : Geo::D), inv_sqrt(Geo::D));
     WHT_CUDA_TRY(cudaGetLastError());
     return WHT_OK;
 }
@@ -211,7 +213,7 @@ int launch_bfly_bwd(const BwdArgs& g, const Ctx& c) {
         kernel<<<n, Geo::THREADS, Geo::SMEM_BWD, c.stream>>>(
             static_cast<const TIO*>(g.dy), static_cast<const TIO*>(g.x), static_cast<const TP*>(g.a),
             static_cast<TIO*>(g.dx), static_cast<float*>(g.ws), static_cast<long long>(c.T),
-            inv_sqrt(Geo::D));
+            static_cast<long long>(c.ld ? c.ld : Geo::D), inv_sqrt(Geo::D));
     });
 }
 
@@ -645,6 +647,95 @@ int wht_affine_bwd_noalloc(const void* dy, const void* x, const void* a, void* d
     if (rc != WHT_OK) return rc;
     BwdArgs g{dy, x, a, dx, da, db, ws, WHT_NOALLOC_SCRATCH_BYTES, false, &need};
     return run_bwd(g, T, d, dtype, static_cast<cudaStream_t>(stream));
+}
+
+// ---- grouped (block-diagonal) form: d = groups * block, every block transformed on its own.
+// Runs the butterfly family on strided views, one launch per group.
+namespace {
+int check_grouped(int64_t T, int32_t d, int32_t block, int dtype) {
+    if (dtype != WHT_F32 && dtype != WHT_BF16 && dtype != WHT_BF16_PF32) return WHT_ERR_BAD_DTYPE;
+    if (!is_pow2(block) || block < 8 || block > 32768 || d < block || d % block != 0) return WHT_ERR_BAD_DIM;
+    if (T < 0) return WHT_ERR_BAD_T;
+    return WHT_OK;
+}
+size_t io_bytes(int dtype) { return dtype == WHT_F32 ? 4 : 2; }
+size_t param_bytes(int dtype) { return dtype == WHT_BF16 ? 2 : 4; }
+const char* at_bytes(const void* p, size_t bytes) { return static_cast<const char*>(p) + bytes; }
+char* at_bytes_mut(void* p, size_t bytes) { return static_cast<char*>(p) + bytes; }
+}  // namespace
+
+int wht_affine_fwd_grouped(const void* x, const void* a, const void* b, void* y, int64_t T, int32_t d,
+                           int32_t block, int dtype, void* stream) {
+    int rc = check_grouped(T, d, block, dtype);
+    if (rc != WHT_OK) return rc;
+    if (!a || !b) return WHT_ERR_NULL;
+    if (T > 0 && (!x || !y)) return WHT_ERR_NULL;
+    if (!aligned16(x) || !aligned16(a) || !aligned16(b) || !aligned16(y)) return WHT_ERR_MISALIGNED;
+    if (T == 0) return WHT_OK;
+    Ctx c{T, 0, 0, static_cast<cudaStream_t>(stream)};
+    c.ld = d;
+    rc = current_device(&c.dev, &c.sms);
+    if (rc != WHT_OK) return rc;
+    const int logb = log2_of(block);
+    for (int32_t g = 0; g < d / block; ++g) {
+        const size_t io = static_cast<size_t>(g) * block * io_bytes(dtype);
+        const size_t pp = static_cast<size_t>(g) * block * param_bytes(dtype);
+        FwdArgs f{at_bytes(x, io), at_bytes(a, pp), at_bytes(b, pp), at_bytes_mut(y, io)};
+        switch (dtype) {
+            case WHT_F32: rc = dispatch_bfly_fwd<float, float>(logb, f, c); break;
+            case WHT_BF16: rc = dispatch_bfly_fwd<__nv_bfloat16, __nv_bfloat16>(logb, f, c); break;
+            default: rc = dispatch_bfly_fwd<__nv_bfloat16, float>(logb, f, c); break;
+        }
+        if (rc != WHT_OK) return rc;
+    }
+    return WHT_OK;
+}
+
+int wht_affine_bwd_grouped(const void* dy, const void* x, const void* a, void* dx, float* da, float* db, int64_t T,
+                           int32_t d, int32_t block, int dtype, void* workspace, size_t workspace_bytes,
+                           void* stream) {
+    int rc = check_grouped(T, d, block, dtype);
+    if (rc != WHT_OK) return rc;
+    if (!a || !da || !db) return WHT_ERR_NULL;
+    if (T > 0 && (!dy || !x || !dx)) return WHT_ERR_NULL;
+    if (!aligned16(dy) || !aligned16(x) || !aligned16(a) || !aligned16(dx) || !aligned16(da) || !aligned16(db) ||
+        !aligned16(workspace))
+        return WHT_ERR_MISALIGNED;
+    Ctx c{T, 0, 0, static_cast<cudaStream_t>(stream)};
+    c.ld = d;
+    rc = current_device(&c.dev, &c.sms);
+    if (rc != WHT_OK) return rc;
+    const int logb = log2_of(block);
+    for (int32_t g = 0; g < d / block; ++g) {
+        const size_t io = static_cast<size_t>(g) * block * io_bytes(dtype);
+        const size_t pp = static_cast<size_t>(g) * block * param_bytes(dtype);
+        size_t need = 0;
+        // the groups run one after another on the stream and share the scratch
+        BwdArgs q{at_bytes(dy, io), at_bytes(x, io), at_bytes(a, pp), at_bytes_mut(dx, io), da + static_cast<size_t>(g) * block,
+                  db + static_cast<size_t>(g) * block, workspace, workspace_bytes, false, &need};
+        switch (dtype) {
+            case WHT_F32: rc = dispatch_bfly_bwd<float, float>(logb, q, c); break;
+            case WHT_BF16: rc = dispatch_bfly_bwd<__nv_bfloat16, __nv_bfloat16>(logb, q, c); break;
+            default: rc = dispatch_bfly_bwd<__nv_bfloat16, float>(logb, q, c); break;
+        }
+        if (rc != WHT_OK) return rc;
+    }
+    return WHT_OK;
+}
+
+size_t wht_affine_bwd_grouped_workspace_bytes(int64_t T, int32_t d, int32_t block, int dtype) {
+    if (check_grouped(T, d, block, dtype) != WHT_OK) return 0;
+    Ctx c{T, 0, 0, nullptr};
+    if (current_device(&c.dev, &c.sms) != WHT_OK) return 0;
+    size_t need = 0;
+    BwdArgs q{nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, 0, true, &need};
+    int rc;
+    switch (dtype) {
+        case WHT_F32: rc = dispatch_bfly_bwd<float, float>(log2_of(block), q, c); break;
+        case WHT_BF16: rc = dispatch_bfly_bwd<__nv_bfloat16, __nv_bfloat16>(log2_of(block), q, c); break;
+        default: rc = dispatch_bfly_bwd<__nv_bfloat16, float>(log2_of(block), q, c); break;
+    }
+    return rc == WHT_OK ? need : 0;
 }
 
 int wht_affine_reduce_grads(const float* parts, int32_t n, int32_t d, float* da, float* db, void* stream) {

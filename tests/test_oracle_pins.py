@@ -143,6 +143,44 @@ def test_residual_form_brute_force_and_special_cases(d):
     assert not np.allclose(oracle.wht_affine_fwd(x, a, b) - r, out)
 
 
+# ---------------------------------------------------------------- grouped (block-diagonal) form
+
+@pytest.mark.parametrize("d,block", [(24, 8), (768, 256), (48, 16), (64, 64)])
+def test_grouped_form(d, block):
+    rng = np.random.default_rng(d + block)
+    T, G = 4, d // block
+    x = rng.standard_normal((T, d))
+    dy = rng.standard_normal((T, d))
+    a = rng.uniform(0.5, 1.5, d)
+    b = rng.normal(0, 0.1, d)
+    y = oracle.wht_affine_fwd_grouped(x, a, b, block)
+    # each group is the plain transform of its own slice (and of nothing else)
+    for g in range(G):
+        sl = slice(g * block, (g + 1) * block)
+        np.testing.assert_allclose(y[:, sl], oracle.wht_affine_fwd(x[:, sl], a[sl], b[sl]), rtol=0, atol=1e-12)
+    # orthonormal: norms preserved, and the matrix squares to block * I in integers
+    M = oracle.grouped_hadamard(d, block).astype(np.int64)
+    np.testing.assert_array_equal(M @ M.T, block * np.eye(d, dtype=np.int64))
+    z = oracle.wht_affine_fwd_grouped(x, np.ones(d), np.zeros(d), block)
+    np.testing.assert_allclose(np.linalg.norm(z, axis=1), np.linalg.norm(x, axis=1), rtol=1e-13)
+    # gradients: adjoint identity and finite differences on a few entries
+    dx, da, db = oracle.wht_affine_bwd_grouped(dy, x, a, block)
+    assert np.sum(dy * (y - b)) == pytest.approx(np.sum(dx * x), rel=1e-12)
+    h = 1e-3
+    for j in (0, block - 1, d - 1):
+        ap, am = a.copy(), a.copy()
+        ap[j] += h
+        am[j] -= h
+        fd = (np.sum(dy * oracle.wht_affine_fwd_grouped(x, ap, b, block)) -
+              np.sum(dy * oracle.wht_affine_fwd_grouped(x, am, b, block))) / (2 * h)
+        assert fd == pytest.approx(da[j], rel=1e-8, abs=1e-8)
+    np.testing.assert_allclose(db, dy.sum(axis=0), rtol=0, atol=1e-13)
+    if G == 1:
+        np.testing.assert_array_equal(y, oracle.wht_affine_fwd(x, a, b))
+    with pytest.raises(ValueError):
+        oracle.grouped_hadamard(d + 1, block)
+
+
 # ---------------------------------------------------------------- Fig. 2 butterfly
 
 def test_butterfly_pairs_of_figure():

@@ -489,6 +489,51 @@ def test_outputs_are_the_correctly_rounded_values_almost_everywhere(B, variant):
         assert worst <= 1.0, f"{what} v{variant}: an output is {worst:.2f}x beyond half a bf16 step + {slack:g}*max|row|"
 
 
+# ------------------------------------------------------------------ grouped (block-diagonal) form
+
+@pytest.mark.parametrize("d,block,dtype,T", [(768, 256, wl.WHT_F32, 70), (768, 256, wl.WHT_BF16, 300),
+                                             (1536, 512, wl.WHT_BF16_PF32, 129), (3072, 1024, wl.WHT_BF16, 33),
+                                             (96, 32, wl.WHT_F32, 1000), (1024, 1024, wl.WHT_BF16, 40)])
+def test_grouped_form(B, d, block, dtype, T):
+    B.wht_affine_set_variant(0)
+    w = wl.Workload("grp", T, block, dtype, "normal", 800 + d, True, "")  # generators take a power of two:
+    G = d // block                                                          # draw G blocks side by side
+    x = torch.cat([wl.gen_full(wl.Workload("grp", T, block, dtype, "normal", 800 + d + g, True, ""), "x")
+                   for g in range(G)], dim=1).contiguous()
+    dy = torch.cat([wl.gen_full(wl.Workload("grp", T, block, dtype, "normal", 800 + d + g, True, ""), "dy")
+                    for g in range(G)], dim=1).contiguous()
+    ab = [wl.gen_params(wl.Workload("grp", T, block, dtype, "normal", 800 + d + g, True, "")) for g in range(G)]
+    a = torch.cat([p[0] for p in ab]).contiguous()
+    b = torch.cat([p[1] for p in ab]).contiguous()
+    xd, dyd, ad, bd = x.cuda(), dy.cuda(), a.cuda(), b.cuda()
+    y = torch.empty_like(xd)
+    B.wht_affine_fwd_grouped(xd, ad, bd, y, T, d, block, dtype)
+    need = B.wht_affine_bwd_grouped_workspace_bytes(T, d, block, dtype)
+    ws = torch.empty(max(need, 16), dtype=torch.uint8, device="cuda")
+    dx = torch.empty_like(xd)
+    da = torch.empty(d, dtype=torch.float32, device="cuda")
+    db = torch.empty_like(da)
+    B.wht_affine_bwd_grouped(dyd, xd, ad, dx, da, db, T, d, block, dtype, ws)
+    torch.cuda.synchronize()
+    ref_y = oracle.wht_affine_fwd_grouped(to_f64(x), to_f64(a), to_f64(b), block)
+    ref_dx, ref_da, ref_db = oracle.wht_affine_bwd_grouped(to_f64(dy), to_f64(x), to_f64(a), block)
+    if dtype == wl.WHT_F32:
+        assert_rows_fp32(to_f64(y.cpu()), ref_y, to_f64(x), "grouped y")
+        assert_rows_fp32(to_f64(dx.cpu()), ref_dx, to_f64(a)[None, :] * to_f64(dy), "grouped dx")
+    else:
+        assert_rows_bf16(to_f64(y.cpu()), ref_y, "grouped y")
+        assert_rows_bf16(to_f64(dx.cpu()), ref_dx, "grouped dx")
+    assert_grad_vec(to_f64(da.cpu()), ref_da, "grouped da")
+    assert_grad_vec(to_f64(db.cpu()), ref_db, "grouped db")
+    if G == 1:  # one group is the plain call (butterfly family)
+        B.wht_affine_set_variant(1)
+        assert torch.equal(y, B.forward(xd, ad, bd))
+        B.wht_affine_set_variant(0)
+    with pytest.raises(B.WhtError) as err:
+        B.wht_affine_fwd_grouped(xd, ad, bd, y, T, d, 48, dtype)
+    assert err.value.status == -2
+
+
 def test_copy_rows(B):
     src = torch.arange(3 * 1024, dtype=torch.float32, device="cuda").view(3, 1024)
     dst = torch.zeros_like(src)
