@@ -1,0 +1,77 @@
+"""Seeded random sweep of shapes, storage types and kernel families against the oracle.
+
+Row counts are drawn both at random and right around multiples of the tcgen05 kernels' tile
+height (one row short, exact, one over, half a tile), where ragged-tile handling lives.
+"""
+import random
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from helpers import to_f64
+from paper_2603_08343_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2603_08343_b200 import build
+    build.build()
+    from paper_2603_08343_b200 import binding
+    yield binding
+    binding.wht_affine_set_variant(0)
+    binding.wht_affine_device_status()
+
+
+def _ratio_rows(got, ref, dtype, fp32_scale):
+    err = np.max(np.abs(got - ref), axis=1)
+    bound = 1e-5 * fp32_scale if dtype == wl.WHT_F32 else 1e-2 * np.max(np.abs(ref), axis=1)
+    return float(np.max(err / np.maximum(bound, 1e-300)))
+
+
+def _cases(seed, count):
+    rng = random.Random(seed)
+    out = []
+    for case in range(count):
+        logd = rng.choice([3, 5, 8, 9, 10, 10, 11, 11, 12, 12, 13, 13, 14])
+        d = 1 << logd
+        dtype = rng.choice([wl.WHT_F32, wl.WHT_BF16, wl.WHT_BF16_PF32, wl.WHT_BF16_PF32, wl.WHT_BF16])
+        variant = rng.choice([0, 0, 1, 2, 3, 4, 4])
+        max_rows = max(1, min(6000, (1 << 25) // (d * d // 64 + 1)))  # keeps the dense oracle to a fraction of a second
+        if 10 <= logd <= 13 and rng.random() < 0.5:
+            tile = 128 // (8 * (d // 1024))
+            k = rng.randint(1, max(1, min(max_rows // tile, 148 * 3)))
+            T = max(1, k * tile + rng.choice([-1, 0, 1, tile // 2]))
+        else:
+            T = rng.randint(1, max_rows)
+        out.append((case, d, min(T, max_rows), dtype, variant, rng.choice(["normal", "student_t3"])))
+    return out
+
+
+@pytest.mark.parametrize("seed", [11, 12])
+def test_random_shapes_match_the_oracle(B, seed):
+    for case, d, T, dtype, variant, dist in _cases(seed, 24):
+        w = wl.Workload("fuzz", T, d, dtype, dist, 5000 + 100 * seed + case, True, "")
+        x, dy = wl.gen_full(w, "x"), wl.gen_full(w, "dy")
+        a, b = wl.gen_params(w)
+        B.wht_affine_set_variant(variant)
+        xd, dyd, ad, bd = x.cuda(), dy.cuda(), a.cuda(), b.cuda()
+        y = B.forward(xd, ad, bd)
+        yr = B.forward(xd, ad, bd, resid=dyd)
+        dx, da, db = B.backward(dyd, xd, ad)
+        torch.cuda.synchronize()
+        x64, dy64, a64, b64 = to_f64(x), to_f64(dy), to_f64(a), to_f64(b)
+        ref_y = oracle.wht_affine_fwd(x64, a64, b64)
+        ref_dx, ref_da, ref_db = oracle.wht_affine_bwd(dy64, x64, a64)
+        xn = np.linalg.norm(x64, axis=1)
+        what = f"d={d} T={T} dtype={dtype} variant={variant} {dist}"
+        assert _ratio_rows(to_f64(y.cpu()), ref_y, dtype, xn) <= 1.0, what + ": y"
+        assert _ratio_rows(to_f64(yr.cpu()), ref_y + dy64, dtype, xn + np.max(np.abs(dy64), axis=1)) <= 1.0, \
+            what + ": y with residual"
+        assert _ratio_rows(to_f64(dx.cpu()), ref_dx, dtype, np.linalg.norm(a64[None, :] * dy64, axis=1)) <= 1.0, \
+            what + ": dx"
+        assert np.max(np.abs(to_f64(da.cpu()) - ref_da)) <= 1e-4 * np.max(np.abs(ref_da)), what + ": da"
+        assert np.max(np.abs(to_f64(db.cpu()) - ref_db)) <= 1e-4 * np.max(np.abs(ref_db)), what + ": db"
