@@ -467,13 +467,14 @@ umma_bwd_kernel(const __nv_bfloat16* dy, const __nv_bfloat16* x, const TP* __res
                 float* __restrict__ partials, long long T, float inv_sqrt_d) {
     using Geo = UmmaGeo<LOGD, NCOL>;
     using L = UmmaBwdSmem<LOGD, NCOL, STAGES>;
-    // How the two groups of four epilogue warps share a tile.  Up to 32 values per row and
-    // thread (d <= 4096) each group takes half of the rows.  Beyond that the per-thread
-    // accumulators for all channels would not fit in registers, so each group takes ALL rows
-    // but only the channels whose top index bit equals its group number: the stage on that
+    // How the two groups of four epilogue warps share a tile.  Up to 16 values per row and
+    // thread (d <= 2048) each group takes half of the rows.  Beyond that the per-thread state
+    // for all channels (da, db, a: three values per channel, next to a tile's worth of
+    // accumulator columns) would not fit in registers, so each group takes ALL rows but
+    // only the channels whose top index bit equals its group number: the stage on that
     // bit is applied first, straight on the accumulator columns (each thread reads both
     // halves from TMEM and keeps lo + hi or lo - hi), and for dx last, in the same way.
-    constexpr bool SPLIT = Geo::R > 32;
+    constexpr bool SPLIT = Geo::R > 16;
     constexpr int RE = SPLIT ? Geo::R / 2 : Geo::R;      // values per row a thread works on
     constexpr int PE = RE / 8;                           // pieces per row a thread works on
     constexpr int NROW = SPLIT ? Geo::ROWS : Geo::RPW;   // rows per tile a thread works on

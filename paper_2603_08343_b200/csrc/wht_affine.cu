@@ -432,7 +432,7 @@ int dispatch_umma_bwd(int logd, const BwdArgs& g, const Ctx& c) {
     switch (logd) {
         case 10: return launch_umma_bwd<10, 128, 3, TP>(g, c);
         case 11: return launch_umma_bwd<11, 128, 3, TP>(g, c);
-        case 12: return launch_umma_bwd<12, 64, 5, TP>(g, c);
+        case 12: return launch_umma_bwd<12, 128, 3, TP>(g, c);
         case 13: return launch_umma_bwd<13, 128, 3, TP>(g, c);
     }
     return WHT_ERR_BAD_DIM;
