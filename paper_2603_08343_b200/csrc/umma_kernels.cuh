@@ -227,12 +227,17 @@ __device__ __forceinline__ void thread_stages(float (&v)[R]) {
 }
 
 // ---- forward ---------------------------------------------------------------------------
-template <int LOGD, int NCOL, int STAGES, typename TP>
+template <int LOGD, int NCOL, int STAGES, typename TP, bool RES = false>
 struct UmmaFwdSmem {
     using Geo = UmmaGeo<LOGD, NCOL>;
     static constexpr int ACC = 512 / NCOL > 4 ? 4 : 512 / NCOL;          // accumulator buffers in TMEM
     static constexpr int TMEM_COLS = ACC * NCOL <= 256 ? 256 : 512;
-    static constexpr bool PARAMS_IN_SMEM = Geo::R > 32;
+    // a and b live in registers while a row's share of them is small.  At d = 8192 the plain
+    // forward splits the channels between its two warp groups instead (SPLIT); with a residual,
+    // whose chunks need registers too, a and b are staged in shared memory as fp32 from d = 4096 on
+    // (measured: the split form is slower there).
+    static constexpr bool SPLIT = Geo::R > 32 && !RES;
+    static constexpr bool PARAMS_IN_SMEM = RES && Geo::R >= 32;
     static constexpr int OFF_H = 0;
     static constexpr int OFF_RING = Geo::H_BYTES;
     static constexpr int OFF_PARAMS = OFF_RING + STAGES * Geo::TILE_BYTES;
@@ -269,7 +274,7 @@ __global__ void __launch_bounds__(UmmaGeo<LOGD, NCOL>::THREADS, 1)
 umma_fwd_kernel(const __nv_bfloat16* x, const TP* __restrict__ a, const TP* __restrict__ b,
                 const __nv_bfloat16* resid, __nv_bfloat16* y, long long T, float inv_sqrt_d) {
     using Geo = UmmaGeo<LOGD, NCOL>;
-    using L = UmmaFwdSmem<LOGD, NCOL, STAGES, TP>;
+    using L = UmmaFwdSmem<LOGD, NCOL, STAGES, TP, RES>;
     constexpr int ACC = L::ACC;
     extern __shared__ __align__(1024) unsigned char umma_smem[];
     unsigned char* const smem_raw = umma_smem;
@@ -358,76 +363,141 @@ umma_fwd_kernel(const __nv_bfloat16* x, const TP* __restrict__ a, const TP* __re
         }
     } else {
         const int q = warp & 3;            // TMEM lane quarter this warp may access
-        const int ch = (warp - 2) >> 2;    // column half of the tile
+        const int ch = (warp - 2) >> 2;    // which of the two 4-warp groups
         const int m = q * 32 + lane;       // index bits 3..9 of every element this thread produces
-        const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + ch * Geo::CPW;
 
-        F2 as[L::PARAMS_IN_SMEM ? 1 : Geo::PIECES][4], bs[L::PARAMS_IN_SMEM ? 1 : Geo::PIECES][4];
-        const float* pa = reinterpret_cast<const float*>(smem_raw + L::OFF_PARAMS);
-        if constexpr (!L::PARAMS_IN_SMEM) {
-            const F2 rs2 = f2(inv_sqrt_d, inv_sqrt_d);
+        if constexpr (L::SPLIT) {
+            // d = 8192 without a residual: each group owns the channels of one value of the top index
+            // bit for ALL rows of the tile, so that its share of a and b (32 values each) stays in
+            // registers; it applies the stage on that bit first, straight on the two column halves
+            // of the accumulator (lo + hi or lo - hi).
+            constexpr int RE = Geo::R / 2, PE = RE / 8;
+            const int piece0 = ch * PE;
+            const F2 top_sign = ch ? f2(-1.0f, -1.0f) : f2(1.0f, 1.0f);
+            const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
+            F2 as[PE][4], bs[PE][4];
+            {
+                const F2 rs2 = f2(inv_sqrt_d, inv_sqrt_d);
 #pragma unroll
-            for (int p = 0; p < Geo::PIECES; ++p) {
-                load_params8(a + p * 1024 + m * 8, as[p]);
-                load_params8(b + p * 1024 + m * 8, bs[p]);
+                for (int p = 0; p < PE; ++p) {
+                    load_params8(a + (piece0 + p) * 1024 + m * 8, as[p]);
+                    load_params8(b + (piece0 + p) * 1024 + m * 8, bs[p]);
 #pragma unroll
-                for (int j = 0; j < 4; ++j) as[p][j] = mul2(as[p][j], rs2);
+                    for (int j = 0; j < 4; ++j) as[p][j] = mul2(as[p][j], rs2);
+                }
             }
-        }
-
-        for (long long it = 0; it < my_tiles; ++it) {
-            const int t = static_cast<int>(it % ACC);
-            const uint32_t pt = static_cast<uint32_t>(it / ACC) & 1u;
-            uint4 res[RES ? Geo::RPW * Geo::PIECES : 1];
-            if constexpr (RES) {
-                const long long tile_r = blockIdx.x + it * gridDim.x;
+            for (long long it = 0; it < my_tiles; ++it) {
+                const int t = static_cast<int>(it % ACC);
+                const uint32_t pt = static_cast<uint32_t>(it / ACC) & 1u;
+                if (!warp_wait_or_abort(acc_full + t, pt, abort_flag)) break;
+                tc_fence_after();
+                const long long tile = blockIdx.x + it * gridDim.x;
 #pragma unroll
-                for (int rl = 0; rl < Geo::RPW; ++rl) {
-                    const long long row = tile_r * Geo::ROWS + ch * Geo::RPW + rl;
+                for (int r = 0; r < Geo::ROWS; ++r) {
+                    const long long row = tile * Geo::ROWS + r;
+                    float lo[RE], hi[RE];
+                    tmem_ld_cols<RE>(lane_addr + t * Geo::N + r * Geo::R, lo);
+                    tmem_ld_cols<RE>(lane_addr + t * Geo::N + r * Geo::R + RE, hi);
+                    tmem_wait_ld();
+                    if (r == Geo::ROWS - 1) {
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(acc_empty + t);  // the accumulator is in registers now
+                    }
+                    float v[RE];
 #pragma unroll
-                    for (int p = 0; p < Geo::PIECES; ++p) {
-                        res[rl * Geo::PIECES + p] = make_uint4(0u, 0u, 0u, 0u);
-                        if (row < T)
-                            res[rl * Geo::PIECES + p] =
-                                __ldcs(reinterpret_cast<const uint4*>(resid + row * Geo::D + m * 8) + p * 128);
+                    for (int i = 0; i < RE; i += 2) {
+                        const F2 o = fma2(f2(hi[i], hi[i + 1]), top_sign, f2(lo[i], lo[i + 1]));
+                        v[i] = o.x;
+                        v[i + 1] = o.y;
+                    }
+                    thread_stages<RE>(v);
+                    if (row < T) {
+                        uint4* dst = reinterpret_cast<uint4*>(y + row * Geo::D + piece0 * 1024 + m * 8);
+#pragma unroll
+                        for (int p = 0; p < PE; ++p) {
+                            F2 w[4];
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) w[j] = f2(v[p * 8 + 2 * j], v[p * 8 + 2 * j + 1]);
+                            fwd_store_chunk(w, as[p], bs[p], dst + p * 128);
+                        }
                     }
                 }
             }
-            if (!warp_wait_or_abort(acc_full + t, pt, abort_flag)) break;
-            tc_fence_after();
-            float u[Geo::CPW];
-            tmem_ld_cols<Geo::CPW>(lane_addr + t * Geo::N, u);
-            tmem_wait_ld();
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(acc_empty + t);  // the accumulator is in registers now
+        } else {
+            // each group takes half of the tile's rows, every channel of them
+            const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + ch * Geo::CPW;
+            F2 as[L::PARAMS_IN_SMEM ? 1 : Geo::PIECES][4], bs[L::PARAMS_IN_SMEM ? 1 : Geo::PIECES][4];
+            const float* pa = reinterpret_cast<const float*>(smem_raw + L::OFF_PARAMS);
+            if constexpr (!L::PARAMS_IN_SMEM) {
+                const F2 rs2 = f2(inv_sqrt_d, inv_sqrt_d);
+#pragma unroll
+                for (int p = 0; p < Geo::PIECES; ++p) {
+                    load_params8(a + p * 1024 + m * 8, as[p]);
+                    load_params8(b + p * 1024 + m * 8, bs[p]);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) as[p][j] = mul2(as[p][j], rs2);
+                }
+            }
 
-            const long long tile = blockIdx.x + it * gridDim.x;
+            for (long long it = 0; it < my_tiles; ++it) {
+                const int t = static_cast<int>(it % ACC);
+                const uint32_t pt = static_cast<uint32_t>(it / ACC) & 1u;
+                const long long tile = blockIdx.x + it * gridDim.x;
+                // the residual chunks of this thread's rows are fetched ahead of the accumulator wait
+                uint4 res[RES ? Geo::RPW * Geo::PIECES : 1];
+                if constexpr (RES) {
 #pragma unroll
-            for (int rl = 0; rl < Geo::RPW; ++rl) {
-                const long long row = tile * Geo::ROWS + ch * Geo::RPW + rl;
-                float v[Geo::R];
+                    for (int rl = 0; rl < Geo::RPW; ++rl) {
+                        const long long row = tile * Geo::ROWS + ch * Geo::RPW + rl;
 #pragma unroll
-                for (int i = 0; i < Geo::R; ++i) v[i] = u[rl * Geo::R + i];
-                thread_stages<Geo::R>(v);
-                if (row < T) {
-                    uint4* dst = reinterpret_cast<uint4*>(y + row * Geo::D + m * 8);
+                        for (int p = 0; p < Geo::PIECES; ++p) {
+                            res[rl * Geo::PIECES + p] = make_uint4(0u, 0u, 0u, 0u);
+                            if (row < T)
+                                res[rl * Geo::PIECES + p] =
+                                    __ldcs(reinterpret_cast<const uint4*>(resid + row * Geo::D + m * 8) + p * 128);
+                        }
+                    }
+                }
+                if (!warp_wait_or_abort(acc_full + t, pt, abort_flag)) break;
+                tc_fence_after();
+                float u[Geo::CPW];
+                tmem_ld_cols<Geo::CPW>(lane_addr + t * Geo::N, u);
+                tmem_wait_ld();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(acc_empty + t);  // the accumulator is in registers now
+
 #pragma unroll
-                    for (int p = 0; p < Geo::PIECES; ++p) {
-                        F2 w[4];
+                for (int rl = 0; rl < Geo::RPW; ++rl) {
+                    const long long row = tile * Geo::ROWS + ch * Geo::RPW + rl;
+                    float v[Geo::R];
 #pragma unroll
-                        for (int j = 0; j < 4; ++j) w[j] = f2(v[p * 8 + 2 * j], v[p * 8 + 2 * j + 1]);
-                        if constexpr (L::PARAMS_IN_SMEM) {
-                            const float4* qa = reinterpret_cast<const float4*>(pa) + (p * 2) * 128 + m;
-                            const float4* qb = reinterpret_cast<const float4*>(pa + Geo::D) + (p * 2) * 128 + m;
-                            const float4 a0 = qa[0], a1 = qa[128], b0 = qb[0], b1 = qb[128];
-                            F2 ap[4] = {f2(a0.x, a0.y), f2(a0.z, a0.w), f2(a1.x, a1.y), f2(a1.z, a1.w)};
-                            F2 bp[4] = {f2(b0.x, b0.y), f2(b0.z, b0.w), f2(b1.x, b1.y), f2(b1.z, b1.w)};
-                            if constexpr (RES) fwd_store_chunk_res(w, ap, bp, res[rl * Geo::PIECES + p], dst + p * 128);
-                            else fwd_store_chunk(w, ap, bp, dst + p * 128);
-                        } else {
-                            if constexpr (RES) fwd_store_chunk_res(w, as[p], bs[p], res[rl * Geo::PIECES + p], dst + p * 128);
-                            else fwd_store_chunk(w, as[p], bs[p], dst + p * 128);
+                    for (int i = 0; i < Geo::R; ++i) v[i] = u[rl * Geo::R + i];
+                    thread_stages<Geo::R>(v);
+                    if (row < T) {
+                        uint4* dst = reinterpret_cast<uint4*>(y + row * Geo::D + m * 8);
+#pragma unroll
+                        for (int p = 0; p < Geo::PIECES; ++p) {
+                            F2 w[4];
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) w[j] = f2(v[p * 8 + 2 * j], v[p * 8 + 2 * j + 1]);
+                            if constexpr (L::PARAMS_IN_SMEM) {
+                                const float4* qa = reinterpret_cast<const float4*>(pa) + (p * 2) * 128 + m;
+                                const float4* qb = reinterpret_cast<const float4*>(pa + Geo::D) + (p * 2) * 128 + m;
+                                const float4 a0 = qa[0], a1 = qa[128], b0 = qb[0], b1 = qb[128];
+                                F2 ap[4] = {f2(a0.x, a0.y), f2(a0.z, a0.w), f2(a1.x, a1.y), f2(a1.z, a1.w)};
+                                F2 bp[4] = {f2(b0.x, b0.y), f2(b0.z, b0.w), f2(b1.x, b1.y), f2(b1.z, b1.w)};
+                                if constexpr (RES)
+                                    fwd_store_chunk_res(w, ap, bp, res[rl * Geo::PIECES + p], dst + p * 128);
+                                else
+                                    fwd_store_chunk(w, ap, bp, dst + p * 128);
+                            } else {
+                                if constexpr (RES)
+                                    fwd_store_chunk_res(w, as[p], bs[p], res[rl * Geo::PIECES + p], dst + p * 128);
+                                else
+                                    fwd_store_chunk(w, as[p], bs[p], dst + p * 128);
+                            }
                         }
                     }
                 }

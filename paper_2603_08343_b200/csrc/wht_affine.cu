@@ -375,7 +375,7 @@ int prepare_umma(Kernel kernel, int smem, int dev, int* cache) {
 template <int LOGD, int NCOL, int STAGES, typename TP, bool RES>
 int launch_umma_fwd_impl(const FwdArgs& f, const Ctx& c) {
     using Geo = UmmaGeo<LOGD, NCOL>;
-    using L = UmmaFwdSmem<LOGD, NCOL, STAGES, TP>;
+    using L = UmmaFwdSmem<LOGD, NCOL, STAGES, TP, RES>;
     static_assert(L::BYTES > 116 * 1024, "must be alone on its SM");
     static int ready[kMaxDevices] = {};
     auto kernel = umma_fwd_kernel<LOGD, NCOL, STAGES, TP, RES>;
