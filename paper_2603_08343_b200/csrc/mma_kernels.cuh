@@ -353,6 +353,21 @@ mma_fwd_kernel(const __nv_bfloat16* x, const TP* __restrict__ a, const TP* __res
     grid_dependency_wait();
     grid_launch_dependents();
 
+    // With few chunks per thread (the few-rows / decode shapes) a and b are fetched once, up front,
+    // so that their latency overlaps the row load instead of following the transform.
+    constexpr bool PRELOAD = NT <= 4;
+    F2 pas[PRELOAD ? NT : 1][4], pbs[PRELOAD ? NT : 1][4];
+    if constexpr (PRELOAD) {
+#pragma unroll
+        for (int idx = 0; idx < NT; ++idx) {
+            const int c = chunk_of<Geo, true>(w, idx);
+            load_params8(a + (c * 32 + lane) * 8, pas[idx]);
+            load_params8(b + (c * 32 + lane) * 8, pbs[idx]);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) pas[idx][j] = mul2(pas[idx][j], rs2);
+        }
+    }
+
     int parity = 0;
     const long long stride = static_cast<long long>(gridDim.x) * RG;
     for (long long row = static_cast<long long>(blockIdx.x) * RG + rg; row < T; row += stride) {
@@ -360,6 +375,13 @@ mma_fwd_kernel(const __nv_bfloat16* x, const TP* __restrict__ a, const TP* __res
         uint4 raw[NT];
 #pragma unroll
         for (int t = 0; t < NT; ++t) raw[t] = __ldcs(src + chunk_of<Geo, false>(w, t) * 32 + lane);
+        uint4 res[NT];
+        if (resid != nullptr) {  // the residual chunks too, ahead of the transform
+#pragma unroll
+            for (int idx = 0; idx < NT; ++idx)
+                res[idx] = __ldcs(reinterpret_cast<const uint4*>(resid + row * Geo::D) +
+                                  chunk_of<Geo, true>(w, idx) * 32 + lane);
+        }
         F2 m[NT][2][2];
         F2 v[NT][4];
         X::pass1_raw(raw, m, hf);
@@ -372,13 +394,17 @@ mma_fwd_kernel(const __nv_bfloat16* x, const TP* __restrict__ a, const TP* __res
         for (int idx = 0; idx < NT; ++idx) {
             const int c = chunk_of<Geo, true>(w, idx);
             F2 as[4], bs[4];
-            load_params8(a + (c * 32 + lane) * 8, as);
-            load_params8(b + (c * 32 + lane) * 8, bs);
+            if constexpr (PRELOAD) {
 #pragma unroll
-            for (int j = 0; j < 4; ++j) as[j] = mul2(as[j], rs2);
+                for (int j = 0; j < 4; ++j) { as[j] = pas[idx][j]; bs[j] = pbs[idx][j]; }
+            } else {
+                load_params8(a + (c * 32 + lane) * 8, as);
+                load_params8(b + (c * 32 + lane) * 8, bs);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) as[j] = mul2(as[j], rs2);
+            }
             if (resid != nullptr) {
-                const uint4 r = __ldcs(reinterpret_cast<const uint4*>(resid + row * Geo::D) + c * 32 + lane);
-                fwd_store_chunk_res(v[idx], as, bs, r, dst + c * 32 + lane);
+                fwd_store_chunk_res(v[idx], as, bs, res[idx], dst + c * 32 + lane);
             } else {
                 fwd_store_chunk(v[idx], as, bs, dst + c * 32 + lane);
             }
