@@ -316,7 +316,8 @@ int dispatch_mma_fwd(int logd, bool few_rows, bool streamed, const FwdArgs& f, c
             case 9: return launch_mma_fwd<9, 1, 4, TP>(f, c);
             case 10: return launch_mma_fwd<10, 1, 2, TP>(f, c);
             case 11: return launch_mma_fwd<11, 2, 2, TP>(f, c);
-            case 12: return launch_mma_fwd<12, 2, 1, TP>(f, c);
+            // one row per CTA while every row gets an SM of its own, two beyond that
+            case 12: return c.T > c.sms ? launch_mma_fwd<12, 2, 2, TP>(f, c) : launch_mma_fwd<12, 2, 1, TP>(f, c);
             case 13: return launch_mma_fwd<13, 3, 1, TP>(f, c);
         }
     } else if (!streamed) {
