@@ -314,13 +314,13 @@ def section_fwd_bwd(B, name, hbm_peak, iters):
     y = torch.empty_like(x)
     da = torch.empty(w.d, dtype=torch.float32, device="cuda")
     db = torch.empty_like(da)
-    f_ms = time_loop(lambda: B.wht_affine_fwd(x, a, b, y, w.T, w.d, w.dtype), iters)
-    b_ms = time_loop(lambda: B.wht_affine_bwd(dy, x, a, y, da, db, w.T, w.d, w.dtype), iters)
-    c_ms = time_loop(lambda: B.wht_copy_rows(x, y, w.T, w.d, w.dtype), iters)
-    r_ms = time_loop(lambda: B.wht_affine_fwd_residual(x, a, b, dy, y, w.T, w.d, w.dtype), iters)
+    f_ms = time_loop(lambda: B.wht_affine_fwd(x, a, b, y, w.T, w.d, w.dtype), iters, warmup=10)
+    b_ms = time_loop(lambda: B.wht_affine_bwd(dy, x, a, y, da, db, w.T, w.d, w.dtype), iters, warmup=10)
+    c_ms = time_loop(lambda: B.wht_copy_rows(x, y, w.T, w.d, w.dtype), iters, warmup=10)
+    r_ms = time_loop(lambda: B.wht_affine_fwd_residual(x, a, b, dy, y, w.T, w.d, w.dtype), iters, warmup=10)
     fb = 2 * w.T * w.d * w.io_bytes / 1e9
     bb = 3 * w.T * w.d * w.io_bytes / 1e9
-    res = {"T": w.T, "d": w.d, "rows_drawn": base_rows, "rows_tiled": reps,
+    res = {"T": w.T, "d": w.d, "rows_drawn": base_rows, "rows_tiled": reps, "iters": iters, "warmup": 10,
            "fwd_us": 1e3 * f_ms, "fwd_GBps": fb / (f_ms * 1e-3), "fwd_frac_of_measured_peak": fb / (f_ms * 1e-3) / hbm_peak,
            "fwd_frac_of_8000": fb / (f_ms * 1e-3) / 8000.0, "fwd_tokens_per_s": w.T / (f_ms * 1e-3),
            "bwd_us": 1e3 * b_ms, "bwd_GBps": bb / (b_ms * 1e-3), "bwd_frac_of_measured_peak": bb / (b_ms * 1e-3) / hbm_peak,
@@ -549,8 +549,8 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         sections = {}
         sections["prefill"] = section_prefill(B, hbm_peak)
         sections["decode"] = section_decode(B)
-        sections["training"] = section_fwd_bwd(B, "training", hbm_peak, 20)
-        sections["large"] = section_fwd_bwd(B, "large", hbm_peak, 5)
+        sections["training"] = section_fwd_bwd(B, "training", hbm_peak, 50)
+        sections["large"] = section_fwd_bwd(B, "large", hbm_peak, 50)
         sections["paper_shapes"] = section_paper_shapes(B, hbm_peak)
         out["sections"] = sections
     print(json.dumps(out))
