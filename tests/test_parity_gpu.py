@@ -534,6 +534,27 @@ def test_grouped_form(B, d, block, dtype, T):
     assert err.value.status == -2
 
 
+def test_autograd_wrapper(B):
+    from paper_2603_08343_b200.autograd import wht_affine
+    B.wht_affine_set_variant(0)
+    w = wl.CONFIGS["training"].with_rows(6 * 50)
+    x, dy, r = wl.gen_full(w, "x"), wl.gen_full(w, "dy"), wl.gen_full(w.with_rows(300), "x").flip(0)
+    a, b = wl.gen_params(w)
+    xd = x.cuda().view(6, 50, w.d).requires_grad_(True)        # [batch, seq, d]
+    ad, bd = a.cuda().requires_grad_(True), b.cuda().requires_grad_(True)
+    rd = r.cuda().view(6, 50, w.d).requires_grad_(True)
+    out = wht_affine(xd, ad, bd, resid=rd)
+    out.backward(dy.cuda().view(6, 50, w.d))
+    torch.cuda.synchronize()
+    ref_y = oracle.wht_affine_fwd_residual(to_f64(x), to_f64(a), to_f64(b), to_f64(r))
+    ref_dx, ref_da, ref_db = oracle.wht_affine_bwd(to_f64(dy), to_f64(x), to_f64(a))
+    assert_rows_bf16(to_f64(out.detach().cpu().view(-1, w.d)), ref_y, "autograd y")
+    assert_rows_bf16(to_f64(xd.grad.cpu().view(-1, w.d)), ref_dx, "autograd dx")
+    assert_grad_vec(to_f64(ad.grad.cpu()), ref_da, "autograd da")
+    assert_grad_vec(to_f64(bd.grad.cpu()), ref_db, "autograd db")
+    assert torch.equal(rd.grad.view(-1, w.d).cpu(), dy)
+
+
 def test_copy_rows(B):
     src = torch.arange(3 * 1024, dtype=torch.float32, device="cuda").view(3, 1024)
     dst = torch.zeros_like(src)
