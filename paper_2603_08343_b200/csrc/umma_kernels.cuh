@@ -293,22 +293,35 @@ umma_fwd_kernel(const __nv_bfloat16* x, const TP* __restrict__ a, const TP* __re
     const long long tiles = (T + Geo::ROWS - 1) / Geo::ROWS;
     const long long my_tiles = blockIdx.x < tiles ? (tiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
 
-    if (tid == 0) {
-        for (int s = 0; s < STAGES; ++s) { mbar_init(full + s, 1); mbar_init(empty + s, 1); }
-        for (int t = 0; t < ACC; ++t) { mbar_init(acc_full + t, 1); mbar_init(acc_empty + t, Geo::EPI_WARPS); }
-        *abort_flag = 0;
-        fence_mbar_init();
+    // Set-up.  The producer warp only needs the barriers: it initialises them, signals the others
+    // (bar.arrive, it does not wait) and starts copying rows while they build H_128 and allocate
+    // tensor memory; calls of a few tiles per SM are mostly ramp-up, so this start counts.
+    uint32_t tmem_base = 0;
+    if (warp == 0) {
+        if (lane == 0) {
+            for (int s = 0; s < STAGES; ++s) { mbar_init(full + s, 1); mbar_init(empty + s, 1); }
+            for (int t = 0; t < ACC; ++t) { mbar_init(acc_full + t, 1); mbar_init(acc_empty + t, Geo::EPI_WARPS); }
+            *abort_flag = 0;
+            fence_mbar_init();
+        }
+        __syncwarp();
+        if constexpr (L::PARAMS_IN_SMEM) {
+            named_barrier(2, Geo::THREADS);
+        } else {
+            asm volatile("bar.arrive 2, %0;" ::"r"(Geo::THREADS) : "memory");
+        }
+    } else {
+        write_h128(smem_raw + L::OFF_H, tid - 32, Geo::THREADS - 32);
+        fence_async_smem();  // H_128 was written by ordinary stores and is read by the tensor core
+        if (warp == 1) {
+            tmem_alloc(tmem_slot, L::TMEM_COLS);
+            tmem_relinquish();
+        }
+        tc_fence_before();
+        named_barrier(2, Geo::THREADS);
+        tc_fence_after();
+        tmem_base = *tmem_slot;
     }
-    write_h128(smem_raw + L::OFF_H, tid, Geo::THREADS);
-    fence_async_smem();  // H_128 was written by ordinary stores and is read by the tensor core
-    if (warp == 1) {
-        tmem_alloc(tmem_slot, L::TMEM_COLS);
-        tmem_relinquish();
-    }
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem_base = *tmem_slot;
     // everything above touched only this CTA's own shared and tensor memory
     grid_dependency_wait();
     grid_launch_dependents();
