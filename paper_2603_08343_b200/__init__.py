@@ -10,13 +10,18 @@ library raises: there is no CPU fallback.
 from . import workloads  # noqa: F401
 
 
+_SUBMODULES = ("binding", "build", "dp", "autograd", "workloads")
+
+
 def __getattr__(name):
-    # The binding (and with it the shared library) is loaded lazily so that
-    # input generation can be imported on machines without the built library.
-    if name == "binding":
-        import importlib
-        return importlib.import_module(".binding", __name__)
-    from . import binding as _b
+    # The binding (and with it the shared library) is loaded lazily so that input generation and
+    # the build step can be imported on machines without the built library.
+    import importlib
+    if name in _SUBMODULES:
+        return importlib.import_module("." + name, __name__)
+    if name.startswith("__"):
+        raise AttributeError(name)
+    _b = importlib.import_module(".binding", __name__)
     if hasattr(_b, name):
         return getattr(_b, name)
     raise AttributeError(name)
