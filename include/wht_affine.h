@@ -175,6 +175,43 @@ int wht_affine_bwd_grouped(const void* dy, const void* x, const void* a,
 size_t wht_affine_bwd_grouped_workspace_bytes(int64_t T, int32_t d, int32_t block, int dtype);
 
 /*
+ * Column-sharded (tensor-parallel) form, for attention whose heads are split over g GPUs: rank s
+ * holds channels [s*w, (s+1)*w) of every row, as a contiguous [T x w] tensor of its own, and the
+ * model width is d = g * w.  The paper trains data-parallel only and has no such form; it follows
+ * from Eq. 1 and the Kronecker structure of the Sylvester matrix, H_d = H_g (x) H_w:
+ *     y_r  = a_r (.) ( (sum_s H_g[s][r] x_s) H_w ) / sqrt(d) + b_r,    H_g[s][r] = (-1)^popcount(s & r)
+ *     dx_r = ( (sum_s H_g[r][s] (a_s (.) dy_s)) H_w ) / sqrt(d)
+ *     da_r = sum_t dy_r (.) z_r,   z_r = ( (sum_s H_g[s][r] x_s) H_w ) / sqrt(d),     db_r = sum_t dy_r
+ * which are exactly column block r of wht_affine_fwd / wht_affine_bwd on the concatenated tensors.
+ * One kernel per call reads the g blocks (its own and the peers') with plain loads, forms the
+ * signed sum of the stored values in fp32 and runs the width-w transform: the exchange of the top
+ * log2 g stages and the local stages are fused, no intermediate is written.  No multicast.
+ *   x_parts, dy_parts, a_parts  HOST arrays of g DEVICE pointers; entry s is rank s's block
+ *                  (x, dy: [T x w] row-major; a: [w]); entry r is this GPU's own memory, the others
+ *                  are peer mappings the caller obtained (CUDA IPC, symmetric memory) and keeps valid
+ *                  and unchanged until the call has completed on `stream`.  The array itself is
+ *                  read before the call returns.
+ *   a, b           this rank's parameter blocks [w]; y, dx: this rank's output blocks [T x w];
+ *                  da, db [w] fp32, overwritten.
+ *   w              power of two in [8, 32768]; g in {1, 2, 4, 8}; 0 <= r < g; g = 1 is the plain call.
+ *   Outputs must not alias any input block (other ranks read the inputs at the same time).
+ * The call does not synchronise ranks: the caller makes sure every rank's inputs are complete before
+ * any rank launches (a barrier across ranks on the host or stream), and that no rank overwrites its
+ * inputs before every rank's call has completed.  Gradients of a and b need no reduction across the
+ * g ranks (each rank owns its channels); across data-parallel replicas they add as usual.
+ * Butterfly kernels; every storage type.  The backward takes caller-owned scratch of at least
+ * wht_affine_bwd_tp_workspace_bytes(T, w, g, dtype) bytes and never allocates.
+ * Errors as for the plain calls; g or r out of range -> WHT_ERR_BAD_DIM.
+ */
+int wht_affine_fwd_tp(const void* const* x_parts, const void* a, const void* b, void* y,
+                      int64_t T, int32_t w, int32_t g, int32_t r, int dtype, void* stream);
+int wht_affine_bwd_tp(const void* const* dy_parts, const void* const* x_parts, const void* const* a_parts,
+                      void* dx, float* da, float* db,
+                      int64_t T, int32_t w, int32_t g, int32_t r, int dtype,
+                      void* workspace, size_t workspace_bytes, void* stream);
+size_t wht_affine_bwd_tp_workspace_bytes(int64_t T, int32_t w, int32_t g, int dtype);
+
+/*
  * Sums the parameter gradients of n backward calls (row chunks of one batch, or micro-batches
  * whose gradients accumulate): da[j] = sum_p parts[p][0][j], db[j] = sum_p parts[p][1][j].
  * da and db of Eq. 1's backward are sums over rows, so the gradients of disjoint row sets add.

@@ -10,7 +10,7 @@ library raises: there is no CPU fallback.
 from . import workloads  # noqa: F401
 
 
-_SUBMODULES = ("binding", "build", "dp", "autograd", "workloads")
+_SUBMODULES = ("binding", "build", "dp", "tp", "autograd", "workloads")
 
 
 def __getattr__(name):

@@ -20,6 +20,7 @@ LIB_PATH = os.path.join(_HERE, "libwht_affine.so")
 EXPORTS = (
     "wht_affine_fwd", "wht_affine_fwd_residual", "wht_affine_fwd_decode", "wht_affine_bwd", "wht_affine_bwd_ws", "wht_affine_bwd_noalloc", "wht_affine_reduce_grads",
     "wht_affine_fwd_grouped", "wht_affine_bwd_grouped", "wht_affine_bwd_grouped_workspace_bytes",
+    "wht_affine_fwd_tp", "wht_affine_bwd_tp", "wht_affine_bwd_tp_workspace_bytes",
     "wht_affine_bwd_workspace_bytes", "wht_affine_set_variant", "wht_affine_get_variant",
     "wht_copy_rows", "wht_affine_device_status", "wht_affine_last_cuda_error", "wht_affine_status_string",
     "wht_affine_shutdown",
@@ -52,6 +53,10 @@ def _load() -> ctypes.CDLL:
     lib.wht_affine_bwd_grouped.argtypes = [vp, vp, vp, vp, vp, vp, i64, i32, i32, ci, vp, sz, vp]
     lib.wht_affine_bwd_grouped_workspace_bytes.argtypes = [i64, i32, i32, ci]
     lib.wht_affine_bwd_grouped_workspace_bytes.restype = sz
+    lib.wht_affine_fwd_tp.argtypes = [vp, vp, vp, vp, i64, i32, i32, i32, ci, vp]
+    lib.wht_affine_bwd_tp.argtypes = [vp, vp, vp, vp, vp, vp, i64, i32, i32, i32, ci, vp, sz, vp]
+    lib.wht_affine_bwd_tp_workspace_bytes.argtypes = [i64, i32, i32, ci]
+    lib.wht_affine_bwd_tp_workspace_bytes.restype = sz
     lib.wht_affine_bwd_workspace_bytes.argtypes = [i64, i32, ci]
     lib.wht_affine_bwd_workspace_bytes.restype = sz
     lib.wht_affine_set_variant.argtypes = [ci]
@@ -168,6 +173,37 @@ def wht_affine_bwd_grouped(dy, x, a, dx, da, db, T: int, d: int, block: int, dty
 
 def wht_affine_bwd_grouped_workspace_bytes(T: int, d: int, block: int, dtype: int) -> int:
     return int(_lib.wht_affine_bwd_grouped_workspace_bytes(T, d, block, dtype))
+
+
+def _ptr_array(parts):
+    """Host array of device pointers; entries are tensors or integer addresses (peer mappings)."""
+    addrs = [p if isinstance(p, int) else p.data_ptr() for p in parts]
+    return (ctypes.c_void_p * len(addrs))(*addrs)
+
+
+def wht_affine_fwd_tp(x_parts, a, b, y, T: int, w: int, g: int, r: int, dtype: int, stream=None) -> None:
+    """Column-sharded forward of rank r: x_parts[s] is rank s's [T, w] block (tensor or device address)."""
+    _require_cuda(a, b, y, *[p for p in x_parts if not isinstance(p, int)])
+    if len(x_parts) != g:
+        raise ValueError(f"{len(x_parts)} blocks for g = {g}")
+    _check(_lib.wht_affine_fwd_tp(_ptr_array(x_parts), _ptr(a), _ptr(b), _ptr(y), T, w, g, r, dtype,
+                                  _stream(stream)), "wht_affine_fwd_tp")
+
+
+def wht_affine_bwd_tp(dy_parts, x_parts, a_parts, dx, da, db, T: int, w: int, g: int, r: int, dtype: int,
+                      workspace, stream=None) -> None:
+    _require_cuda(dx, da, db, workspace,
+                  *[p for p in (*dy_parts, *x_parts, *a_parts) if not isinstance(p, int)])
+    if not len(dy_parts) == len(x_parts) == len(a_parts) == g:
+        raise ValueError(f"every list needs g = {g} blocks")
+    nbytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(_lib.wht_affine_bwd_tp(_ptr_array(dy_parts), _ptr_array(x_parts), _ptr_array(a_parts), _ptr(dx),
+                                  _ptr(da), _ptr(db), T, w, g, r, dtype, _ptr(workspace), nbytes,
+                                  _stream(stream)), "wht_affine_bwd_tp")
+
+
+def wht_affine_bwd_tp_workspace_bytes(T: int, w: int, g: int, dtype: int) -> int:
+    return int(_lib.wht_affine_bwd_tp_workspace_bytes(T, w, g, dtype))
 
 
 def wht_affine_bwd_workspace_bytes(T: int, d: int, dtype: int) -> int:

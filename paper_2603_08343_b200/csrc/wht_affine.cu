@@ -10,6 +10,7 @@
 #include "bfly_kernels.cuh"
 #include "mma_kernels.cuh"
 #include "mma_pipe_kernels.cuh"
+#include "tp_kernels.cuh"
 #include "umma_kernels.cuh"
 
 namespace {
@@ -154,13 +155,14 @@ struct BwdArgs {
     size_t* need;
 };
 
-int launch_finalize(const BwdArgs& g, int nparts, int d, cudaStream_t s) {
+// da = scale * (sum of the partials' first slots), db = sum of their second slots
+int launch_finalize(const BwdArgs& g, int nparts, int d, float scale, cudaStream_t s) {
     if (d >= 32) {
         launch_overlapped(dadb_finalize32_kernel, 2 * d / 32, 1024, 0, s, static_cast<const float*>(g.ws), nparts, d,
-                          inv_sqrt(d), g.da, g.db);
+                          scale, g.da, g.db);
     } else {
         launch_overlapped(dadb_finalize_kernel, (2 * d + 255) / 256, 256, 0, s, static_cast<const float*>(g.ws),
-                          nparts, d, inv_sqrt(d), g.da, g.db);
+                          nparts, d, scale, g.da, g.db);
     }
     WHT_CUDA_TRY(cudaGetLastError());
     return WHT_OK;
@@ -168,7 +170,7 @@ int launch_finalize(const BwdArgs& g, int nparts, int d, cudaStream_t s) {
 
 // Common tail of every backward launcher: size the scratch, check it, launch.
 template <typename Launch>
-int run_bwd_with_grid(const BwdArgs& g, const Ctx& c, int grid, int d, Launch launch) {
+int run_bwd_with_grid(const BwdArgs& g, const Ctx& c, int grid, int d, Launch launch, float scale = 0.0f) {
     *g.need = static_cast<size_t>(grid) * 2 * d * sizeof(float);
     if (g.query_only) return WHT_OK;
     if (*g.need > 0 && (g.ws == nullptr || g.ws_bytes < *g.need)) return WHT_ERR_WORKSPACE;
@@ -176,7 +178,7 @@ int run_bwd_with_grid(const BwdArgs& g, const Ctx& c, int grid, int d, Launch la
         launch(grid);
         WHT_CUDA_TRY(cudaGetLastError());
     }
-    return launch_finalize(g, grid, d, c.stream);
+    return launch_finalize(g, grid, d, scale > 0.0f ? scale : inv_sqrt(d), c.stream);
 }
 
 int capped_grid(int64_t tiles, int sms, int per_sm) {
@@ -538,6 +540,108 @@ int noalloc_scratch_for_current_device(int dev, void** out) {
     return WHT_OK;
 }
 
+// ------------------------------------------------------------------ column-sharded (tensor-parallel) form
+struct TpCall {
+    TpParts xs;       // the g blocks of x (this rank's own and the peers')
+    TpParts dys;      // backward only
+    TpParts as;       // backward only: every rank's a block
+    int g;
+    int r;
+    unsigned neg_mask;  // bit s set: H_g[s][r] = -1
+    float scale;        // 1/sqrt(g*w)
+};
+
+template <int LOGW, typename TIO, typename TP>
+int launch_bfly_fwd_tp(const TpCall& t, const FwdArgs& f, const Ctx& c) {
+    using Geo = BflyGeo<LOGW>;
+    static int occ[kMaxDevices] = {};
+    auto kernel = bfly_fwd_tp_kernel<LOGW, TIO, TP>;
+    const int per_sm = resident_ctas(kernel, Geo::THREADS, Geo::SMEM_FWD, c.dev, occ);
+    if (per_sm <= 0) return cuda_fail(cudaGetLastError());
+    const int grid = capped_grid(ceil_div(c.T, Geo::R), c.sms, per_sm);
+    kernel<<<grid, Geo::THREADS, Geo::SMEM_FWD, c.stream>>>(t.xs, t.g, t.neg_mask, static_cast<const TP*>(f.a),
+                                                            static_cast<const TP*>(f.b), static_cast<TIO*>(f.y),
+                                                            static_cast<long long>(c.T), t.scale);
+    WHT_CUDA_TRY(cudaGetLastError());
+    return WHT_OK;
+}
+
+template <int LOGW, typename TIO, typename TP>
+int launch_bfly_bwd_tp(const TpCall& t, const BwdArgs& g, const Ctx& c) {
+    using Geo = BflyGeo<LOGW>;
+    static int occ[kMaxDevices] = {};
+    auto kernel = bfly_bwd_tp_kernel<LOGW, TIO, TP>;
+    const int per_sm = resident_ctas(kernel, Geo::THREADS, Geo::SMEM_BWD, c.dev, occ);
+    if (per_sm <= 0) return cuda_fail(cudaGetLastError());
+    const int grid = capped_grid(ceil_div(c.T, Geo::R), c.sms, per_sm);
+    return run_bwd_with_grid(
+        g, c, grid, Geo::D,
+        [&](int n) {
+            kernel<<<n, Geo::THREADS, Geo::SMEM_BWD, c.stream>>>(t.dys, t.xs, t.as, t.g, t.r, t.neg_mask,
+                                                                 static_cast<TIO*>(g.dx), static_cast<float*>(g.ws),
+                                                                 static_cast<long long>(c.T), t.scale);
+        },
+        t.scale);
+}
+
+template <typename TIO, typename TP>
+int dispatch_bfly_fwd_tp(int logw, const TpCall& t, const FwdArgs& f, const Ctx& c) {
+    switch (logw) {
+#define M(L) case L: return launch_bfly_fwd_tp<L, TIO, TP>(t, f, c);
+        WHT_FOR_EACH_LOGD(M)
+#undef M
+    }
+    return WHT_ERR_BAD_DIM;
+}
+
+template <typename TIO, typename TP>
+int dispatch_bfly_bwd_tp(int logw, const TpCall& t, const BwdArgs& g, const Ctx& c) {
+    switch (logw) {
+#define M(L) case L: return launch_bfly_bwd_tp<L, TIO, TP>(t, g, c);
+        WHT_FOR_EACH_LOGD(M)
+#undef M
+    }
+    return WHT_ERR_BAD_DIM;
+}
+
+int check_tp(int64_t T, int32_t w, int32_t g, int32_t r, int dtype) {
+    int rc = check_common(T, w, dtype);
+    if (rc != WHT_OK) return rc;
+    if (!is_pow2(g) || g > kTpMaxRanks || r < 0 || r >= g) return WHT_ERR_BAD_DIM;
+    return WHT_OK;
+}
+
+// Copies g device pointers out of a host array, checking each.
+int gather_parts(const void* const* parts, int g, bool need_data, TpParts* out) {
+    if (!parts) return WHT_ERR_NULL;
+    for (int s = 0; s < kTpMaxRanks; ++s) out->p[s] = nullptr;
+    for (int s = 0; s < g; ++s) {
+        if (need_data && !parts[s]) return WHT_ERR_NULL;
+        if (!aligned16(parts[s])) return WHT_ERR_MISALIGNED;
+        out->p[s] = parts[s];
+    }
+    return WHT_OK;
+}
+
+unsigned tp_neg_mask(int g, int r) {
+    unsigned m = 0;
+    for (int s = 0; s < g; ++s)
+        if (__builtin_popcount(static_cast<unsigned>(s & r)) & 1) m |= 1u << s;
+    return m;
+}
+
+int run_bwd_tp(const TpCall& t, const BwdArgs& g, int64_t T, int32_t w, int dtype, cudaStream_t s) {
+    Ctx c{T, 0, 0, s};
+    int rc = current_device(&c.dev, &c.sms);
+    if (rc != WHT_OK) return rc;
+    const int logw = log2_of(w);
+    switch (dtype) {
+        case WHT_F32: return dispatch_bfly_bwd_tp<float, float>(logw, t, g, c);
+        case WHT_BF16: return dispatch_bfly_bwd_tp<__nv_bfloat16, __nv_bfloat16>(logw, t, g, c);
+        default: return dispatch_bfly_bwd_tp<__nv_bfloat16, float>(logw, t, g, c);
+    }
+}
+
 int query_bwd_bytes(int64_t T, int32_t d, int dtype, size_t* need) {
     BwdArgs q{nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, 0, true, need};
     return run_bwd(q, T, d, dtype, nullptr);
@@ -737,6 +841,64 @@ size_t wht_affine_bwd_grouped_workspace_bytes(int64_t T, int32_t d, int32_t bloc
         default: rc = dispatch_bfly_bwd<__nv_bfloat16, float>(log2_of(block), q, c); break;
     }
     return rc == WHT_OK ? need : 0;
+}
+
+// ---- column-sharded (tensor-parallel) form: see the header.
+int wht_affine_fwd_tp(const void* const* x_parts, const void* a, const void* b, void* y, int64_t T, int32_t w,
+                      int32_t g, int32_t r, int dtype, void* stream) {
+    int rc = check_tp(T, w, g, r, dtype);
+    if (rc != WHT_OK) return rc;
+    if (!a || !b || (T > 0 && !y)) return WHT_ERR_NULL;
+    if (!aligned16(a) || !aligned16(b) || !aligned16(y)) return WHT_ERR_MISALIGNED;
+    TpCall t{};
+    rc = gather_parts(x_parts, g, T > 0, &t.xs);
+    if (rc != WHT_OK) return rc;
+    if (T == 0) return WHT_OK;
+    t.g = g;
+    t.r = r;
+    t.neg_mask = tp_neg_mask(g, r);
+    t.scale = static_cast<float>(1.0 / sqrt(static_cast<double>(g) * w));
+    Ctx c{T, 0, 0, static_cast<cudaStream_t>(stream)};
+    rc = current_device(&c.dev, &c.sms);
+    if (rc != WHT_OK) return rc;
+    const FwdArgs f{nullptr, a, b, y};
+    const int logw = log2_of(w);
+    switch (dtype) {
+        case WHT_F32: return dispatch_bfly_fwd_tp<float, float>(logw, t, f, c);
+        case WHT_BF16: return dispatch_bfly_fwd_tp<__nv_bfloat16, __nv_bfloat16>(logw, t, f, c);
+        default: return dispatch_bfly_fwd_tp<__nv_bfloat16, float>(logw, t, f, c);
+    }
+}
+
+size_t wht_affine_bwd_tp_workspace_bytes(int64_t T, int32_t w, int32_t g, int dtype) {
+    if (check_tp(T, w, g, 0, dtype) != WHT_OK) return 0;
+    size_t need = 0;
+    BwdArgs q{nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, 0, true, &need};
+    TpCall t{};
+    t.g = g;
+    if (run_bwd_tp(t, q, T, w, dtype, nullptr) != WHT_OK) return 0;
+    return need;
+}
+
+int wht_affine_bwd_tp(const void* const* dy_parts, const void* const* x_parts, const void* const* a_parts, void* dx,
+                      float* da, float* db, int64_t T, int32_t w, int32_t g, int32_t r, int dtype, void* workspace,
+                      size_t workspace_bytes, void* stream) {
+    int rc = check_tp(T, w, g, r, dtype);
+    if (rc != WHT_OK) return rc;
+    if (!da || !db || (T > 0 && !dx)) return WHT_ERR_NULL;
+    if (!aligned16(dx) || !aligned16(da) || !aligned16(db) || !aligned16(workspace)) return WHT_ERR_MISALIGNED;
+    TpCall t{};
+    rc = gather_parts(dy_parts, g, T > 0, &t.dys);
+    if (rc == WHT_OK) rc = gather_parts(x_parts, g, T > 0, &t.xs);
+    if (rc == WHT_OK) rc = gather_parts(a_parts, g, true, &t.as);
+    if (rc != WHT_OK) return rc;
+    t.g = g;
+    t.r = r;
+    t.neg_mask = tp_neg_mask(g, r);
+    t.scale = static_cast<float>(1.0 / sqrt(static_cast<double>(g) * w));
+    size_t need = 0;
+    BwdArgs b{nullptr, nullptr, nullptr, dx, da, db, workspace, workspace_bytes, false, &need};
+    return run_bwd_tp(t, b, T, w, dtype, static_cast<cudaStream_t>(stream));
 }
 
 int wht_affine_reduce_grads(const float* parts, int32_t n, int32_t d, float* da, float* db, void* stream) {

@@ -1,0 +1,100 @@
+"""Column-sharded (tensor-parallel) calls on one GPU: the g ranks' blocks live in separate tensors of
+the same device and every rank's call runs in turn (the calls only read their inputs, no kernel waits
+for another), then the concatenated blocks are compared with the fp64 oracle at the full width."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from helpers import assert_grad_vec, assert_rows_bf16, assert_rows_fp32, to_f64
+from paper_2603_08343_b200 import tp
+from paper_2603_08343_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2603_08343_b200 import build
+    build.build()
+    from paper_2603_08343_b200 import binding
+    yield binding
+    binding.wht_affine_device_status()
+
+
+CASES = [
+    (2, 128, wl.WHT_F32, 70), (4, 64, wl.WHT_F32, 33), (8, 8, wl.WHT_F32, 100),
+    (2, 1024, wl.WHT_BF16, 300), (4, 512, wl.WHT_BF16_PF32, 129), (8, 256, wl.WHT_BF16, 517),
+    (8, 1024, wl.WHT_BF16_PF32, 65), (2, 4096, wl.WHT_BF16, 19), (4, 2048, wl.WHT_BF16_PF32, 1111),
+    (1, 2048, wl.WHT_BF16, 40),
+]
+
+
+@pytest.mark.parametrize("g,w,dtype,T", CASES)
+def test_column_sharded_calls_match_the_full_width_oracle(B, g, w, dtype, T):
+    d = g * w
+    wk = wl.Workload("tp", T, d, dtype, "normal", 900 + d + g, True, "")
+    x, dy = wl.gen_full(wk, "x"), wl.gen_full(wk, "dy")
+    a, b = wl.gen_params(wk)
+    xs = [p.cuda() for p in tp.split_columns(x, g)]
+    dys = [p.cuda() for p in tp.split_columns(dy, g)]
+    as_ = [a[s * w:(s + 1) * w].contiguous().cuda() for s in range(g)]
+    bs = [b[s * w:(s + 1) * w].contiguous().cuda() for s in range(g)]
+    ys, dxs, das, dbs = [], [], [], []
+    for r in range(g):
+        rank = tp.TpWht(g, r)
+        ys.append(rank.forward(xs, as_[r], bs[r], T, w))
+        dx, da, db = rank.backward(dys, xs, as_, T, w)
+        dxs.append(dx); das.append(da); dbs.append(db)
+    torch.cuda.synchronize()
+    y = torch.cat(ys, dim=1).cpu()
+    dx = torch.cat(dxs, dim=1).cpu()
+    da, db = torch.cat(das).cpu(), torch.cat(dbs).cpu()
+    ref_y = oracle.wht_affine_fwd(to_f64(x), to_f64(a), to_f64(b))
+    ref_dx, ref_da, ref_db = oracle.wht_affine_bwd(to_f64(dy), to_f64(x), to_f64(a))
+    if dtype == wl.WHT_F32:
+        assert_rows_fp32(to_f64(y), ref_y, to_f64(x), "tp y")
+        assert_rows_fp32(to_f64(dx), ref_dx, to_f64(a)[None, :] * to_f64(dy), "tp dx")
+    else:
+        assert_rows_bf16(to_f64(y), ref_y, "tp y")
+        assert_rows_bf16(to_f64(dx), ref_dx, "tp dx")
+    assert_grad_vec(to_f64(da), ref_da, "tp da")
+    assert_grad_vec(to_f64(db), ref_db, "tp db")
+    if g == 1:  # one rank is the plain call (butterfly family)
+        B.wht_affine_set_variant(1)
+        assert torch.equal(ys[0], B.forward(xs[0], as_[0], bs[0]))
+        B.wht_affine_set_variant(0)
+
+
+def test_blocks_given_as_addresses_and_repeat_calls_are_bit_identical(B):
+    g, w, T, dtype = 4, 512, 257, wl.WHT_BF16_PF32
+    wk = wl.Workload("tp", T, g * w, dtype, "normal", 77, True, "")
+    x, dy = wl.gen_full(wk, "x"), wl.gen_full(wk, "dy")
+    a, b = wl.gen_params(wk)
+    xs = [p.cuda() for p in tp.split_columns(x, g)]
+    dys = [p.cuda() for p in tp.split_columns(dy, g)]
+    as_ = [a[s * w:(s + 1) * w].contiguous().cuda() for s in range(g)]
+    r = 3
+    rank = tp.TpWht(g, r)
+    b_r = b[r * w:(r + 1) * w].contiguous().cuda()
+    y1 = rank.forward(xs, as_[r], b_r, T, w)
+    y2 = torch.empty_like(y1)
+    rank.forward([t.data_ptr() for t in xs], as_[r], b_r, T, w, out=y2)   # peer mappings arrive as addresses
+    out1 = rank.backward(dys, xs, as_, T, w)
+    out2 = rank.backward([t.data_ptr() for t in dys], [t.data_ptr() for t in xs], as_, T, w, like=dys[r])
+    torch.cuda.synchronize()
+    assert torch.equal(y1, y2)
+    for u, v in zip(out1, out2):
+        assert torch.equal(u, v)
+
+
+def test_no_rows(B):
+    g, w = 2, 256
+    rank = tp.TpWht(g, 1)
+    a = torch.ones(w, device="cuda")
+    empty = [torch.empty((0, w), device="cuda") for _ in range(g)]
+    y = rank.forward(empty, a, a, 0, w)
+    dx, da, db = rank.backward(empty, empty, [a, a], 0, w)
+    torch.cuda.synchronize()
+    assert y.shape == (0, w) and dx.shape == (0, w)
+    assert torch.all(da == 0) and torch.all(db == 0)
