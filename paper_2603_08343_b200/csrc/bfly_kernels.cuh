@@ -6,33 +6,54 @@
 // bf16).  Stages on the e bits and the c bits run in registers, stages on the
 // low 5 bits of t run across lanes with __shfl_xor_sync, and stages on the
 // remaining bits of t (rows wider than one warp) run through a shared-memory
-// copy of the row in radix-8 rounds.  The 1/sqrt(d) scale, a and b are applied
-// when the row is written out.  Works for every power of two 8 <= d <= 32768
-// and every storage type; it is also the only family for fp32 storage.
+// copy of the row in radix-8 rounds.  Where the registers allow (up to 8 chunks
+// in the forward, 2 in the backward, which also carries dy and the da/db
+// accumulators) C is chosen so that a row stays inside ONE warp: d <= 2048 in the
+// forward, d <= 512 in the backward need no shared memory and no CTA barrier.
+// The 1/sqrt(d) scale, a and b are applied when the row is written out.  Works
+// for every power of two 8 <= d <= 32768 and every storage type; it is also the
+// only family for fp32 storage.
 #pragma once
 #include "wht_common.cuh"
 
+#ifndef WHT_BFLY_FWD_MAXC
+#define WHT_BFLY_FWD_MAXC 8
+#endif
+#ifndef WHT_BFLY_MIN_THREADS
+#define WHT_BFLY_MIN_THREADS 256
+#endif
+#ifndef WHT_BFLY_BWD_MAXC
+#define WHT_BFLY_BWD_MAXC 2
+#endif
+
 namespace wht {
 
-template <int LOGD>
+template <int LOGD, int MAXC>
 struct BflyGeo {
     static constexpr int D = 1 << LOGD;
-    static constexpr int C = imax_c(1, D / 8192);      // chunks of 8 per thread
+    // chunks of 8 per thread: D/256 of them put the whole row in ONE warp (no shared memory, no CTA
+    // barrier) -- used when MAXC (registers) allows; otherwise as few as keep the row within 1024
+    // threads (measured: between those two, more chunks per thread only cost occupancy)
+    static constexpr int C = (D >= 256 && D / 256 <= MAXC) ? D / 256 : imax_c(1, D / 8192);
     static constexpr int G = D / (8 * C);              // threads per row, 1..1024
     static constexpr int LOGG = ilog2_c(G);
-    static constexpr int THREADS = imax_c(G, 256);
+    static constexpr int THREADS = imax_c(G, WHT_BFLY_MIN_THREADS);
     static constexpr int R = THREADS / G;              // rows per CTA tile
     static constexpr int LANE_BITS = imin_c(5, LOGG);
     static constexpr int WARP_BITS = LOGG - LANE_BITS; // stages that cross warps
     static constexpr int SMEM_ROW_BYTES = D * 4;
     static constexpr int SMEM_FWD = WARP_BITS > 0 ? R * D * 4 : 0;
     static constexpr int SMEM_BWD = R * D * 4;
+    // few chunks per thread: little data in flight per thread, so the next tile's rows are
+    // requested before this tile's are transformed, and a / b stay in registers
+    static constexpr bool PREFETCH = C <= 2;
 };
+template <int LOGD> using BflyFwdGeo = BflyGeo<LOGD, WHT_BFLY_FWD_MAXC>;
+template <int LOGD> using BflyBwdGeo = BflyGeo<LOGD, WHT_BFLY_BWD_MAXC>;
 
 // One radix-2^NB round on row bits [P, P+NB) through shared memory.
-template <int LOGD, int P, int NB>
+template <typename Geo, int P, int NB>
 __device__ __forceinline__ void bfly_smem_round(float* srow, int t) {
-    using Geo = BflyGeo<LOGD>;
     constexpr int SETS = (8 * Geo::C) >> NB;
     constexpr int N = 1 << NB;
 #pragma unroll
@@ -58,26 +79,25 @@ __device__ __forceinline__ void bfly_smem_round(float* srow, int t) {
     }
 }
 
-template <int LOGD, int P, int REM>
+template <typename Geo, int P, int REM>
 struct BflyCrossRounds {
     static __device__ __forceinline__ void run(float* srow, int t) {
         constexpr int NB = imin_c(3, REM);
-        bfly_smem_round<LOGD, P, NB>(srow, t);
+        bfly_smem_round<Geo, P, NB>(srow, t);
         __syncthreads();
-        BflyCrossRounds<LOGD, P + NB, REM - NB>::run(srow, t);
+        BflyCrossRounds<Geo, P + NB, REM - NB>::run(srow, t);
     }
 };
-template <int LOGD, int P>
-struct BflyCrossRounds<LOGD, P, 0> {
+template <typename Geo, int P>
+struct BflyCrossRounds<Geo, P, 0> {
     static __device__ __forceinline__ void run(float*, int) {}
 };
 
 // Unnormalised H_d applied in place to the row held by one thread group.
 // Every thread of the CTA must call this (it contains __syncthreads when the
 // row spans several warps).
-template <int LOGD>
-__device__ __forceinline__ void bfly_row_transform(float (&v)[BflyGeo<LOGD>::C][8], float* srow, int t) {
-    using Geo = BflyGeo<LOGD>;
+template <typename Geo>
+__device__ __forceinline__ void bfly_row_transform(float (&v)[Geo::C][8], float* srow, int t) {
 #pragma unroll
     for (int c = 0; c < Geo::C; ++c) bfly8(v[c]);
     // chunk bits (the top log2 C bits of the row index)
@@ -117,7 +137,7 @@ __device__ __forceinline__ void bfly_row_transform(float (&v)[BflyGeo<LOGD>::C][
             dst[1] = make_float4(v[c][4], v[c][5], v[c][6], v[c][7]);
         }
         __syncthreads();
-        BflyCrossRounds<LOGD, 3 + Geo::LANE_BITS, Geo::WARP_BITS>::run(srow, t);
+        BflyCrossRounds<Geo, 3 + Geo::LANE_BITS, Geo::WARP_BITS>::run(srow, t);
 #pragma unroll
         for (int c = 0; c < Geo::C; ++c) {
             const float4* src = reinterpret_cast<const float4*>(srow + (c * Geo::G + t) * 8);
@@ -128,19 +148,37 @@ __device__ __forceinline__ void bfly_row_transform(float (&v)[BflyGeo<LOGD>::C][
     }
 }
 
-// Streaming row access: rows are touched once, so mark them evict-first.
-__device__ __forceinline__ void load8_stream(const float* p, float (&v)[8]) {
-    const float4 q0 = __ldcs(reinterpret_cast<const float4*>(p));
-    const float4 q1 = __ldcs(reinterpret_cast<const float4*>(p) + 1);
-    v[0] = q0.x; v[1] = q0.y; v[2] = q0.z; v[3] = q0.w;
-    v[4] = q1.x; v[5] = q1.y; v[6] = q1.z; v[7] = q1.w;
-}
-__device__ __forceinline__ void load8_stream(const __nv_bfloat16* p, float (&v)[8]) {
-    const uint4 q = __ldcs(reinterpret_cast<const uint4*>(p));
-    v[0] = bf16lo_to_f32(q.x); v[1] = bf16hi_to_f32(q.x);
-    v[2] = bf16lo_to_f32(q.y); v[3] = bf16hi_to_f32(q.y);
-    v[4] = bf16lo_to_f32(q.z); v[5] = bf16hi_to_f32(q.z);
-    v[6] = bf16lo_to_f32(q.w); v[7] = bf16hi_to_f32(q.w);
+// 8 contiguous row elements as loaded (bf16: one 128-bit word, fp32: two), widened on use.
+// Rows are touched once, so they are marked evict-first.
+template <typename TIO> struct Raw8;
+template <> struct Raw8<__nv_bfloat16> {
+    uint4 q;
+    __device__ __forceinline__ void load(const __nv_bfloat16* p) { q = __ldcs(reinterpret_cast<const uint4*>(p)); }
+    __device__ __forceinline__ void zero() { q = make_uint4(0u, 0u, 0u, 0u); }
+    __device__ __forceinline__ void widen(float (&v)[8]) const {
+        v[0] = bf16lo_to_f32(q.x); v[1] = bf16hi_to_f32(q.x);
+        v[2] = bf16lo_to_f32(q.y); v[3] = bf16hi_to_f32(q.y);
+        v[4] = bf16lo_to_f32(q.z); v[5] = bf16hi_to_f32(q.z);
+        v[6] = bf16lo_to_f32(q.w); v[7] = bf16hi_to_f32(q.w);
+    }
+};
+template <> struct Raw8<float> {
+    float4 q0, q1;
+    __device__ __forceinline__ void load(const float* p) {
+        q0 = __ldcs(reinterpret_cast<const float4*>(p));
+        q1 = __ldcs(reinterpret_cast<const float4*>(p) + 1);
+    }
+    __device__ __forceinline__ void zero() { q0 = q1 = make_float4(0.0f, 0.0f, 0.0f, 0.0f); }
+    __device__ __forceinline__ void widen(float (&v)[8]) const {
+        v[0] = q0.x; v[1] = q0.y; v[2] = q0.z; v[3] = q0.w;
+        v[4] = q1.x; v[5] = q1.y; v[6] = q1.z; v[7] = q1.w;
+    }
+};
+template <typename TIO>
+__device__ __forceinline__ void load8_stream(const TIO* p, float (&v)[8]) {
+    Raw8<TIO> r;
+    r.load(p);
+    r.widen(v);
 }
 __device__ __forceinline__ void store8_stream(float* p, const float (&v)[8]) {
     __stcs(reinterpret_cast<float4*>(p), make_float4(v[0], v[1], v[2], v[3]));
@@ -155,46 +193,70 @@ __device__ __forceinline__ void store8_stream(__nv_bfloat16* p, const float (&v)
     __stcs(reinterpret_cast<uint4*>(p), q);
 }
 
+// The C chunks of one thread's share of a row, as loaded (zeros for a row past the end).
+template <typename Geo, typename TIO>
+__device__ __forceinline__ void bfly_load_row(const TIO* base, long long row, long long T, long long ld, int t,
+                                              Raw8<TIO> (&raw)[Geo::C]) {
+#pragma unroll
+    for (int c = 0; c < Geo::C; ++c) {
+        if (row < T) raw[c].load(base + row * ld + (c * Geo::G + t) * 8);
+        else raw[c].zero();
+    }
+}
+
 // ---- forward: y = a (.) (x H)/sqrt(d) + b ------------------------------------
 template <int LOGD, typename TIO, typename TP>
-__global__ void __launch_bounds__(BflyGeo<LOGD>::THREADS)
+__global__ void __launch_bounds__(BflyFwdGeo<LOGD>::THREADS)
 bfly_fwd_kernel(const TIO* x, const TP* __restrict__ a, const TP* __restrict__ b, const TIO* resid, TIO* y,
                 long long T, long long ld, float inv_sqrt_d) {  // ld: elements between consecutive rows (>= D)
-    using Geo = BflyGeo<LOGD>;
+    using Geo = BflyFwdGeo<LOGD>;
     extern __shared__ __align__(16) float smem[];
     const int rg = threadIdx.x / Geo::G;  // row group inside the CTA
     const int t = threadIdx.x % Geo::G;
     float* srow = smem + (Geo::WARP_BITS > 0 ? rg * Geo::D : 0);
 
-    float as[Geo::C][8], bs[Geo::C][8];
+    constexpr int PC = Geo::PREFETCH ? Geo::C : 1;  // a, b in registers only when a thread has few channels
+    float as[PC][8], bs[PC][8];
+    if constexpr (Geo::PREFETCH) {
 #pragma unroll
-    for (int c = 0; c < Geo::C; ++c) {
-        load8(a + (c * Geo::G + t) * 8, as[c]);
-        load8(b + (c * Geo::G + t) * 8, bs[c]);
+        for (int c = 0; c < Geo::C; ++c) {
+            load8(a + (c * Geo::G + t) * 8, as[c]);
+            load8(b + (c * Geo::G + t) * 8, bs[c]);
 #pragma unroll
-        for (int e = 0; e < 8; ++e) as[c][e] *= inv_sqrt_d;
+            for (int e = 0; e < 8; ++e) as[c][e] *= inv_sqrt_d;
+        }
     }
 
     const long long tiles = (T + Geo::R - 1) / Geo::R;
+    Raw8<TIO> raw[Geo::C];
+    if constexpr (Geo::PREFETCH) {
+        if (blockIdx.x < tiles) bfly_load_row<Geo, TIO>(x, blockIdx.x * static_cast<long long>(Geo::R) + rg, T, ld, t, raw);
+    }
     for (long long tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
         const long long row = tile * Geo::R + rg;
         const bool valid = row < T;
+        if constexpr (!Geo::PREFETCH) bfly_load_row<Geo, TIO>(x, row, T, ld, t, raw);
         float v[Geo::C][8];
 #pragma unroll
-        for (int c = 0; c < Geo::C; ++c) {
-            if (valid) {
-                load8_stream(x + row * ld + (c * Geo::G + t) * 8, v[c]);
-            } else {
-#pragma unroll
-                for (int e = 0; e < 8; ++e) v[c][e] = 0.0f;
-            }
+        for (int c = 0; c < Geo::C; ++c) raw[c].widen(v[c]);
+        if constexpr (Geo::PREFETCH) {
+            const long long next = tile + gridDim.x;
+            if (next < tiles) bfly_load_row<Geo, TIO>(x, next * Geo::R + rg, T, ld, t, raw);
         }
-        bfly_row_transform<LOGD>(v, srow, t);
+        bfly_row_transform<Geo>(v, srow, t);
         if (valid) {
 #pragma unroll
             for (int c = 0; c < Geo::C; ++c) {
+                if constexpr (Geo::PREFETCH) {
 #pragma unroll
-                for (int e = 0; e < 8; ++e) v[c][e] = fmaf(v[c][e], as[c][e], bs[c][e]);
+                    for (int e = 0; e < 8; ++e) v[c][e] = fmaf(v[c][e], as[c][e], bs[c][e]);
+                } else {
+                    float av[8], bv[8];  // L1-resident after the first tile
+                    load8(a + (c * Geo::G + t) * 8, av);
+                    load8(b + (c * Geo::G + t) * 8, bv);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) v[c][e] = fmaf(v[c][e], av[e] * inv_sqrt_d, bv[e]);
+                }
                 if (resid != nullptr) {  // fused residual: summed in fp32, rounded once at the store
                     float r[8];
                     load8_stream(resid + row * ld + (c * Geo::G + t) * 8, r);
@@ -211,10 +273,10 @@ bfly_fwd_kernel(const TIO* x, const TP* __restrict__ a, const TP* __restrict__ b
 // partials layout: [gridDim.x][2][D] fp32; slot 0 holds sum_t dy (.) (x H) WITHOUT
 // the 1/sqrt(d) factor (the finalize pass applies it), slot 1 holds sum_t dy.
 template <int LOGD, typename TIO, typename TP>
-__global__ void __launch_bounds__(BflyGeo<LOGD>::THREADS)
+__global__ void __launch_bounds__(BflyBwdGeo<LOGD>::THREADS)
 bfly_bwd_kernel(const TIO* dy, const TIO* x, const TP* __restrict__ a, TIO* dx,
                 float* __restrict__ partials, long long T, long long ld, float inv_sqrt_d) {
-    using Geo = BflyGeo<LOGD>;
+    using Geo = BflyBwdGeo<LOGD>;
     extern __shared__ __align__(16) float smem[];
     const int rg = threadIdx.x / Geo::G;
     const int t = threadIdx.x % Geo::G;
@@ -228,21 +290,32 @@ bfly_bwd_kernel(const TIO* dy, const TIO* x, const TP* __restrict__ a, TIO* dx,
     }
 
     const long long tiles = (T + Geo::R - 1) / Geo::R;
+    Raw8<TIO> rx[Geo::C], rdy[Geo::C];
+    if constexpr (Geo::PREFETCH) {
+        if (blockIdx.x < tiles) {
+            const long long row0 = blockIdx.x * static_cast<long long>(Geo::R) + rg;
+            bfly_load_row<Geo, TIO>(x, row0, T, ld, t, rx);
+            bfly_load_row<Geo, TIO>(dy, row0, T, ld, t, rdy);
+        }
+    }
     for (long long tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
         const long long row = tile * Geo::R + rg;
         const bool valid = row < T;
+        if constexpr (!Geo::PREFETCH) {
+            bfly_load_row<Geo, TIO>(x, row, T, ld, t, rx);
+            bfly_load_row<Geo, TIO>(dy, row, T, ld, t, rdy);
+        }
         float v[Geo::C][8], w[Geo::C][8];
 #pragma unroll
-        for (int c = 0; c < Geo::C; ++c) {
-            if (valid) {
-                load8_stream(x + row * ld + (c * Geo::G + t) * 8, v[c]);
-                load8_stream(dy + row * ld + (c * Geo::G + t) * 8, w[c]);
-            } else {
-#pragma unroll
-                for (int e = 0; e < 8; ++e) { v[c][e] = 0.0f; w[c][e] = 0.0f; }
+        for (int c = 0; c < Geo::C; ++c) { rx[c].widen(v[c]); rdy[c].widen(w[c]); }
+        if constexpr (Geo::PREFETCH) {
+            const long long next = tile + gridDim.x;
+            if (next < tiles) {
+                bfly_load_row<Geo, TIO>(x, next * Geo::R + rg, T, ld, t, rx);
+                bfly_load_row<Geo, TIO>(dy, next * Geo::R + rg, T, ld, t, rdy);
             }
         }
-        bfly_row_transform<LOGD>(v, srow, t);  // v = x H (unnormalised)
+        bfly_row_transform<Geo>(v, srow, t);  // v = x H (unnormalised)
 #pragma unroll
         for (int c = 0; c < Geo::C; ++c) {
             float as[8];
@@ -255,7 +328,7 @@ bfly_bwd_kernel(const TIO* dy, const TIO* x, const TP* __restrict__ a, TIO* dx,
             }
         }
         if constexpr (Geo::WARP_BITS > 0) __syncthreads();  // srow is reused by the second transform
-        bfly_row_transform<LOGD>(v, srow, t);  // v = (a (.) dy) H
+        bfly_row_transform<Geo>(v, srow, t);  // v = (a (.) dy) H
         if (valid) {
 #pragma unroll
             for (int c = 0; c < Geo::C; ++c) {

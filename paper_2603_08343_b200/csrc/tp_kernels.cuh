@@ -25,38 +25,13 @@ struct TpParts {
     const void* p[kTpMaxRanks];
 };
 
-// 8 contiguous elements as loaded (bf16: one 128-bit word, fp32: two), widened on use
-template <typename TIO> struct Raw8;
-template <> struct Raw8<__nv_bfloat16> {
-    uint4 q;
-    __device__ __forceinline__ void load(const __nv_bfloat16* p) { q = __ldcs(reinterpret_cast<const uint4*>(p)); }
-    __device__ __forceinline__ void widen(float (&v)[8]) const {
-        v[0] = bf16lo_to_f32(q.x); v[1] = bf16hi_to_f32(q.x);
-        v[2] = bf16lo_to_f32(q.y); v[3] = bf16hi_to_f32(q.y);
-        v[4] = bf16lo_to_f32(q.z); v[5] = bf16hi_to_f32(q.z);
-        v[6] = bf16lo_to_f32(q.w); v[7] = bf16hi_to_f32(q.w);
-    }
-};
-template <> struct Raw8<float> {
-    float4 q0, q1;
-    __device__ __forceinline__ void load(const float* p) {
-        q0 = __ldcs(reinterpret_cast<const float4*>(p));
-        q1 = __ldcs(reinterpret_cast<const float4*>(p) + 1);
-    }
-    __device__ __forceinline__ void widen(float (&v)[8]) const {
-        v[0] = q0.x; v[1] = q0.y; v[2] = q0.z; v[3] = q0.w;
-        v[4] = q1.x; v[5] = q1.y; v[6] = q1.z; v[7] = q1.w;
-    }
-};
-
 // Sources are fetched kTpBatch at a time: all loads of a batch are issued before the first use.
 constexpr int kTpBatch = 4;
 
 // v = sum_s sign_s * part_s[row, chunk], summed in rank order
-template <int LOGW, typename TIO>
+template <typename Geo, typename TIO>
 __device__ __forceinline__ void tp_load_signed_sum(const TpParts& parts, int g, unsigned neg_mask, long long row,
-                                                   int t, float (&v)[BflyGeo<LOGW>::C][8]) {
-    using Geo = BflyGeo<LOGW>;
+                                                   int t, float (&v)[Geo::C][8]) {
 #pragma unroll
     for (int c = 0; c < Geo::C; ++c) {
         const long long off = row * Geo::D + (c * Geo::G + t) * 8;
@@ -85,22 +60,25 @@ __device__ __forceinline__ void tp_load_signed_sum(const TpParts& parts, int g, 
 }
 
 template <int LOGW, typename TIO, typename TP>
-__global__ void __launch_bounds__(BflyGeo<LOGW>::THREADS)
+__global__ void __launch_bounds__(BflyFwdGeo<LOGW>::THREADS)
 bfly_fwd_tp_kernel(TpParts xs, int g, unsigned neg_mask, const TP* __restrict__ a, const TP* __restrict__ b, TIO* y,
                    long long T, float inv_sqrt_d) {
-    using Geo = BflyGeo<LOGW>;
+    using Geo = BflyFwdGeo<LOGW>;
     extern __shared__ __align__(16) float smem[];
     const int rg = threadIdx.x / Geo::G;
     const int t = threadIdx.x % Geo::G;
     float* srow = smem + (Geo::WARP_BITS > 0 ? rg * Geo::D : 0);
 
-    float as[Geo::C][8], bs[Geo::C][8];
+    constexpr int PC = Geo::PREFETCH ? Geo::C : 1;  // a, b in registers only when a thread has few channels
+    float as[PC][8], bs[PC][8];
+    if constexpr (Geo::PREFETCH) {
 #pragma unroll
-    for (int c = 0; c < Geo::C; ++c) {
-        load8(a + (c * Geo::G + t) * 8, as[c]);
-        load8(b + (c * Geo::G + t) * 8, bs[c]);
+        for (int c = 0; c < Geo::C; ++c) {
+            load8(a + (c * Geo::G + t) * 8, as[c]);
+            load8(b + (c * Geo::G + t) * 8, bs[c]);
 #pragma unroll
-        for (int e = 0; e < 8; ++e) as[c][e] *= inv_sqrt_d;
+            for (int e = 0; e < 8; ++e) as[c][e] *= inv_sqrt_d;
+        }
     }
 
     const long long tiles = (T + Geo::R - 1) / Geo::R;
@@ -109,19 +87,27 @@ bfly_fwd_tp_kernel(TpParts xs, int g, unsigned neg_mask, const TP* __restrict__ 
         const bool valid = row < T;
         float v[Geo::C][8];
         if (valid) {
-            tp_load_signed_sum<LOGW, TIO>(xs, g, neg_mask, row, t, v);
+            tp_load_signed_sum<Geo, TIO>(xs, g, neg_mask, row, t, v);
         } else {
 #pragma unroll
             for (int c = 0; c < Geo::C; ++c)
 #pragma unroll
                 for (int e = 0; e < 8; ++e) v[c][e] = 0.0f;
         }
-        bfly_row_transform<LOGW>(v, srow, t);
+        bfly_row_transform<Geo>(v, srow, t);
         if (valid) {
 #pragma unroll
             for (int c = 0; c < Geo::C; ++c) {
+                if constexpr (Geo::PREFETCH) {
 #pragma unroll
-                for (int e = 0; e < 8; ++e) v[c][e] = fmaf(v[c][e], as[c][e], bs[c][e]);
+                    for (int e = 0; e < 8; ++e) v[c][e] = fmaf(v[c][e], as[c][e], bs[c][e]);
+                } else {
+                    float av[8], bv[8];  // L1-resident after the first tile
+                    load8(a + (c * Geo::G + t) * 8, av);
+                    load8(b + (c * Geo::G + t) * 8, bv);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) v[c][e] = fmaf(v[c][e], av[e] * inv_sqrt_d, bv[e]);
+                }
                 store8_stream(y + row * Geo::D + (c * Geo::G + t) * 8, v[c]);
             }
         }
@@ -130,10 +116,10 @@ bfly_fwd_tp_kernel(TpParts xs, int g, unsigned neg_mask, const TP* __restrict__ 
 
 // partials layout as in bfly_bwd_kernel: [gridDim.x][2][W], slot 0 without the 1/sqrt(d) factor.
 template <int LOGW, typename TIO, typename TP>
-__global__ void __launch_bounds__(BflyGeo<LOGW>::THREADS)
+__global__ void __launch_bounds__(BflyBwdGeo<LOGW>::THREADS)
 bfly_bwd_tp_kernel(TpParts dys, TpParts xs, TpParts as, int g, int r, unsigned neg_mask, TIO* dx,
                    float* __restrict__ partials, long long T, float inv_sqrt_d) {
-    using Geo = BflyGeo<LOGW>;
+    using Geo = BflyBwdGeo<LOGW>;
     extern __shared__ __align__(16) float smem[];
     const int rg = threadIdx.x / Geo::G;
     const int t = threadIdx.x % Geo::G;
@@ -152,14 +138,14 @@ bfly_bwd_tp_kernel(TpParts dys, TpParts xs, TpParts as, int g, int r, unsigned n
         const bool valid = row < T;
         float v[Geo::C][8];
         if (valid) {
-            tp_load_signed_sum<LOGW, TIO>(xs, g, neg_mask, row, t, v);
+            tp_load_signed_sum<Geo, TIO>(xs, g, neg_mask, row, t, v);
         } else {
 #pragma unroll
             for (int c = 0; c < Geo::C; ++c)
 #pragma unroll
                 for (int e = 0; e < 8; ++e) v[c][e] = 0.0f;
         }
-        bfly_row_transform<LOGW>(v, srow, t);  // v = (sum_s +-x_s) H_w, unnormalised
+        bfly_row_transform<Geo>(v, srow, t);  // v = (sum_s +-x_s) H_w, unnormalised
         // v <- sum_s +- a_s (.) dy_s; this rank's own dy block also feeds da, db
 #pragma unroll
         for (int c = 0; c < Geo::C; ++c) {
@@ -202,7 +188,7 @@ bfly_bwd_tp_kernel(TpParts dys, TpParts xs, TpParts as, int g, int r, unsigned n
             for (int e = 0; e < 8; ++e) v[c][e] = gsum[e];
         }
         if constexpr (Geo::WARP_BITS > 0) __syncthreads();  // srow is reused by the second transform
-        bfly_row_transform<LOGW>(v, srow, t);
+        bfly_row_transform<Geo>(v, srow, t);
         if (valid) {
 #pragma unroll
             for (int c = 0; c < Geo::C; ++c) {

@@ -189,7 +189,7 @@ int capped_grid(int64_t tiles, int sms, int per_sm) {
 // ------------------------------------------------------------------ butterfly family
 template <int LOGD, typename TIO, typename TP>
 int launch_bfly_fwd(const FwdArgs& f, const Ctx& c) {
-    using Geo = BflyGeo<LOGD>;
+    using Geo = BflyFwdGeo<LOGD>;
     static int occ[kMaxDevices] = {};
     auto kernel = bfly_fwd_kernel<LOGD, TIO, TP>;
     const int per_sm = resident_ctas(kernel, Geo::THREADS, Geo::SMEM_FWD, c.dev, occ);
@@ -205,7 +205,7 @@ int launch_bfly_fwd(const FwdArgs& f, const Ctx& c) {
 
 template <int LOGD, typename TIO, typename TP>
 int launch_bfly_bwd(const BwdArgs& g, const Ctx& c) {
-    using Geo = BflyGeo<LOGD>;
+    using Geo = BflyBwdGeo<LOGD>;
     static int occ[kMaxDevices] = {};
     auto kernel = bfly_bwd_kernel<LOGD, TIO, TP>;
     const int per_sm = resident_ctas(kernel, Geo::THREADS, Geo::SMEM_BWD, c.dev, occ);
@@ -553,7 +553,7 @@ struct TpCall {
 
 template <int LOGW, typename TIO, typename TP>
 int launch_bfly_fwd_tp(const TpCall& t, const FwdArgs& f, const Ctx& c) {
-    using Geo = BflyGeo<LOGW>;
+    using Geo = BflyFwdGeo<LOGW>;
     static int occ[kMaxDevices] = {};
     auto kernel = bfly_fwd_tp_kernel<LOGW, TIO, TP>;
     const int per_sm = resident_ctas(kernel, Geo::THREADS, Geo::SMEM_FWD, c.dev, occ);
@@ -568,7 +568,7 @@ int launch_bfly_fwd_tp(const TpCall& t, const FwdArgs& f, const Ctx& c) {
 
 template <int LOGW, typename TIO, typename TP>
 int launch_bfly_bwd_tp(const TpCall& t, const BwdArgs& g, const Ctx& c) {
-    using Geo = BflyGeo<LOGW>;
+    using Geo = BflyBwdGeo<LOGW>;
     static int occ[kMaxDevices] = {};
     auto kernel = bfly_bwd_tp_kernel<LOGW, TIO, TP>;
     const int per_sm = resident_ctas(kernel, Geo::THREADS, Geo::SMEM_BWD, c.dev, occ);
