@@ -199,7 +199,10 @@ size_t wht_affine_bwd_grouped_workspace_bytes(int64_t T, int32_t d, int32_t bloc
  * any rank launches (a barrier across ranks on the host or stream), and that no rank overwrites its
  * inputs before every rank's call has completed.  Gradients of a and b need no reduction across the
  * g ranks (each rank owns its channels); across data-parallel replicas they add as usual.
- * Butterfly kernels; every storage type.  The backward takes caller-owned scratch of at least
+ * Every storage type.  Forward of bf16 rows with 1024 <= w <= 4096 and T*w >= 4 Mi elements: tcgen05
+ * kernel (each source block's tile is bulk-copied into shared memory and multiplied by H_128 into one
+ * accumulator, negated where the sign is -1); otherwise, and for the backward, butterfly kernels with
+ * multi-source loads.  The backward takes caller-owned scratch of at least
  * wht_affine_bwd_tp_workspace_bytes(T, w, g, dtype) bytes and never allocates.
  * Errors as for the plain calls; g or r out of range -> WHT_ERR_BAD_DIM.
  */

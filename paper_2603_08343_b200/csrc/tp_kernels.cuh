@@ -19,12 +19,6 @@
 
 namespace wht {
 
-constexpr int kTpMaxRanks = 8;
-
-struct TpParts {
-    const void* p[kTpMaxRanks];
-};
-
 // Sources are fetched kTpBatch at a time: all loads of a batch are issued before the first use.
 constexpr int kTpBatch = 4;
 

@@ -37,7 +37,8 @@
 // flag and the device status word; every role then leaves its loop, copies in flight
 // are waited for (bounded), TMEM is freed and the kernel returns: a fault in the
 // pipeline shows up as WHT_ERR_DEVICE_WAIT on the host, never as a hang.
-// No copy uses cluster multicast; every source is this GPU's own memory.
+// No copy uses cluster multicast; every source is this GPU's own memory, except in the
+// column-sharded forward, whose source blocks may be peer mappings.
 #pragma once
 #include "mma_pipe_kernels.cuh"
 
@@ -169,6 +170,9 @@ __host__ __device__ constexpr uint32_t umma_idesc(int n) {
            (static_cast<uint32_t>(128 >> 4) << 24);
 }
 
+// Instruction-descriptor bit that multiplies by -A instead of A.
+constexpr int kUmmaNegateABit = 13;
+
 template <int LOGD, int NCOL_>
 struct UmmaGeo {
     static constexpr int D = 1 << LOGD;
@@ -269,10 +273,21 @@ __device__ __forceinline__ void stage_params_umma(const TP* __restrict__ src, fl
 
 // RES: y = resid + (a (.) (x H)/sqrt(d) + b), the residual read in the store layout (each thread
 // its own 16-byte chunks, fetched before the accumulator is waited for).
-template <int LOGD, int NCOL, int STAGES, typename TP, bool RES>
+//
+// MULTI (column-sharded form): the rows come as nsrc blocks of D channels, one per rank, and the
+// transform input is their signed sum, sign H_g[s][r].  Each block's tile is copied into a ring slot
+// of its own (from this GPU's memory or through a peer mapping; plain bulk copies, never multicast)
+// and multiplied by H_128 into the SAME accumulator, with the instruction descriptor's negate-A bit
+// set for the blocks whose sign is -1: the signed sum happens in the tensor core's fp32 accumulation
+// of exact +-1 products, and the epilogue is the ordinary one.  inv_sqrt_d is then 1/sqrt(nsrc * D).
+template <int LOGD, int NCOL, int STAGES, typename TP, bool RES, bool MULTI = false>
 __global__ void __launch_bounds__(UmmaGeo<LOGD, NCOL>::THREADS, 1)
 umma_fwd_kernel(const __nv_bfloat16* x, const TP* __restrict__ a, const TP* __restrict__ b,
-                const __nv_bfloat16* resid, __nv_bfloat16* y, long long T, float inv_sqrt_d) {
+                const __nv_bfloat16* resid, __nv_bfloat16* y, long long T, float inv_sqrt_d,
+                const __grid_constant__ TpParts parts,
+                int nsrc_arg, unsigned neg_mask) {
+    static_assert(!(RES && MULTI), "the column-sharded form has no fused residual");
+    const int nsrc = MULTI ? nsrc_arg : 1;
     using Geo = UmmaGeo<LOGD, NCOL>;
     using L = UmmaFwdSmem<LOGD, NCOL, STAGES, TP, RES>;
     constexpr int ACC = L::ACC;
@@ -335,43 +350,52 @@ umma_fwd_kernel(const __nv_bfloat16* x, const TP* __restrict__ a, const TP* __re
     if (warp == 0) {
         if (lane == 0) {
             const uint64_t stream_policy = l2_policy_evict_first();
-            long long it = 0;
-            for (; it < my_tiles; ++it) {
-                const int s = static_cast<int>(it % STAGES);
-                const uint32_t ph = static_cast<uint32_t>(it / STAGES) & 1u;
-                if (!wait_or_abort(empty + s, ph ^ 1u, abort_flag)) break;
+            long long j = 0;  // ring slots filled so far: one per tile and source block
+            bool ok = true;
+            for (long long it = 0; ok && it < my_tiles; ++it) {
                 const long long tile = blockIdx.x + it * gridDim.x;
                 const long long row0 = tile * Geo::ROWS;
                 const long long rows = T - row0 < Geo::ROWS ? T - row0 : Geo::ROWS;
                 const uint32_t bytes = static_cast<uint32_t>(rows) * Geo::D * 2;
-                mbar_expect_tx(full + s, bytes);
-                bulk_load_stream(ring + s * Geo::TILE_BYTES, x + row0 * Geo::D, bytes, full + s, stream_policy);
+                for (int src = 0; src < nsrc; ++src, ++j) {
+                    const int s = static_cast<int>(j % STAGES);
+                    const uint32_t ph = static_cast<uint32_t>(j / STAGES) & 1u;
+                    if (!wait_or_abort(empty + s, ph ^ 1u, abort_flag)) { ok = false; break; }
+                    const __nv_bfloat16* from = MULTI ? static_cast<const __nv_bfloat16*>(parts.p[src]) : x;
+                    mbar_expect_tx(full + s, bytes);
+                    bulk_load_stream(ring + s * Geo::TILE_BYTES, from + row0 * Geo::D, bytes, full + s, stream_policy);
+                }
             }
             if (*abort_flag) {
                 // copies already issued still land in shared memory: wait for them before leaving
-                const long long lo = it > STAGES ? it - STAGES : 0;
-                for (long long j = lo; j < it; ++j)
-                    mbar_wait_bounded(full + (j % STAGES), static_cast<uint32_t>(j / STAGES) & 1u);
+                const long long lo = j > STAGES ? j - STAGES : 0;
+                for (long long k = lo; k < j; ++k)
+                    mbar_wait_bounded(full + (k % STAGES), static_cast<uint32_t>(k / STAGES) & 1u);
             }
         }
     } else if (warp == 1) {
         if (lane == 0) {
             const uint64_t adesc = umma_smem_desc(smem_u32(smem_raw + L::OFF_H));
             constexpr uint32_t idesc = umma_idesc(Geo::N);
-            for (long long it = 0; it < my_tiles; ++it) {
-                const int s = static_cast<int>(it % STAGES);
-                const uint32_t ph = static_cast<uint32_t>(it / STAGES) & 1u;
+            long long j = 0;
+            bool ok = true;
+            for (long long it = 0; ok && it < my_tiles; ++it) {
                 const int t = static_cast<int>(it % ACC);
                 const uint32_t pt = static_cast<uint32_t>(it / ACC) & 1u;
-                if (!wait_or_abort(full + s, ph, abort_flag)) break;
-                if (!wait_or_abort(acc_empty + t, pt ^ 1u, abort_flag)) break;
-                tc_fence_after();
-                const uint64_t bdesc = umma_smem_desc(smem_u32(ring + s * Geo::TILE_BYTES));
+                for (int src = 0; src < nsrc; ++src, ++j) {
+                    const int s = static_cast<int>(j % STAGES);
+                    const uint32_t ph = static_cast<uint32_t>(j / STAGES) & 1u;
+                    if (!wait_or_abort(full + s, ph, abort_flag)) { ok = false; break; }
+                    if (src == 0 && !wait_or_abort(acc_empty + t, pt ^ 1u, abort_flag)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint64_t bdesc = umma_smem_desc(smem_u32(ring + s * Geo::TILE_BYTES));
+                    const uint32_t idesc_s = MULTI ? (idesc | (((neg_mask >> src) & 1u) << kUmmaNegateABit)) : idesc;
 #pragma unroll
-                for (int k = 0; k < 8; ++k)  // K = 16 per instruction: 256 bytes further in both operands
-                    umma_bf16(tmem_base + t * Geo::N, adesc + k * 16, bdesc + k * 16, idesc, k > 0);
-                umma_commit(acc_full + t);
-                umma_commit(empty + s);
+                    for (int k = 0; k < 8; ++k)  // K = 16 per instruction: 256 bytes further in both operands
+                        umma_bf16(tmem_base + t * Geo::N, adesc + k * 16, bdesc + k * 16, idesc_s, (src | k) != 0);
+                    if (src == nsrc - 1) umma_commit(acc_full + t);
+                    umma_commit(empty + s);
+                }
             }
         }
     } else {

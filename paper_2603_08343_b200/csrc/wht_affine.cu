@@ -388,7 +388,7 @@ int launch_umma_fwd_impl(const FwdArgs& f, const Ctx& c) {
     launch_overlapped(kernel, grid, Geo::THREADS, L::BYTES, c.stream,
                       static_cast<const __nv_bfloat16*>(f.x), static_cast<const TP*>(f.a), static_cast<const TP*>(f.b),
                       static_cast<const __nv_bfloat16*>(f.resid), static_cast<__nv_bfloat16*>(f.y),
-                      static_cast<long long>(c.T), inv_sqrt(Geo::D));
+                      static_cast<long long>(c.T), inv_sqrt(Geo::D), TpParts{}, 1, 0u);
     WHT_CUDA_TRY(cudaGetLastError());
     return WHT_OK;
 }
@@ -582,6 +582,37 @@ int launch_bfly_bwd_tp(const TpCall& t, const BwdArgs& g, const Ctx& c) {
                                                                  static_cast<long long>(c.T), t.scale);
         },
         t.scale);
+}
+
+// tcgen05 form of the column-sharded forward: one product per source block into one accumulator
+template <int LOGW, typename TP>
+int launch_umma_fwd_tp(const TpCall& t, const FwdArgs& f, const Ctx& c) {
+    constexpr int NCOL = 128, STAGES = 4;
+    using Geo = UmmaGeo<LOGW, NCOL>;
+    using L = UmmaFwdSmem<LOGW, NCOL, STAGES, TP, false>;
+    static_assert(L::BYTES > 116 * 1024, "must be alone on its SM");
+    static_assert(!L::SPLIT, "widths handled here keep every channel of a row in one thread group");
+    static int ready[kMaxDevices] = {};
+    auto kernel = umma_fwd_kernel<LOGW, NCOL, STAGES, TP, false, true>;
+    int rc = prepare_umma(kernel, L::BYTES, c.dev, ready);
+    if (rc != WHT_OK) return rc;
+    const int grid = capped_grid(ceil_div(c.T, Geo::ROWS), c.sms, 1);
+    launch_overlapped(kernel, grid, Geo::THREADS, L::BYTES, c.stream, static_cast<const __nv_bfloat16*>(nullptr),
+                      static_cast<const TP*>(f.a), static_cast<const TP*>(f.b),
+                      static_cast<const __nv_bfloat16*>(nullptr), static_cast<__nv_bfloat16*>(f.y),
+                      static_cast<long long>(c.T), t.scale, t.xs, t.g, t.neg_mask);
+    WHT_CUDA_TRY(cudaGetLastError());
+    return WHT_OK;
+}
+
+template <typename TP>
+int dispatch_umma_fwd_tp(int logw, const TpCall& t, const FwdArgs& f, const Ctx& c) {
+    switch (logw) {
+        case 10: return launch_umma_fwd_tp<10, TP>(t, f, c);
+        case 11: return launch_umma_fwd_tp<11, TP>(t, f, c);
+        case 12: return launch_umma_fwd_tp<12, TP>(t, f, c);
+    }
+    return WHT_ERR_BAD_DIM;
 }
 
 template <typename TIO, typename TP>
@@ -863,6 +894,12 @@ int wht_affine_fwd_tp(const void* const* x_parts, const void* a, const void* b, 
     if (rc != WHT_OK) return rc;
     const FwdArgs f{nullptr, a, b, y};
     const int logw = log2_of(w);
+    // bf16 rows of 1024 ... 4096 channels per rank with enough rows for 32 KiB tiles: tcgen05 form
+    if (dtype != WHT_F32 && logw >= 10 && logw <= 12 && (g_variant == 0 || g_variant == 4) &&
+        (g_variant == 4 || enough_work_for_tiles(T, w))) {
+        return dtype == WHT_BF16 ? dispatch_umma_fwd_tp<__nv_bfloat16>(logw, t, f, c)
+                                 : dispatch_umma_fwd_tp<float>(logw, t, f, c);
+    }
     switch (dtype) {
         case WHT_F32: return dispatch_bfly_fwd_tp<float, float>(logw, t, f, c);
         case WHT_BF16: return dispatch_bfly_fwd_tp<__nv_bfloat16, __nv_bfloat16>(logw, t, f, c);

@@ -74,6 +74,12 @@ __device__ __forceinline__ void grid_launch_dependents() {
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 }
 
+// Column-sharded (tensor-parallel) calls: one device pointer per rank's block.
+constexpr int kTpMaxRanks = 8;
+struct TpParts {
+    const void* p[kTpMaxRanks];
+};
+
 constexpr __host__ __device__ int ilog2_c(int v) { return v <= 1 ? 0 : 1 + ilog2_c(v >> 1); }
 constexpr __host__ __device__ int imin_c(int a, int b) { return a < b ? a : b; }
 constexpr __host__ __device__ int imax_c(int a, int b) { return a > b ? a : b; }

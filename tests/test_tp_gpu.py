@@ -19,6 +19,7 @@ def B():
     build.build()
     from paper_2603_08343_b200 import binding
     yield binding
+    binding.wht_affine_set_variant(0)
     binding.wht_affine_device_status()
 
 
@@ -30,8 +31,18 @@ CASES = [
 ]
 
 
-@pytest.mark.parametrize("g,w,dtype,T", CASES)
-def test_column_sharded_calls_match_the_full_width_oracle(B, g, w, dtype, T):
+# the tcgen05 form of the forward (one product per source block, signs by the negate-A bit): forced by
+# variant 4 on small cases, and chosen by itself once T*w reaches 4 Mi elements
+UMMA_CASES = [
+    (2, 1024, wl.WHT_BF16, 300, 4), (8, 1024, wl.WHT_BF16_PF32, 65, 4), (4, 2048, wl.WHT_BF16_PF32, 1111, 4),
+    (2, 4096, wl.WHT_BF16, 19, 4), (8, 2048, wl.WHT_BF16, 7, 4), (4, 4096, wl.WHT_BF16_PF32, 130, 4),
+    (2, 1024, wl.WHT_BF16_PF32, 4100, 0), (1, 1024, wl.WHT_BF16, 129, 4),
+]
+
+
+@pytest.mark.parametrize("g,w,dtype,T,variant", [c + (0,) for c in CASES] + UMMA_CASES)
+def test_column_sharded_calls_match_the_full_width_oracle(B, g, w, dtype, T, variant):
+    B.wht_affine_set_variant(variant)
     d = g * w
     wk = wl.Workload("tp", T, d, dtype, "normal", 900 + d + g, True, "")
     x, dy = wl.gen_full(wk, "x"), wl.gen_full(wk, "dy")
@@ -60,10 +71,10 @@ def test_column_sharded_calls_match_the_full_width_oracle(B, g, w, dtype, T):
         assert_rows_bf16(to_f64(dx), ref_dx, "tp dx")
     assert_grad_vec(to_f64(da), ref_da, "tp da")
     assert_grad_vec(to_f64(db), ref_db, "tp db")
-    if g == 1:  # one rank is the plain call (butterfly family)
-        B.wht_affine_set_variant(1)
+    if g == 1:  # one rank is the plain call of the same kernel family
+        B.wht_affine_set_variant(variant or 1)
         assert torch.equal(ys[0], B.forward(xs[0], as_[0], bs[0]))
-        B.wht_affine_set_variant(0)
+    B.wht_affine_set_variant(0)
 
 
 def test_blocks_given_as_addresses_and_repeat_calls_are_bit_identical(B):
