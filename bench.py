@@ -300,6 +300,65 @@ def section_paper_shapes(B, hbm_peak):
     return out
 
 
+def section_tensor_parallel_local(B, hbm_peak):
+    """Column-sharded calls of ONE rank with every rank's block in this GPU's memory (the kernels read the
+    blocks through a pointer table; on several GPUs the other entries are peer mappings and the NVLink
+    transfer, not the kernel, sets the time).  Bytes: (g+1) blocks forward, (2g+1) backward."""
+    from paper_2603_08343_b200 import tp
+    out = {}
+    for g, w_, T in ((2, 1024, 65536), (8, 1024, 16384), (8, 256, 65536)):
+        wk = wl.Workload("tp", T, w_, wl.WHT_BF16_PF32, "normal", 20 + g, True, "")
+        base = wl.gen_full(wk.with_rows(4096), "x").cuda()
+        xs = [base.roll(s, 0).repeat(T // 4096, 1) for s in range(g)]
+        dys = [base.roll(s + g, 0).repeat(T // 4096, 1) for s in range(g)]
+        a, b = (t.cuda() for t in wl.gen_params(wk))
+        as_ = [a.clone() for _ in range(g)]
+        rank = tp.TpWht(g, g - 1)
+        y = torch.empty_like(xs[0])
+        f_ms = time_loop(lambda: rank.forward(xs, a, b, T, w_, out=y), 20, warmup=5)
+        b_ms = time_loop(lambda: rank.backward(dys, xs, as_, T, w_), 20, warmup=5)
+        fb, bb = (g + 1) * T * w_ * 2 / 1e9, (2 * g + 1) * T * w_ * 2 / 1e9
+        out[f"g{g}_w{w_}"] = {"T": T, "fwd_us": 1e3 * f_ms, "fwd_GBps": fb / (f_ms * 1e-3),
+                             "fwd_frac_of_measured_peak": fb / (f_ms * 1e-3) / hbm_peak,
+                             "bwd_us": 1e3 * b_ms, "bwd_GBps": bb / (b_ms * 1e-3),
+                             "bwd_frac_of_measured_peak": bb / (b_ms * 1e-3) / hbm_peak}
+        del xs, dys, y, base
+    return out
+
+
+def section_other_shapes(B, hbm_peak):
+    """Shapes outside the five configs, 256 MiB per row tensor: fp32 storage and the block-diagonal form
+    (butterfly kernels)."""
+    out = {}
+    for d in (256, 512, 2048):
+        T = (256 << 20) // (4 * d)
+        x = torch.randn(T, d, device="cuda")
+        a = torch.rand(d, device="cuda") + 0.5
+        y = torch.empty_like(x)
+        da, db = torch.empty(d, device="cuda"), torch.empty(d, device="cuda")
+        f_ms = time_loop(lambda: B.wht_affine_fwd(x, a, a, y, T, d, wl.WHT_F32), 20, warmup=5)
+        b_ms = time_loop(lambda: B.wht_affine_bwd(x, x, a, y, da, db, T, d, wl.WHT_F32), 20, warmup=5)
+        out[f"fp32_d{d}"] = {"T": T, "fwd_us": 1e3 * f_ms, "fwd_frac_of_measured_peak": 8 * T * d / (f_ms * 1e6) / hbm_peak,
+                            "bwd_us": 1e3 * b_ms, "bwd_frac_of_measured_peak": 12 * T * d / (b_ms * 1e6) / hbm_peak}
+        del x, y
+    for d, block in ((768, 256), (1536, 512)):
+        T = 65536
+        x = torch.randn(T, d, device="cuda").bfloat16()
+        a = torch.rand(d, device="cuda") + 0.5
+        y = torch.empty_like(x)
+        da, db = torch.empty(d, device="cuda"), torch.empty(d, device="cuda")
+        ws = torch.empty(max(B.wht_affine_bwd_grouped_workspace_bytes(T, d, block, wl.WHT_BF16_PF32), 16),
+                         dtype=torch.uint8, device="cuda")
+        f_ms = time_loop(lambda: B.wht_affine_fwd_grouped(x, a, a, y, T, d, block, wl.WHT_BF16_PF32), 20, warmup=5)
+        b_ms = time_loop(lambda: B.wht_affine_bwd_grouped(x, x, a, y, da, db, T, d, block, wl.WHT_BF16_PF32, ws),
+                         20, warmup=5)
+        out[f"grouped_d{d}"] = {"T": T, "block": block, "fwd_us": 1e3 * f_ms,
+                               "fwd_frac_of_measured_peak": 4 * T * d / (f_ms * 1e6) / hbm_peak,
+                               "bwd_us": 1e3 * b_ms, "bwd_frac_of_measured_peak": 6 * T * d / (b_ms * 1e6) / hbm_peak}
+        del x, y
+    return out
+
+
 def section_fwd_bwd(B, name, hbm_peak, iters):
     """Forward and backward timed separately on a workload larger than L2."""
     w = wl.CONFIGS[name]
@@ -552,6 +611,8 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         sections["training"] = section_fwd_bwd(B, "training", hbm_peak, 50)
         sections["large"] = section_fwd_bwd(B, "large", hbm_peak, 50)
         sections["paper_shapes"] = section_paper_shapes(B, hbm_peak)
+        sections["tensor_parallel_local"] = section_tensor_parallel_local(B, hbm_peak)
+        sections["other_shapes"] = section_other_shapes(B, hbm_peak)
         out["sections"] = sections
     print(json.dumps(out))
     if world > 1:

@@ -75,3 +75,56 @@ def test_random_shapes_match_the_oracle(B, seed):
             what + ": dx"
         assert np.max(np.abs(to_f64(da.cpu()) - ref_da)) <= 1e-4 * np.max(np.abs(ref_da)), what + ": da"
         assert np.max(np.abs(to_f64(db.cpu()) - ref_db)) <= 1e-4 * np.max(np.abs(ref_db)), what + ": db"
+
+
+def _tp_cases(seed, count):
+    rng = random.Random(seed)
+    out = []
+    for case in range(count):
+        g = rng.choice([2, 2, 4, 4, 8])
+        logw = rng.choice([3, 6, 8, 9, 10, 10, 11, 11, 12])
+        while g << logw > 16384:      # keeps the dense oracle at the full width small
+            logw -= 1
+        w = 1 << logw
+        dtype = rng.choice([wl.WHT_F32, wl.WHT_BF16, wl.WHT_BF16_PF32, wl.WHT_BF16_PF32])
+        variant = rng.choice([0, 1, 4, 4])
+        d = g * w
+        max_rows = max(1, min(3000, (1 << 25) // (d * d // 64 + 1)))
+        if logw >= 10 and rng.random() < 0.5:
+            tile = 128 // (8 * (w // 1024))
+            T = max(1, rng.randint(1, max(1, max_rows // tile)) * tile + rng.choice([-1, 0, 1, tile // 2]))
+        else:
+            T = rng.randint(1, max_rows)
+        out.append((case, g, w, min(T, max_rows), dtype, variant))
+    return out
+
+
+@pytest.mark.parametrize("seed", [21])
+def test_random_column_sharded_shapes_match_the_oracle(B, seed):
+    from paper_2603_08343_b200 import tp
+    for case, g, w, T, dtype, variant in _tp_cases(seed, 20):
+        d = g * w
+        wk = wl.Workload("fuzz-tp", T, d, dtype, "normal", 7000 + 100 * seed + case, True, "")
+        x, dy = wl.gen_full(wk, "x"), wl.gen_full(wk, "dy")
+        a, b = wl.gen_params(wk)
+        B.wht_affine_set_variant(variant)
+        xs = [p.cuda() for p in tp.split_columns(x, g)]
+        dys = [p.cuda() for p in tp.split_columns(dy, g)]
+        as_ = [a[s * w:(s + 1) * w].contiguous().cuda() for s in range(g)]
+        outs = []
+        for r in range(g):
+            rank = tp.TpWht(g, r)
+            y = rank.forward(xs, as_[r], b[r * w:(r + 1) * w].contiguous().cuda(), T, w)
+            outs.append((y,) + rank.backward(dys, xs, as_, T, w))
+        torch.cuda.synchronize()
+        y = torch.cat([o[0] for o in outs], dim=1).cpu()
+        dx = torch.cat([o[1] for o in outs], dim=1).cpu()
+        da, db = torch.cat([o[2] for o in outs]).cpu(), torch.cat([o[3] for o in outs]).cpu()
+        x64, dy64, a64, b64 = to_f64(x), to_f64(dy), to_f64(a), to_f64(b)
+        ref_y = oracle.wht_affine_fwd(x64, a64, b64)
+        ref_dx, ref_da, ref_db = oracle.wht_affine_bwd(dy64, x64, a64)
+        what = f"g={g} w={w} T={T} dtype={dtype} variant={variant}"
+        assert _ratio_rows(to_f64(y), ref_y, dtype, np.linalg.norm(x64, axis=1)) <= 1.0, what + ": y"
+        assert _ratio_rows(to_f64(dx), ref_dx, dtype, np.linalg.norm(a64[None, :] * dy64, axis=1)) <= 1.0, what + ": dx"
+        assert np.max(np.abs(to_f64(da) - ref_da)) <= 1e-4 * np.max(np.abs(ref_da)), what + ": da"
+        assert np.max(np.abs(to_f64(db) - ref_db)) <= 1e-4 * np.max(np.abs(ref_db)), what + ": db"
