@@ -162,8 +162,8 @@ int wht_affine_bwd_noalloc(const void* dy, const void* x, const void* a,
  * within a group only.  The paper does not say what its implementation does at those widths, so this
  * is an explicit alternative of this library, not a claim about the paper's choice; groups = 1 is
  * exactly wht_affine_fwd / wht_affine_bwd.  Same layouts, storage types, aliasing and error rules as
- * the plain calls; rows are still contiguous [T x d].  One launch per group of the butterfly
- * kernels on strided views (this form is not tuned).  The backward takes caller-owned scratch of at
+ * the plain calls; rows are still contiguous [T x d].  One launch of the butterfly kernels, the
+ * channel group being the second grid dimension.  The backward takes caller-owned scratch of at
  * least wht_affine_bwd_grouped_workspace_bytes(T, d, block, dtype) bytes and never allocates.
  */
 int wht_affine_fwd_grouped(const void* x, const void* a, const void* b, void* y,

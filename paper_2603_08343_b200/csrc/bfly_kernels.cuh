@@ -214,6 +214,11 @@ bfly_fwd_kernel(const TIO* x, const TP* __restrict__ a, const TP* __restrict__ b
     const int rg = threadIdx.x / Geo::G;  // row group inside the CTA
     const int t = threadIdx.x % Geo::G;
     float* srow = smem + (Geo::WARP_BITS > 0 ? rg * Geo::D : 0);
+    {   // block-diagonal form: blockIdx.y picks the channel group [y*D, (y+1)*D) of rows ld wide
+        const long long goff = static_cast<long long>(blockIdx.y) * Geo::D;
+        x += goff; y += goff; a += goff; b += goff;
+        if (resid != nullptr) resid += goff;
+    }
 
     constexpr int PC = Geo::PREFETCH ? Geo::C : 1;  // a, b in registers only when a thread has few channels
     float as[PC][8], bs[PC][8];
@@ -270,7 +275,7 @@ bfly_fwd_kernel(const TIO* x, const TP* __restrict__ a, const TP* __restrict__ b
 }
 
 // ---- backward: dx = ((a (.) dy) H)/sqrt(d); per-CTA partial da, db -------------
-// partials layout: [gridDim.x][2][D] fp32; slot 0 holds sum_t dy (.) (x H) WITHOUT
+// partials layout: [gridDim.y][gridDim.x][2][D] fp32; slot 0 holds sum_t dy (.) (x H) WITHOUT
 // the 1/sqrt(d) factor (the finalize pass applies it), slot 1 holds sum_t dy.
 template <int LOGD, typename TIO, typename TP>
 __global__ void __launch_bounds__(BflyBwdGeo<LOGD>::THREADS)
@@ -281,6 +286,11 @@ bfly_bwd_kernel(const TIO* dy, const TIO* x, const TP* __restrict__ a, TIO* dx,
     const int rg = threadIdx.x / Geo::G;
     const int t = threadIdx.x % Geo::G;
     float* srow = smem + rg * Geo::D;
+    {   // block-diagonal form: blockIdx.y picks the channel group; its partials follow the previous group's
+        const long long goff = static_cast<long long>(blockIdx.y) * Geo::D;
+        dy += goff; x += goff; dx += goff; a += goff;
+        partials += static_cast<size_t>(blockIdx.y) * gridDim.x * 2 * Geo::D;
+    }
 
     float da_acc[Geo::C][8], db_acc[Geo::C][8];
 #pragma unroll

@@ -132,6 +132,7 @@ struct Ctx {
     int sms;
     cudaStream_t stream;
     int64_t ld = 0;  // elements between consecutive rows; 0 = contiguous rows (ld == d)
+    int groups = 1;  // block-diagonal form: channel groups of d side by side in a row (butterfly family only)
 };
 
 struct FwdArgs {
@@ -156,29 +157,34 @@ struct BwdArgs {
 };
 
 // da = scale * (sum of the partials' first slots), db = sum of their second slots
-int launch_finalize(const BwdArgs& g, int nparts, int d, float scale, cudaStream_t s) {
+int launch_finalize(const float* parts, int nparts, int d, float scale, float* da, float* db, cudaStream_t s) {
     if (d >= 32) {
-        launch_overlapped(dadb_finalize32_kernel, 2 * d / 32, 1024, 0, s, static_cast<const float*>(g.ws), nparts, d,
-                          scale, g.da, g.db);
+        launch_overlapped(dadb_finalize32_kernel, 2 * d / 32, 1024, 0, s, parts, nparts, d, scale, da, db);
     } else {
-        launch_overlapped(dadb_finalize_kernel, (2 * d + 255) / 256, 256, 0, s, static_cast<const float*>(g.ws),
-                          nparts, d, scale, g.da, g.db);
+        launch_overlapped(dadb_finalize_kernel, (2 * d + 255) / 256, 256, 0, s, parts, nparts, d, scale, da, db);
     }
     WHT_CUDA_TRY(cudaGetLastError());
     return WHT_OK;
 }
 
-// Common tail of every backward launcher: size the scratch, check it, launch.
+// Common tail of every backward launcher: size the scratch, check it, launch, then the second pass
+// (one per channel group; `grid` is the CTA count per group).
 template <typename Launch>
 int run_bwd_with_grid(const BwdArgs& g, const Ctx& c, int grid, int d, Launch launch, float scale = 0.0f) {
-    *g.need = static_cast<size_t>(grid) * 2 * d * sizeof(float);
+    *g.need = static_cast<size_t>(grid) * c.groups * 2 * d * sizeof(float);
     if (g.query_only) return WHT_OK;
     if (*g.need > 0 && (g.ws == nullptr || g.ws_bytes < *g.need)) return WHT_ERR_WORKSPACE;
     if (grid > 0) {
         launch(grid);
         WHT_CUDA_TRY(cudaGetLastError());
     }
-    return launch_finalize(g, grid, d, scale > 0.0f ? scale : inv_sqrt(d), c.stream);
+    for (int grp = 0; grp < c.groups; ++grp) {
+        const int rc = launch_finalize(static_cast<const float*>(g.ws) + static_cast<size_t>(grp) * grid * 2 * d, grid, d,
+                                       scale > 0.0f ? scale : inv_sqrt(d), g.da + static_cast<size_t>(grp) * d,
+                                       g.db + static_cast<size_t>(grp) * d, c.stream);
+        if (rc != WHT_OK) return rc;
+    }
+    return WHT_OK;
 }
 
 int capped_grid(int64_t tiles, int sms, int per_sm) {
@@ -194,8 +200,9 @@ int launch_bfly_fwd(const FwdArgs& f, const Ctx& c) {
     auto kernel = bfly_fwd_kernel<LOGD, TIO, TP>;
     const int per_sm = resident_ctas(kernel, Geo::THREADS, Geo::SMEM_FWD, c.dev, occ);
     if (per_sm <= 0) return cuda_fail(cudaGetLastError());
-    const int grid = capped_grid(ceil_div(c.T, Geo::R), c.sms, per_sm);
-    kernel<<<grid, Geo::THREADS, Geo::SMEM_FWD, c.stream>>>(
+    int grid = capped_grid(ceil_div(c.T, Geo::R), c.sms, per_sm);
+    if (c.groups > 1) grid = grid / c.groups > 0 ? grid / c.groups : 1;  // CTAs per channel group
+    kernel<<<dim3(grid, c.groups), Geo::THREADS, Geo::SMEM_FWD, c.stream>>>(
         static_cast<const TIO*>(f.x), static_cast<const TP*>(f.a), static_cast<const TP*>(f.b),
         static_cast<const TIO*>(f.resid), static_cast<TIO*>(f.y), static_cast<long long>(c.T),
         static_cast<long long>(c.ld ? c.ld : Geo::D), inv_sqrt(Geo::D));
@@ -210,9 +217,10 @@ int launch_bfly_bwd(const BwdArgs& g, const Ctx& c) {
     auto kernel = bfly_bwd_kernel<LOGD, TIO, TP>;
     const int per_sm = resident_ctas(kernel, Geo::THREADS, Geo::SMEM_BWD, c.dev, occ);
     if (per_sm <= 0) return cuda_fail(cudaGetLastError());
-    const int grid = capped_grid(ceil_div(c.T, Geo::R), c.sms, per_sm);
+    int grid = capped_grid(ceil_div(c.T, Geo::R), c.sms, per_sm);
+    if (c.groups > 1) grid = grid / c.groups > 0 ? grid / c.groups : 1;  // CTAs per channel group
     return run_bwd_with_grid(g, c, grid, Geo::D, [&](int n) {
-        kernel<<<n, Geo::THREADS, Geo::SMEM_BWD, c.stream>>>(
+        kernel<<<dim3(n, c.groups), Geo::THREADS, Geo::SMEM_BWD, c.stream>>>(
             static_cast<const TIO*>(g.dy), static_cast<const TIO*>(g.x), static_cast<const TP*>(g.a),
             static_cast<TIO*>(g.dx), static_cast<float*>(g.ws), static_cast<long long>(c.T),
             static_cast<long long>(c.ld ? c.ld : Geo::D), inv_sqrt(Geo::D));
@@ -786,7 +794,7 @@ int wht_affine_bwd_noalloc(const void* dy, const void* x, const void* a, void* d
 }
 
 // ---- grouped (block-diagonal) form: d = groups * block, every block transformed on its own.
-// Runs the butterfly family on strided views, one launch per group.
+// One launch of the butterfly family with the channel group as the grid's second dimension.
 namespace {
 int check_grouped(int64_t T, int32_t d, int32_t block, int dtype) {
     if (dtype != WHT_F32 && dtype != WHT_BF16 && dtype != WHT_BF16_PF32) return WHT_ERR_BAD_DTYPE;
@@ -794,10 +802,6 @@ int check_grouped(int64_t T, int32_t d, int32_t block, int dtype) {
     if (T < 0) return WHT_ERR_BAD_T;
     return WHT_OK;
 }
-size_t io_bytes(int dtype) { return dtype == WHT_F32 ? 4 : 2; }
-size_t param_bytes(int dtype) { return dtype == WHT_BF16 ? 2 : 4; }
-const char* at_bytes(const void* p, size_t bytes) { return static_cast<const char*>(p) + bytes; }
-char* at_bytes_mut(void* p, size_t bytes) { return static_cast<char*>(p) + bytes; }
 }  // namespace
 
 int wht_affine_fwd_grouped(const void* x, const void* a, const void* b, void* y, int64_t T, int32_t d,
@@ -812,19 +816,14 @@ int wht_affine_fwd_grouped(const void* x, const void* a, const void* b, void* y,
     c.ld = d;
     rc = current_device(&c.dev, &c.sms);
     if (rc != WHT_OK) return rc;
+    c.groups = d / block;
     const int logb = log2_of(block);
-    for (int32_t g = 0; g < d / block; ++g) {
-        const size_t io = static_cast<size_t>(g) * block * io_bytes(dtype);
-        const size_t pp = static_cast<size_t>(g) * block * param_bytes(dtype);
-        FwdArgs f{at_bytes(x, io), at_bytes(a, pp), at_bytes(b, pp), at_bytes_mut(y, io)};
-        switch (dtype) {
-            case WHT_F32: rc = dispatch_bfly_fwd<float, float>(logb, f, c); break;
-            case WHT_BF16: rc = dispatch_bfly_fwd<__nv_bfloat16, __nv_bfloat16>(logb, f, c); break;
-            default: rc = dispatch_bfly_fwd<__nv_bfloat16, float>(logb, f, c); break;
-        }
-        if (rc != WHT_OK) return rc;
+    const FwdArgs f{x, a, b, y};
+    switch (dtype) {
+        case WHT_F32: return dispatch_bfly_fwd<float, float>(logb, f, c);
+        case WHT_BF16: return dispatch_bfly_fwd<__nv_bfloat16, __nv_bfloat16>(logb, f, c);
+        default: return dispatch_bfly_fwd<__nv_bfloat16, float>(logb, f, c);
     }
-    return WHT_OK;
 }
 
 int wht_affine_bwd_grouped(const void* dy, const void* x, const void* a, void* dx, float* da, float* db, int64_t T,
@@ -841,28 +840,22 @@ int wht_affine_bwd_grouped(const void* dy, const void* x, const void* a, void* d
     c.ld = d;
     rc = current_device(&c.dev, &c.sms);
     if (rc != WHT_OK) return rc;
+    c.groups = d / block;
     const int logb = log2_of(block);
-    for (int32_t g = 0; g < d / block; ++g) {
-        const size_t io = static_cast<size_t>(g) * block * io_bytes(dtype);
-        const size_t pp = static_cast<size_t>(g) * block * param_bytes(dtype);
-        size_t need = 0;
-        // the groups run one after another on the stream and share the scratch
-        BwdArgs q{at_bytes(dy, io), at_bytes(x, io), at_bytes(a, pp), at_bytes_mut(dx, io), da + static_cast<size_t>(g) * block,
-                  db + static_cast<size_t>(g) * block, workspace, workspace_bytes, false, &need};
-        switch (dtype) {
-            case WHT_F32: rc = dispatch_bfly_bwd<float, float>(logb, q, c); break;
-            case WHT_BF16: rc = dispatch_bfly_bwd<__nv_bfloat16, __nv_bfloat16>(logb, q, c); break;
-            default: rc = dispatch_bfly_bwd<__nv_bfloat16, float>(logb, q, c); break;
-        }
-        if (rc != WHT_OK) return rc;
+    size_t need = 0;
+    const BwdArgs q{dy, x, a, dx, da, db, workspace, workspace_bytes, false, &need};
+    switch (dtype) {
+        case WHT_F32: return dispatch_bfly_bwd<float, float>(logb, q, c);
+        case WHT_BF16: return dispatch_bfly_bwd<__nv_bfloat16, __nv_bfloat16>(logb, q, c);
+        default: return dispatch_bfly_bwd<__nv_bfloat16, float>(logb, q, c);
     }
-    return WHT_OK;
 }
 
 size_t wht_affine_bwd_grouped_workspace_bytes(int64_t T, int32_t d, int32_t block, int dtype) {
     if (check_grouped(T, d, block, dtype) != WHT_OK) return 0;
     Ctx c{T, 0, 0, nullptr};
     if (current_device(&c.dev, &c.sms) != WHT_OK) return 0;
+    c.groups = d / block;
     size_t need = 0;
     BwdArgs q{nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, 0, true, &need};
     int rc;
