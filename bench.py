@@ -19,6 +19,7 @@ from __future__ import annotations
 
 import argparse
 import json
+import math
 import os
 import statistics
 import subprocess
@@ -160,9 +161,11 @@ def run_reference(args, rank: int, world: int):
     if rank != 0:
         return
     w = wl.CONFIGS[args.workload]
-    rows = {"tiny": 64, "prefill": 2048, "training": 1024, "large": 128}[args.workload]
-    # keep the whole run to about a minute of CPU work whatever K is: the per-row cost is constant
-    rows = max(16, min(rows, (32 * rows) // max(args.steps, 1)))
+    # keep the whole run to about a minute of CPU work whatever K is: a short pilot gives the rate, the
+    # rows per step follow from it (the per-row cost is constant)
+    pilot = {"tiny": 64, "prefill": 2048, "training": 1024, "large": 128}[args.workload]
+    rate = pilot / oracle_step_seconds(w, pilot, repeats=2)
+    rows = max(16, min(w.T, 16384, int(rate * 60.0 / max(args.steps, 1)) // 16 * 16))
     for _ in range(min(args.warmup, 3)):
         oracle_step_seconds(w, min(rows, 64))
     times = [oracle_step_seconds(w, rows) for _ in range(args.steps)]
@@ -595,12 +598,17 @@ def run_ours(args, rank: int, world: int, local_rank: int):
                       "frac_of_nominal_8000": achieved / 8000.0, "tokens_per_s": w.T / (dom_ms * 1e-3)}
 
     # ---- CPU baseline: the oracle as it stands, on a bounded sample of the same workload
-    rows = {"tiny": 64, "prefill": 4096, "training": 2048, "large": 256}[w.name]
-    sec = oracle_step_seconds(w, rows)
-    out["cpu_baseline"] = {"value": rows / sec, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+    # (a short pilot sizes it: up to 16384 rows per pass, passes until about 12 s of CPU work)
+    pilot = {"tiny": 64, "prefill": 4096, "training": 2048, "large": 256}[w.name]
+    rate = pilot / oracle_step_seconds(w, pilot)
+    rows = min(w.T, 16384, max(pilot, int(rate * 4) // 256 * 256))
+    passes = max(1, min(16, math.ceil(12.0 * rate / rows)))
+    sec = sum(oracle_step_seconds(w, rows) for _ in range(passes))
+    out["cpu_baseline"] = {"value": rows * passes / sec, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
                            "seconds": sec,
-                           "sample": f"{rows} rows of the {w.name} workload (d={w.d}), fp64 dense product, "
-                                     f"fwd{'+bwd' if w.has_bwd else ''}; tokens/s from that sample (per-row cost is constant)"}
+                           "sample": f"{passes} passes over {rows} rows of the {w.name} workload (d={w.d}), fp64 dense "
+                                     f"product, fwd{'+bwd' if w.has_bwd else ''}; tokens/s from that sample "
+                                     "(per-row cost is constant)"}
 
     if not args.no_sections and world == 1:
         del xs, ys, dys, dxs, x, y, dy, dx
