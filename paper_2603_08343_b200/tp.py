@@ -87,3 +87,32 @@ def _dtype_of(part, a):
 def _code(rows, a):
     from . import binding
     return binding.dtype_code(rows, a)
+
+
+class SymmetricBlocks:
+    """This rank's [T, w] block in torch symmetric memory, with every rank's address of it.
+
+    `tensor` is the local block (fill it, or have the producing kernel write into it);
+    `addresses[s]` is rank s's block as mapped into THIS process (entry `rank` is the local
+    one), ready to be passed as `x_parts` / `dy_parts` / `a_parts`.  `barrier()` is the
+    cross-rank synchronisation the calls need: once after every rank has written its block
+    and before any rank launches, once after the launches and before anybody overwrites.
+    All ranks of `group` must construct it together (the rendezvous is collective).
+    """
+
+    def __init__(self, T: int, w: int, dtype, group=None, device=None):
+        import torch.distributed as dist
+        import torch.distributed._symmetric_memory as symm_mem
+        if group is None:
+            group = dist.group.WORLD
+        device = torch.device("cuda", torch.cuda.current_device()) if device is None else torch.device(device)
+        self.tensor = symm_mem.empty((T, w), dtype=dtype, device=device)
+        self.handle = symm_mem.rendezvous(self.tensor, group)
+        self.rank = int(self.handle.rank)
+        self.world_size = int(self.handle.world_size)
+        self.addresses = [int(p) for p in self.handle.buffer_ptrs]
+        if self.addresses[self.rank] != self.tensor.data_ptr():
+            raise RuntimeError("symmetric memory handed back a block that is not at the tensor's address")
+
+    def barrier(self):
+        self.handle.barrier()

@@ -109,3 +109,40 @@ def test_no_rows(B):
     torch.cuda.synchronize()
     assert y.shape == (0, w) and dx.shape == (0, w)
     assert torch.all(da == 0) and torch.all(db == 0)
+
+
+def test_blocks_in_symmetric_memory_single_rank(B):
+    """The helper that hands out peer addresses, with a process group of one rank (all that one GPU allows):
+    the address table has this rank's own block, and a call through it equals the plain call."""
+    import os
+    import socket
+    import torch.distributed as dist
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    os.environ["MASTER_ADDR"], os.environ["MASTER_PORT"] = "127.0.0.1", str(port)
+    started = not dist.is_initialized()
+    if started:
+        dist.init_process_group("nccl", rank=0, world_size=1, device_id=torch.device("cuda", 0))
+    try:
+        T, w = 257, 1024
+        try:
+            blk = tp.SymmetricBlocks(T, w, torch.bfloat16)
+        except Exception as exc:  # driver or build without symmetric memory support
+            pytest.skip(f"torch symmetric memory is not available here: {exc}")
+        assert blk.world_size == 1 and blk.rank == 0 and blk.addresses == [blk.tensor.data_ptr()]
+        wk = wl.Workload("tp", T, w, wl.WHT_BF16_PF32, "normal", 31, True, "")
+        x = wl.gen_full(wk, "x").cuda()
+        a, b = (t.cuda() for t in wl.gen_params(wk))
+        blk.tensor.copy_(x)
+        blk.barrier()
+        y = torch.empty_like(x)
+        tp.TpWht(1, 0).forward(blk.addresses, a, b, T, w, out=y)
+        blk.barrier()
+        torch.cuda.synchronize()
+        B.wht_affine_set_variant(1)
+        assert torch.equal(y, B.forward(x, a, b))
+        B.wht_affine_set_variant(0)
+    finally:
+        if started:
+            dist.destroy_process_group()
