@@ -555,6 +555,37 @@ def test_autograd_wrapper(B):
     assert torch.equal(rd.grad.view(-1, w.d).cpu(), dy)
 
 
+def test_layer_module(B):
+    from paper_2603_08343_b200.autograd import WhtAffine
+    B.wht_affine_set_variant(0)
+    for d, block, T in ((1024, None, 130), (768, 256, 77)):
+        layer = WhtAffine(d, block=block, device="cuda")
+        assert sorted(n for n, _ in layer.named_parameters()) == ["a", "b"] and layer.a.numel() == d
+        gen = torch.Generator().manual_seed(d)
+        x = torch.randn(T, d, generator=gen).bfloat16()
+        dy = torch.randn(T, d, generator=gen).bfloat16()
+        with torch.no_grad():  # move the parameters off their initial 1 / 0 so that they matter
+            layer.a.copy_(torch.rand(d, generator=gen) + 0.5)
+            layer.b.copy_(torch.randn(d, generator=gen) * 0.1)
+        xd = x.cuda().view(1, T, d).requires_grad_(True)
+        out = layer(xd)
+        out.backward(dy.cuda().view(1, T, d))
+        torch.cuda.synchronize()
+        a64, b64 = to_f64(layer.a.detach().cpu()), to_f64(layer.b.detach().cpu())
+        if block is None:
+            ref_y = oracle.wht_affine_fwd(to_f64(x), a64, b64)
+            ref_dx, ref_da, ref_db = oracle.wht_affine_bwd(to_f64(dy), to_f64(x), a64)
+        else:
+            ref_y = oracle.wht_affine_fwd_grouped(to_f64(x), a64, b64, block)
+            ref_dx, ref_da, ref_db = oracle.wht_affine_bwd_grouped(to_f64(dy), to_f64(x), a64, block)
+        assert_rows_bf16(to_f64(out.detach().cpu().view(T, d)), ref_y, "layer y")
+        assert_rows_bf16(to_f64(xd.grad.cpu().view(T, d)), ref_dx, "layer dx")
+        assert_grad_vec(to_f64(layer.a.grad.cpu()), ref_da, "layer da")
+        assert_grad_vec(to_f64(layer.b.grad.cpu()), ref_db, "layer db")
+    with pytest.raises(ValueError):
+        WhtAffine(768)
+
+
 def test_copy_rows(B):
     src = torch.arange(3 * 1024, dtype=torch.float32, device="cuda").view(3, 1024)
     dst = torch.zeros_like(src)
