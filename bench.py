@@ -271,6 +271,35 @@ def section_decode(B):
     return out
 
 
+def section_tiny(B):
+    """The Tiny config (64 x 256, fp32): latency-bound; device time per call from a CUDA-graph replay of 50
+    forward + backward pairs (the backward is its main kernel plus the small second pass)."""
+    w = wl.CONFIGS["tiny"]
+    x, dy = wl.gen_full(w, "x").cuda(), wl.gen_full(w, "dy").cuda()
+    a, b = (t.cuda() for t in wl.gen_params(w))
+    y, dx = torch.empty_like(x), torch.empty_like(x)
+    da, db = torch.empty(w.d, device="cuda"), torch.empty(w.d, device="cuda")
+    ws = torch.empty(max(B.wht_affine_bwd_workspace_bytes(w.T, w.d, w.dtype), 16), dtype=torch.uint8, device="cuda")
+    out = {"T": w.T, "d": w.d, "dtype": "fp32"}
+    s = torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        for which in ("fwd", "bwd"):
+            def call():
+                if which == "fwd":
+                    B.wht_affine_fwd(x, a, b, y, w.T, w.d, w.dtype)
+                else:
+                    B.wht_affine_bwd_ws(dy, x, a, dx, da, db, w.T, w.d, w.dtype, ws)
+            for _ in range(3):
+                call()
+            torch.cuda.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=s):
+                for _ in range(50):
+                    call()
+            out[f"{which}_graph_replay_us_per_call"] = 1e3 * time_loop(g.replay, 40, warmup=3) / 50
+    return out
+
+
 def section_paper_shapes(B, hbm_peak):
     """The paper's own inference shapes (its prefill table: batch 1024 x 64 tokens = 65536 rows; its
     decode table: batch 2048, one row per sequence and step) at its two power-of-two model widths."""
@@ -614,6 +643,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         del xs, ys, dys, dxs, x, y, dy, dx
         torch.cuda.empty_cache()
         sections = {}
+        sections["tiny"] = section_tiny(B)
         sections["prefill"] = section_prefill(B, hbm_peak)
         sections["decode"] = section_decode(B)
         sections["training"] = section_fwd_bwd(B, "training", hbm_peak, 50)
