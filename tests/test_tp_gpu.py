@@ -123,7 +123,10 @@ def test_blocks_in_symmetric_memory_single_rank(B):
     os.environ["MASTER_ADDR"], os.environ["MASTER_PORT"] = "127.0.0.1", str(port)
     started = not dist.is_initialized()
     if started:
-        dist.init_process_group("nccl", rank=0, world_size=1, device_id=torch.device("cuda", 0))
+        try:
+            dist.init_process_group("nccl", rank=0, world_size=1, device_id=torch.device("cuda", 0))
+        except Exception as exc:
+            pytest.skip(f"no NCCL process group on this box: {exc}")
     try:
         T, w = 257, 1024
         try:
