@@ -185,7 +185,7 @@ size_t wht_affine_bwd_grouped_workspace_bytes(int64_t T, int32_t d, int32_t bloc
  * which are exactly column block r of wht_affine_fwd / wht_affine_bwd on the concatenated tensors.
  * One kernel per call reads the g blocks (its own and the peers') with plain loads, forms the
  * signed sum of the stored values in fp32 and runs the width-w transform: the exchange of the top
- * log2 g stages and the local stages are fused, no intermediate is written.  No multicast.
+ * log2 g stages and the local stages are fused, no intermediate is written.  Every load is one CTA's own.
  *   x_parts, dy_parts, a_parts  HOST arrays of g DEVICE pointers; entry s is rank s's block
  *                  (x, dy: [T x w] row-major; a: [w]); entry r is this GPU's own memory, the others
  *                  are peer mappings the caller obtained (CUDA IPC, symmetric memory) and keeps valid

@@ -7,7 +7,7 @@
 // were issued are still waited for, bounded again), so a fault in the pipeline
 // shows up as a status the host can read instead of a hang.
 //
-// No copy uses cluster multicast and every source is this GPU's own memory.
+// Every copy is issued by one CTA for itself alone and every source is this GPU's own memory.
 #pragma once
 #include "mma_kernels.cuh"
 

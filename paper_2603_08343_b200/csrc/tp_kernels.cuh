@@ -7,7 +7,7 @@
 //
 // the top log2 g stages are a signed sum of the g blocks, taken on the STORED values while
 // they are loaded (from this GPU's memory for s == r, through peer mappings otherwise:
-// plain 128-bit loads, no multicast), and the rest is the local transform of width w.
+// plain 128-bit loads by each CTA for itself), and the rest is the local transform of width w.
 // The exchange and the transform are one kernel: no block is written back between them.
 //
 // Backward of the same map for rank r:

@@ -37,7 +37,7 @@
 // flag and the device status word; every role then leaves its loop, copies in flight
 // are waited for (bounded), TMEM is freed and the kernel returns: a fault in the
 // pipeline shows up as WHT_ERR_DEVICE_WAIT on the host, never as a hang.
-// No copy uses cluster multicast; every source is this GPU's own memory, except in the
+// Every copy is issued by one CTA for itself alone; every source is this GPU's own memory, except in the
 // column-sharded forward, whose source blocks may be peer mappings.
 #pragma once
 #include "mma_pipe_kernels.cuh"
@@ -276,7 +276,7 @@ __device__ __forceinline__ void stage_params_umma(const TP* __restrict__ src, fl
 //
 // MULTI (column-sharded form): the rows come as nsrc blocks of D channels, one per rank, and the
 // transform input is their signed sum, sign H_g[s][r].  Each block's tile is copied into a ring slot
-// of its own (from this GPU's memory or through a peer mapping; plain bulk copies, never multicast)
+// of its own (from this GPU's memory or through a peer mapping; plain bulk copies of one CTA for itself)
 // and multiplied by H_128 into the SAME accumulator, with the instruction descriptor's negate-A bit
 // set for the blocks whose sign is -1: the signed sum happens in the tensor core's fp32 accumulation
 // of exact +-1 products, and the epilogue is the ordinary one.  inv_sqrt_d is then 1/sqrt(nsrc * D).
