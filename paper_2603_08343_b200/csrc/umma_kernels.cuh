@@ -31,7 +31,8 @@
 // The backward pass runs two products per tile: D1 = H_128 X (for da) and
 // D2 = H_128 G, where G = (a/sqrt(d)) (.) dy after ITS register stages, written back
 // into the ring slot as bf16 hi + lo (two products into one accumulator; the pair
-// carries 16-17 significant bits, and the accumulation is again fp32).
+// carries 16-17 significant bits, and the accumulation is again fp32).  The backward keeps H_128
+// in tensor memory and feeds it to the products from there (less shared-memory traffic per product).
 //
 // Every wait on an mbarrier is bounded.  A wait that expires raises a CTA-wide abort
 // flag and the device status word; every role then leaves its loop, copies in flight
@@ -71,6 +72,44 @@ __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint6
         ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
+// The same with the A operand read from tensor memory (lane = row m, two bf16 per 32-bit column,
+// K = 16 per instruction = 8 columns) instead of shared memory.
+__device__ __forceinline__ void umma_bf16_a_tmem(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc,
+                                                 uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// 16 consecutive columns of this thread's TMEM lane, written from registers
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+          "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+        : "memory");
+}
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// Row m of H_128 into columns [taddr, taddr + 64) of this thread's TMEM lane: column c holds
+// H[m][2c] (low half) and H[m][2c+1] (high half) as bf16.
+__device__ __forceinline__ void write_h128_row_tmem(uint32_t taddr, int m) {
+#pragma unroll
+    for (int c0 = 0; c0 < 64; c0 += 16) {
+        uint32_t r[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const int k = 2 * (c0 + i);
+            const uint32_t lo = (__popc(m & k) & 1) ? 0xBF80u : 0x3F80u;
+            const uint32_t hi = (__popc(m & (k + 1)) & 1) ? 0xBF80u : 0x3F80u;
+            r[i] = lo | (hi << 16);
+        }
+        tmem_st16(taddr + c0, r);
+    }
+    tmem_wait_st();
+}
+
 // mbarrier arrive once all tcgen05 operations issued so far by this thread are complete
 __device__ __forceinline__ void umma_commit(uint64_t* bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
@@ -556,7 +595,7 @@ template <int LOGD, int NCOL, int STAGES>
 struct UmmaBwdSmem {
     using Geo = UmmaGeo<LOGD, NCOL>;
     static constexpr int STAGE_BYTES = 2 * Geo::TILE_BYTES;  // x tile, then dy tile
-    static constexpr int TMEM_COLS = 4 * NCOL <= 256 ? 256 : 512;  // D1 x2, D2 x2
+    static constexpr int TMEM_COLS = 4 * NCOL <= 256 ? 256 : 512;  // D1 x2, D2 x2 (or D2 x1 and H_128)
     static constexpr int OFF_H = 0;
     static constexpr int OFF_RING = Geo::H_BYTES;
     static constexpr int OFF_BARS = OFF_RING + STAGES * STAGE_BYTES;
@@ -568,7 +607,7 @@ struct UmmaBwdSmem {
 
 // partials layout: [gridDim.x][2][D] fp32; slot 0: sum_t dy (.) (x H) WITHOUT the
 // 1/sqrt(d) factor (the second pass applies it), slot 1: sum_t dy.
-template <int LOGD, int NCOL, int STAGES, typename TP>
+template <int LOGD, int NCOL, int STAGES, typename TP, bool A_TMEM = false>
 __global__ void __launch_bounds__(UmmaGeo<LOGD, NCOL>::THREADS, 1)
 umma_bwd_kernel(const __nv_bfloat16* dy, const __nv_bfloat16* x, const TP* __restrict__ a, __nv_bfloat16* dx,
                 float* __restrict__ partials, long long T, float inv_sqrt_d) {
@@ -621,8 +660,10 @@ umma_bwd_kernel(const __nv_bfloat16* dy, const __nv_bfloat16* x, const TP* __res
         *abort_flag = 0;
         fence_mbar_init();
     }
-    write_h128(smem_raw + L::OFF_H, tid, Geo::THREADS);
-    fence_async_smem();
+    if constexpr (!A_TMEM) {
+        write_h128(smem_raw + L::OFF_H, tid, Geo::THREADS);
+        fence_async_smem();
+    }
     if (warp == 1) {
         tmem_alloc(tmem_slot, L::TMEM_COLS);
         tmem_relinquish();
@@ -636,6 +677,17 @@ umma_bwd_kernel(const __nv_bfloat16* dy, const __nv_bfloat16* x, const TP* __res
     grid_launch_dependents();
     const uint32_t tmem_d1 = tmem_base;
     const uint32_t tmem_d2 = tmem_base + 2 * Geo::N;
+    // A_TMEM: H_128 is kept in tensor memory (64 columns after a single D2 buffer) and the products read
+    // it from there, which takes a third of their operand traffic off the shared memory
+    const uint32_t tmem_a = tmem_base + 3 * Geo::N;
+    if constexpr (A_TMEM) {
+        static_assert(3 * Geo::N + 64 <= L::TMEM_COLS, "no room for H_128 in tensor memory");
+        if (warp >= 2 && warp < 6)
+            write_h128_row_tmem(tmem_a + (static_cast<uint32_t>((warp & 3) * 32) << 16), (warp & 3) * 32 + lane);
+        tc_fence_before();
+        __syncthreads();
+        tc_fence_after();
+    }
 
     // per-thread partial column sums (epilogue warps only; declared here so that the fold
     // after the role loops can see them)
@@ -684,8 +736,12 @@ umma_bwd_kernel(const __nv_bfloat16* dy, const __nv_bfloat16* x, const TP* __res
                 tc_fence_after();
                 const uint64_t bdesc = umma_smem_desc(smem_u32(ring + s * L::STAGE_BYTES));
 #pragma unroll
-                for (int k = 0; k < 8; ++k)
-                    umma_bf16(tmem_d1 + t * Geo::N, adesc + k * 16, bdesc + k * 16, idesc, k > 0);
+                for (int k = 0; k < 8; ++k) {
+                    if constexpr (A_TMEM)
+                        umma_bf16_a_tmem(tmem_d1 + t * Geo::N, tmem_a + k * 8, bdesc + k * 16, idesc, k > 0);
+                    else
+                        umma_bf16(tmem_d1 + t * Geo::N, adesc + k * 16, bdesc + k * 16, idesc, k > 0);
+                }
                 umma_commit(d1_full + t);
                 return true;
             };
@@ -693,18 +749,27 @@ umma_bwd_kernel(const __nv_bfloat16* dy, const __nv_bfloat16* x, const TP* __res
             auto step_g = [&](long long i) -> bool {
                 const int s = static_cast<int>(i % STAGES);
                 const uint32_t ph = static_cast<uint32_t>(i / STAGES) & 1u;
-                const int t = static_cast<int>(i & 1);
-                const uint32_t pt = static_cast<uint32_t>(i >> 1) & 1u;
+                const int t = A_TMEM ? 0 : static_cast<int>(i & 1);  // A_TMEM: one D2 buffer
+                const uint32_t pt = static_cast<uint32_t>(A_TMEM ? i : (i >> 1)) & 1u;
                 if (!wait_or_abort(g_ready + s, ph, abort_flag)) return false;
                 if (!wait_or_abort(d2_empty + t, pt ^ 1u, abort_flag)) return false;
                 tc_fence_after();
                 const uint64_t bhi = umma_smem_desc(smem_u32(ring + s * L::STAGE_BYTES));
                 const uint64_t blo = umma_smem_desc(smem_u32(ring + s * L::STAGE_BYTES + Geo::TILE_BYTES));
 #pragma unroll
-                for (int k = 0; k < 8; ++k)
-                    umma_bf16(tmem_d2 + t * Geo::N, adesc + k * 16, bhi + k * 16, idesc, k > 0);
+                for (int k = 0; k < 8; ++k) {
+                    if constexpr (A_TMEM)
+                        umma_bf16_a_tmem(tmem_d2 + t * Geo::N, tmem_a + k * 8, bhi + k * 16, idesc, k > 0);
+                    else
+                        umma_bf16(tmem_d2 + t * Geo::N, adesc + k * 16, bhi + k * 16, idesc, k > 0);
+                }
 #pragma unroll
-                for (int k = 0; k < 8; ++k) umma_bf16(tmem_d2 + t * Geo::N, adesc + k * 16, blo + k * 16, idesc, 1);
+                for (int k = 0; k < 8; ++k) {
+                    if constexpr (A_TMEM)
+                        umma_bf16_a_tmem(tmem_d2 + t * Geo::N, tmem_a + k * 8, blo + k * 16, idesc, 1);
+                    else
+                        umma_bf16(tmem_d2 + t * Geo::N, adesc + k * 16, blo + k * 16, idesc, 1);
+                }
                 umma_commit(d2_full + t);
                 umma_commit(stage_empty + s);
                 return true;
@@ -767,8 +832,8 @@ umma_bwd_kernel(const __nv_bfloat16* dy, const __nv_bfloat16* x, const TP* __res
 
         // dx rows of tile j: read D2, (split: top-bit stage,) round, store
         auto store_dx = [&](int j) -> bool {
-            const int t = j & 1;
-            const uint32_t pt = static_cast<uint32_t>(j >> 1) & 1u;
+            const int t = A_TMEM ? 0 : (j & 1);
+            const uint32_t pt = static_cast<uint32_t>(A_TMEM ? j : (j >> 1)) & 1u;
             if (!warp_wait_or_abort(d2_full + t, pt, abort_flag)) return false;
             tc_fence_after();
             const uint32_t acc = tmem_d2 + t * Geo::N;

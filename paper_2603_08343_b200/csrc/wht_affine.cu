@@ -407,13 +407,13 @@ int launch_umma_fwd(const FwdArgs& f, const Ctx& c) {
                    : launch_umma_fwd_impl<LOGD, NCOL, STAGES, TP, false>(f, c);
 }
 
-template <int LOGD, int NCOL, int STAGES, typename TP>
-int launch_umma_bwd(const BwdArgs& g, const Ctx& c) {
+template <int LOGD, int NCOL, int STAGES, typename TP, bool A_TMEM>
+int launch_umma_bwd_impl(const BwdArgs& g, const Ctx& c) {
     using Geo = UmmaGeo<LOGD, NCOL>;
     using L = UmmaBwdSmem<LOGD, NCOL, STAGES>;
     static_assert(L::BYTES > 116 * 1024, "must be alone on its SM");
     static int ready[kMaxDevices] = {};
-    auto kernel = umma_bwd_kernel<LOGD, NCOL, STAGES, TP>;
+    auto kernel = umma_bwd_kernel<LOGD, NCOL, STAGES, TP, A_TMEM>;
     if (!g.query_only) {
         int rc = prepare_umma(kernel, L::BYTES, c.dev, ready);
         if (rc != WHT_OK) return rc;
@@ -425,6 +425,13 @@ int launch_umma_bwd(const BwdArgs& g, const Ctx& c) {
                           static_cast<const TP*>(g.a), static_cast<__nv_bfloat16*>(g.dx), static_cast<float*>(g.ws),
                           static_cast<long long>(c.T), inv_sqrt(Geo::D));
     });
+}
+
+// H_128 in tensor memory: measured 1-2 % faster than the shared-memory operand in long runs under the
+// power cap (less shared-memory traffic per product), the same in short bursts.
+template <int LOGD, int NCOL, int STAGES, typename TP>
+int launch_umma_bwd(const BwdArgs& g, const Ctx& c) {
+    return launch_umma_bwd_impl<LOGD, NCOL, STAGES, TP, true>(g, c);
 }
 
 template <typename TP>
