@@ -41,7 +41,7 @@ METRIC = "wht_affine_tokens_per_s_fwd_bwd"
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the dominant kernel,
 # from the one-pass ncu capture at full size quoted in profiles/umma_bwd_training_d2048.txt;
 # keyed by (workload, rows).  Reset to {} when the kernel changes.
-NCU_TRAFFIC_BYTES = {("training", 65536): 537070336 + 228010496}  # umma_bwd_kernel<11,128,3>, full size
+NCU_TRAFFIC_BYTES = {("training", 65536): 537027072 + 228779264}  # umma_bwd_kernel<11,128,3,float,1>, full size
 UNIT = "tokens/s"
 
 
