@@ -219,6 +219,8 @@ bfly_fwd_kernel(const TIO* x, const TP* __restrict__ a, const TP* __restrict__ b
         x += goff; y += goff; a += goff; b += goff;
         if (resid != nullptr) resid += goff;
     }
+    grid_dependency_wait();  // nothing above touched global memory
+    grid_launch_dependents();
 
     constexpr int PC = Geo::PREFETCH ? Geo::C : 1;  // a, b in registers only when a thread has few channels
     float as[PC][8], bs[PC][8];
@@ -291,6 +293,8 @@ bfly_bwd_kernel(const TIO* dy, const TIO* x, const TP* __restrict__ a, TIO* dx,
         dy += goff; x += goff; dx += goff; a += goff;
         partials += static_cast<size_t>(blockIdx.y) * gridDim.x * 2 * Geo::D;
     }
+    grid_dependency_wait();  // nothing above touched global memory
+    grid_launch_dependents();
 
     float da_acc[Geo::C][8], db_acc[Geo::C][8];
 #pragma unroll

@@ -109,9 +109,9 @@ int resident_ctas(Kernel kernel, int threads, size_t smem, int dev, int* cache) 
 // while its predecessor in the stream drains.  Only for kernels that call
 // grid_dependency_wait() before they touch global memory.
 template <typename... KArgs, typename... Args>
-void launch_overlapped(void (*kernel)(KArgs...), int grid, int block, size_t smem, cudaStream_t s, Args... args) {
+void launch_overlapped(void (*kernel)(KArgs...), dim3 grid, int block, size_t smem, cudaStream_t s, Args... args) {
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(static_cast<unsigned>(grid));
+    cfg.gridDim = grid;
     cfg.blockDim = dim3(static_cast<unsigned>(block));
     cfg.dynamicSmemBytes = smem;
     cfg.stream = s;
@@ -202,10 +202,10 @@ int launch_bfly_fwd(const FwdArgs& f, const Ctx& c) {
     if (per_sm <= 0) return cuda_fail(cudaGetLastError());
     int grid = capped_grid(ceil_div(c.T, Geo::R), c.sms, per_sm);
     if (c.groups > 1) grid = grid / c.groups > 0 ? grid / c.groups : 1;  // CTAs per channel group
-    kernel<<<dim3(grid, c.groups), Geo::THREADS, Geo::SMEM_FWD, c.stream>>>(
-        static_cast<const TIO*>(f.x), static_cast<const TP*>(f.a), static_cast<const TP*>(f.b),
-        static_cast<const TIO*>(f.resid), static_cast<TIO*>(f.y), static_cast<long long>(c.T),
-        static_cast<long long>(c.ld ? c.ld : Geo::D), inv_sqrt(Geo::D));
+    launch_overlapped(kernel, dim3(grid, c.groups), Geo::THREADS, Geo::SMEM_FWD, c.stream,
+                      static_cast<const TIO*>(f.x), static_cast<const TP*>(f.a), static_cast<const TP*>(f.b),
+                      static_cast<const TIO*>(f.resid), static_cast<TIO*>(f.y), static_cast<long long>(c.T),
+                      static_cast<long long>(c.ld ? c.ld : Geo::D), inv_sqrt(Geo::D));
     WHT_CUDA_TRY(cudaGetLastError());
     return WHT_OK;
 }
@@ -220,10 +220,10 @@ int launch_bfly_bwd(const BwdArgs& g, const Ctx& c) {
     int grid = capped_grid(ceil_div(c.T, Geo::R), c.sms, per_sm);
     if (c.groups > 1) grid = grid / c.groups > 0 ? grid / c.groups : 1;  // CTAs per channel group
     return run_bwd_with_grid(g, c, grid, Geo::D, [&](int n) {
-        kernel<<<dim3(n, c.groups), Geo::THREADS, Geo::SMEM_BWD, c.stream>>>(
-            static_cast<const TIO*>(g.dy), static_cast<const TIO*>(g.x), static_cast<const TP*>(g.a),
-            static_cast<TIO*>(g.dx), static_cast<float*>(g.ws), static_cast<long long>(c.T),
-            static_cast<long long>(c.ld ? c.ld : Geo::D), inv_sqrt(Geo::D));
+        launch_overlapped(kernel, dim3(n, c.groups), Geo::THREADS, Geo::SMEM_BWD, c.stream,
+                          static_cast<const TIO*>(g.dy), static_cast<const TIO*>(g.x), static_cast<const TP*>(g.a),
+                          static_cast<TIO*>(g.dx), static_cast<float*>(g.ws), static_cast<long long>(c.T),
+                          static_cast<long long>(c.ld ? c.ld : Geo::D), inv_sqrt(Geo::D));
     });
 }
 
