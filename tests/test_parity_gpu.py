@@ -555,6 +555,58 @@ def test_autograd_wrapper(B):
     assert torch.equal(rd.grad.view(-1, w.d).cpu(), dy)
 
 
+@pytest.mark.parametrize("variant", VARIANTS)
+@pytest.mark.parametrize("d,T", [(2048, 301), (8192, 37), (256, 100)])
+def test_a_non_finite_row_stays_in_its_row(B, d, T, variant):
+    """Rows are independent: Inf or NaN in one row of x (or dy) must leave every other row of y (dx)
+    bit-identical -- tiles hold several rows side by side in shared and tensor memory -- while da, db,
+    which sum over rows, follow the arithmetic (non-finite)."""
+    B.wht_affine_set_variant(variant)
+    w = wl.Workload("poison", T, d, wl.WHT_BF16_PF32, "normal", 4242 + d, True, "")
+    x, dy = wl.gen_full(w, "x").cuda(), wl.gen_full(w, "dy").cuda()
+    a, b = (t.cuda() for t in wl.gen_params(w))
+    y0 = B.forward(x, a, b)
+    dx0, da0, db0 = B.backward(dy, x, a)
+    bad_row, other = T // 2, [r for r in range(T) if r != T // 2]
+    xp = x.clone()
+    xp[bad_row, 7] = float("inf")
+    xp[bad_row, d - 3] = float("nan")
+    y1 = B.forward(xp, a, b)
+    dx1, da1, db1 = B.backward(dy, xp, a)          # x enters da only
+    dyp = dy.clone()
+    dyp[bad_row, 1] = float("-inf")
+    dx2, da2, db2 = B.backward(dyp, x, a)
+    torch.cuda.synchronize()
+    assert torch.equal(y1[other], y0[other]) and not torch.isfinite(y1[bad_row]).any()
+    assert torch.equal(dx1, dx0) and torch.equal(db1, db0) and not torch.isfinite(da1).any()
+    assert torch.equal(dx2[other], dx0[other]) and not torch.isfinite(dx2[bad_row]).any()
+    assert not torch.isfinite(db2[1]) and torch.isfinite(db2[2:]).all()
+    B.wht_affine_set_variant(0)
+
+
+def test_calls_on_two_streams_at_once(B):
+    """A forward and a backward (caller-owned scratch) issued on two streams with no ordering between them
+    give the bits of the serial calls: the kernels share SMs, tensor memory and the device-wide status word
+    but no data."""
+    B.wht_affine_set_variant(0)
+    w = wl.CONFIGS["training"].with_rows(8192)
+    x1, x2, dy2 = wl.gen_full(w, "x").cuda(), wl.gen_full(w, "dy").cuda(), wl.gen_full(w, "x").cuda().flip(0).contiguous()
+    a, b = (t.cuda() for t in wl.gen_params(w))
+    y_ref = B.forward(x1, a, b)
+    dx_ref, da_ref, db_ref = B.backward(dy2, x2, a)
+    ws = torch.empty(max(B.wht_affine_bwd_workspace_bytes(w.T, w.d, w.dtype), 16), dtype=torch.uint8, device="cuda")
+    y, dx = torch.empty_like(x1), torch.empty_like(x2)
+    da, db = torch.empty_like(da_ref), torch.empty_like(db_ref)
+    torch.cuda.synchronize()
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    for _ in range(10):
+        B.wht_affine_fwd(x1, a, b, y, w.T, w.d, w.dtype, stream=s1)
+        B.wht_affine_bwd_ws(dy2, x2, a, dx, da, db, w.T, w.d, w.dtype, ws, stream=s2)
+    torch.cuda.synchronize()
+    assert torch.equal(y, y_ref) and torch.equal(dx, dx_ref)
+    assert torch.equal(da, da_ref) and torch.equal(db, db_ref)
+
+
 def test_layer_module(B):
     from paper_2603_08343_b200.autograd import WhtAffine
     B.wht_affine_set_variant(0)
