@@ -24,7 +24,9 @@ the Kronecker recursion, H H^T = d I in integers, norm preservation, involution,
 impulse and constant rows, brute force at d <= 16 (also with a residual row added),
 the Fig. 2 butterfly with its
 d*log2(d) operation count, central finite differences and the adjoint identity
-for the gradients.  No function here is "parity unpinned".
+for the gradients; the column form of da, db over several of its row blocks (ragged
+last block) against the full definition and a per-row loop.  No function here is
+"parity unpinned".
 """
 from __future__ import annotations
 

@@ -275,6 +275,65 @@ def test_da_db_columns_agrees_with_full():
     np.testing.assert_allclose(db_c, db[cols], rtol=1e-12, atol=1e-13)
 
 
+def test_da_db_columns_over_several_row_blocks():
+    """The column form walks the rows in blocks of 4096: with T = 9001 it takes three trips, the last
+    one ragged.  Pinned against the full definition (chain rule on Eq. 1; itself pinned by finite
+    differences above) on ALL columns and on a sample, and against a plain per-row loop written from
+    the definition da[j] = sum_t dy[t, j] * (sum_i x[t, i] H[i][j]) / sqrt(d).  A block read without its
+    row offset, a dropped last block or a block counted twice fails it."""
+    rng = np.random.default_rng(2603)
+    T, d = 9001, 64
+    x = rng.standard_normal((T, d)).astype(np.float32)
+    dy = rng.standard_normal((T, d)).astype(np.float32)
+    # rows differ in scale from block to block, so that a block taken for another cannot cancel out
+    x *= (1.0 + np.arange(T) // 4096)[:, None].astype(np.float32)
+    _, da, db = oracle.wht_affine_bwd(dy, x, np.ones(d))
+    every = np.arange(d)
+    da_c, db_c = oracle.da_db_columns(dy, x, every)
+    np.testing.assert_allclose(da_c, da, rtol=1e-11, atol=1e-9)
+    np.testing.assert_allclose(db_c, db, rtol=1e-11, atol=1e-9)
+    some = np.array([0, 1, 31, 32, 63])
+    da_s, db_s = oracle.da_db_columns(dy, x, some)
+    np.testing.assert_allclose(da_s, da[some], rtol=1e-11, atol=1e-9)
+    np.testing.assert_allclose(db_s, db[some], rtol=1e-11, atol=1e-9)
+    # the definition as a loop over rows, for two columns
+    H = oracle.sylvester_hadamard(d)
+    for j in (1, 63):
+        acc_a = acc_b = 0.0
+        for t in range(T):
+            acc_a += float(dy[t, j]) * float(np.dot(x[t].astype(np.float64), H[:, j])) / math.sqrt(d)
+            acc_b += float(dy[t, j])
+        assert da_c[j] == pytest.approx(acc_a, rel=1e-10, abs=1e-9)
+        assert db_c[j] == pytest.approx(acc_b, rel=1e-10, abs=1e-9)
+    # what the pin would catch: the sums over the first two blocks only, or with the first block twice
+    da_short, _ = oracle.da_db_columns(dy[:8192], x[:8192], every)
+    da_twice = da_short + oracle.da_db_columns(dy[:4096], x[:4096], every)[0] \
+        - oracle.da_db_columns(dy[4096:8192], x[4096:8192], every)[0]
+    assert np.max(np.abs(da_short - da)) > 1e-3 * np.max(np.abs(da))
+    assert np.max(np.abs(da_twice - da)) > 1e-3 * np.max(np.abs(da))
+
+
+def test_da_db_columns_adds_over_row_blocks_like_the_parity_tests_use_it():
+    """The full-size parity tests call the column form on 8192-row slices and add the results; the sum
+    over slices must be the value over all rows (da and db are sums over rows)."""
+    rng = np.random.default_rng(8343)
+    T, d = 20000, 32
+    x = rng.standard_normal((T, d))
+    dy = rng.standard_normal((T, d))
+    cols = np.array([0, 7, 16, 31])
+    whole_a, whole_b = oracle.da_db_columns(dy, x, cols)
+    parts_a, parts_b = np.zeros(cols.size), np.zeros(cols.size)
+    for r0 in range(0, T, 8192):
+        pa, pb = oracle.da_db_columns(dy[r0:r0 + 8192], x[r0:r0 + 8192], cols)
+        parts_a += pa
+        parts_b += pb
+    np.testing.assert_allclose(parts_a, whole_a, rtol=1e-11, atol=1e-9)
+    np.testing.assert_allclose(parts_b, whole_b, rtol=1e-11, atol=1e-9)
+    _, da, db = oracle.wht_affine_bwd(dy, x, np.ones(d))
+    np.testing.assert_allclose(whole_a, da[cols], rtol=1e-11, atol=1e-9)
+    np.testing.assert_allclose(whole_b, db[cols], rtol=1e-11, atol=1e-9)
+
+
 def test_widen_bf16_bits_exact():
     # 0x3F80 = 1.0, 0xC000 = -2.0, 0x3DCD ~ 0.100098 (bf16 nearest to 0.1), 0x0000 = 0
     bits = np.array([0x3F80, 0xC000, 0x3DCD, 0x0000, 0x7F7F], dtype=np.uint16)
