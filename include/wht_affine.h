@@ -21,7 +21,14 @@
  *     (the row tensors may then be NULL; a, b, da, db are always required).
  *   - `dtype` selects the storage types (wht_dtype below).  All arithmetic is
  *     fp32 whatever the storage type; bf16 outputs are rounded once, to nearest
- *     even, at the store.
+ *     even, at the store.  One exception: in the tensor-core kernels (bf16 rows,
+ *     512 <= d <= 8192) an fp32 intermediate that feeds a second +-1 product is
+ *     split into a bf16 pair hi + lo, which carries 16-17 significant bits
+ *     (relative error 2^-17) instead of 24.  This touches dx of the backward
+ *     calls (and y of the mma.sync forward, variants 2 and 3); sums are still
+ *     fp32.  The effect, about 4e-5 of a row's largest output, is far inside the
+ *     bf16 rounding of the result (2^-9) and is bounded by the library's test
+ *     test_outputs_are_the_correctly_rounded_values_almost_everywhere.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
  *     Calls are asynchronous: they enqueue work and return without synchronising.
  *   - Exact aliasing y == x and dx == dy is allowed (a row is read completely

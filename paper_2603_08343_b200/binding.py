@@ -298,19 +298,21 @@ def forward_host(x_host, a_host, b_host, y_host, staging, stream=None, pipe: Hos
     all copies are asynchronous on the current stream; with a HostPipe the rows move in chunks
     on its copy streams and the caller ends the step with pipe.join().
     """
-    if pipe is None:
-        staging["x"].copy_(x_host, non_blocking=True)
-        staging["a"].copy_(a_host, non_blocking=True)
-        staging["b"].copy_(b_host, non_blocking=True)
-        forward(staging["x"], staging["a"], staging["b"], out=staging["y"], stream=stream)
-        y_host.copy_(staging["y"], non_blocking=True)
-        return y_host
     cur = torch.cuda.current_stream() if stream is None else stream
+    if pipe is None:
+        with torch.cuda.stream(cur):  # copies and kernels on ONE stream: ordered by it
+            staging["x"].copy_(x_host, non_blocking=True)
+            staging["a"].copy_(a_host, non_blocking=True)
+            staging["b"].copy_(b_host, non_blocking=True)
+            forward(staging["x"], staging["a"], staging["b"], out=staging["y"], stream=cur)
+            y_host.copy_(staging["y"], non_blocking=True)
+        return y_host
     xs, ys, a, b = staging["x"], staging["y"], staging["a"], staging["b"]
     d = xs.shape[-1]
     code = dtype_code(xs, a)
     pipe.s_in.wait_stream(cur)   # the staging buffers may still be in use by earlier work
     pipe.s_out.wait_stream(cur)
+    cur.wait_stream(pipe.s_out)  # ... and an earlier step's copies out may still be reading staging["y"]
     with torch.cuda.stream(pipe.s_in):
         a.copy_(a_host, non_blocking=True)
         b.copy_(b_host, non_blocking=True)
@@ -338,17 +340,23 @@ def backward_host(dy_host, x_host, a_host, dx_host, da_host, db_host, staging, s
     d = st["x"].shape[-1]
     T = st["x"].numel() // d
     code = dtype_code(st["x"], st["a"])
-    if pipe is None:
-        st["dy"].copy_(dy_host, non_blocking=True)
-        if not x_resident:
-            st["x"].copy_(x_host, non_blocking=True)
-            st["a"].copy_(a_host, non_blocking=True)
-        wht_affine_bwd(st["dy"], st["x"], st["a"], st["dx"], st["da"], st["db"], T, d, code, stream)
-        dx_host.copy_(st["dx"], non_blocking=True)
-        da_host.copy_(st["da"], non_blocking=True)
-        db_host.copy_(st["db"], non_blocking=True)
-        return
     cur = torch.cuda.current_stream() if stream is None else stream
+    if pipe is None:
+        with torch.cuda.stream(cur):  # copies and kernels on ONE stream: ordered by it
+            st["dy"].copy_(dy_host, non_blocking=True)
+            if not x_resident:
+                st["x"].copy_(x_host, non_blocking=True)
+                st["a"].copy_(a_host, non_blocking=True)
+            wht_affine_bwd(st["dy"], st["x"], st["a"], st["dx"], st["da"], st["db"], T, d, code, cur)
+            dx_host.copy_(st["dx"], non_blocking=True)
+            da_host.copy_(st["da"], non_blocking=True)
+            db_host.copy_(st["db"], non_blocking=True)
+        return
+    # the staging buffers (and the per-chunk gradient pairs) may still be in use by earlier work on `cur`:
+    # a previous step's kernels read st["dy"] / st["x"], its copies out read st["dx"]
+    pipe.s_in.wait_stream(cur)
+    pipe.s_out.wait_stream(cur)
+    cur.wait_stream(pipe.s_out)
     # dy comes in chunk by chunk on the copy stream (sharing the link with the forward's y going
     # out); each chunk is transformed as it lands and its dx leaves on the other copy stream, so the
     # two directions of the link stay busy together.  da, db are sums over rows: every chunk writes

@@ -34,6 +34,13 @@ int cuda_fail(cudaError_t e) {
     return WHT_ERR_CUDA;
 }
 
+// A kernel of which not even one CTA fits on an SM: report the runtime's error if it raised one,
+// else "launch out of resources", so that WHT_ERR_CUDA never comes with a last-error of 0.
+int occupancy_fail() {
+    const cudaError_t e = cudaGetLastError();
+    return cuda_fail(e != cudaSuccess ? e : cudaErrorLaunchOutOfResources);
+}
+
 #define WHT_CUDA_TRY(expr)                                   \
     do {                                                     \
         cudaError_t e__ = (expr);                            \
@@ -199,7 +206,7 @@ int launch_bfly_fwd(const FwdArgs& f, const Ctx& c) {
     static int occ[kMaxDevices] = {};
     auto kernel = bfly_fwd_kernel<LOGD, TIO, TP>;
     const int per_sm = resident_ctas(kernel, Geo::THREADS, Geo::SMEM_FWD, c.dev, occ);
-    if (per_sm <= 0) return cuda_fail(cudaGetLastError());
+    if (per_sm <= 0) return occupancy_fail();
     int grid = capped_grid(ceil_div(c.T, Geo::R), c.sms, per_sm);
     if (c.groups > 1) grid = grid / c.groups > 0 ? grid / c.groups : 1;  // CTAs per channel group
     launch_overlapped(kernel, dim3(grid, c.groups), Geo::THREADS, Geo::SMEM_FWD, c.stream,
@@ -216,7 +223,7 @@ int launch_bfly_bwd(const BwdArgs& g, const Ctx& c) {
     static int occ[kMaxDevices] = {};
     auto kernel = bfly_bwd_kernel<LOGD, TIO, TP>;
     const int per_sm = resident_ctas(kernel, Geo::THREADS, Geo::SMEM_BWD, c.dev, occ);
-    if (per_sm <= 0) return cuda_fail(cudaGetLastError());
+    if (per_sm <= 0) return occupancy_fail();
     int grid = capped_grid(ceil_div(c.T, Geo::R), c.sms, per_sm);
     if (c.groups > 1) grid = grid / c.groups > 0 ? grid / c.groups : 1;  // CTAs per channel group
     return run_bwd_with_grid(g, c, grid, Geo::D, [&](int n) {
@@ -257,7 +264,7 @@ int launch_mma_fwd(const FwdArgs& f, const Ctx& c) {
     static int occ[kMaxDevices] = {};
     auto kernel = mma_fwd_kernel<LOGD, TB, RG, TP>;
     const int per_sm = resident_ctas(kernel, Geo::THREADS, Geo::SMEM_FWD, c.dev, occ);
-    if (per_sm <= 0) return cuda_fail(cudaGetLastError());
+    if (per_sm <= 0) return occupancy_fail();
     const int grid = capped_grid(ceil_div(c.T, RG), c.sms, per_sm);
     launch_overlapped(kernel, grid, Geo::THREADS, Geo::SMEM_FWD, c.stream,
                       static_cast<const __nv_bfloat16*>(f.x), static_cast<const TP*>(f.a), static_cast<const TP*>(f.b),
@@ -273,7 +280,7 @@ int launch_mma_bwd(const BwdArgs& g, const Ctx& c) {
     static int occ[kMaxDevices] = {};
     auto kernel = mma_bwd_kernel<LOGD, TB, RG, TP>;
     const int per_sm = resident_ctas(kernel, Geo::THREADS, Geo::SMEM_BWD, c.dev, occ);
-    if (per_sm <= 0) return cuda_fail(cudaGetLastError());
+    if (per_sm <= 0) return occupancy_fail();
     const int grid = capped_grid(ceil_div(c.T, RG), c.sms, per_sm);
     return run_bwd_with_grid(g, c, grid, Geo::D, [&](int n) {
         kernel<<<n, Geo::THREADS, Geo::SMEM_BWD, c.stream>>>(
@@ -290,7 +297,7 @@ int launch_mma_fwd_pipe(const FwdArgs& f, const Ctx& c) {
     static int occ[kMaxDevices] = {};
     auto kernel = mma_fwd_pipe_kernel<LOGD, TB, RG, S, MINB, TP>;
     const int per_sm = resident_ctas(kernel, Geo::THREADS, Geo::SMEM, c.dev, occ);
-    if (per_sm <= 0) return cuda_fail(cudaGetLastError());
+    if (per_sm <= 0) return occupancy_fail();
     const int grid = capped_grid(ceil_div(c.T, RG), c.sms, per_sm);
     kernel<<<grid, Geo::THREADS, Geo::SMEM, c.stream>>>(
         static_cast<const __nv_bfloat16*>(f.x), static_cast<const TP*>(f.a), static_cast<const TP*>(f.b),
@@ -306,7 +313,7 @@ int launch_mma_bwd_pipe(const BwdArgs& g, const Ctx& c) {
     static int occ[kMaxDevices] = {};
     auto kernel = mma_bwd_pipe_kernel<LOGD, TB, RG, S, MINB, TP>;
     const int per_sm = resident_ctas(kernel, Geo::THREADS, Geo::SMEM, c.dev, occ);
-    if (per_sm <= 0) return cuda_fail(cudaGetLastError());
+    if (per_sm <= 0) return occupancy_fail();
     const int grid = capped_grid(ceil_div(c.T, RG), c.sms, per_sm);
     return run_bwd_with_grid(g, c, grid, Geo::D, [&](int n) {
         kernel<<<n, Geo::THREADS, Geo::SMEM, c.stream>>>(
@@ -572,7 +579,7 @@ int launch_bfly_fwd_tp(const TpCall& t, const FwdArgs& f, const Ctx& c) {
     static int occ[kMaxDevices] = {};
     auto kernel = bfly_fwd_tp_kernel<LOGW, TIO, TP>;
     const int per_sm = resident_ctas(kernel, Geo::THREADS, Geo::SMEM_FWD, c.dev, occ);
-    if (per_sm <= 0) return cuda_fail(cudaGetLastError());
+    if (per_sm <= 0) return occupancy_fail();
     const int grid = capped_grid(ceil_div(c.T, Geo::R), c.sms, per_sm);
     kernel<<<grid, Geo::THREADS, Geo::SMEM_FWD, c.stream>>>(t.xs, t.g, t.neg_mask, static_cast<const TP*>(f.a),
                                                             static_cast<const TP*>(f.b), static_cast<TIO*>(f.y),
@@ -587,7 +594,7 @@ int launch_bfly_bwd_tp(const TpCall& t, const BwdArgs& g, const Ctx& c) {
     static int occ[kMaxDevices] = {};
     auto kernel = bfly_bwd_tp_kernel<LOGW, TIO, TP>;
     const int per_sm = resident_ctas(kernel, Geo::THREADS, Geo::SMEM_BWD, c.dev, occ);
-    if (per_sm <= 0) return cuda_fail(cudaGetLastError());
+    if (per_sm <= 0) return occupancy_fail();
     const int grid = capped_grid(ceil_div(c.T, Geo::R), c.sms, per_sm);
     return run_bwd_with_grid(
         g, c, grid, Geo::D,

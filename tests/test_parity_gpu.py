@@ -135,7 +135,25 @@ def _sample_rows(T, n, seed):
     return np.array(sorted(rows))
 
 
-def _full_size_case(B, w, n_rows, n_cols, variant):
+def _spread_columns(d, per_cell, seed):
+    """Column sample that reaches every part of the kernels' channel layouts: for every 1024-channel
+    piece of a row and every group of 32 consecutive 8-channel chunks (the tensor-memory lane quarter
+    that owns them in the tcgen05 kernels; both halves of the channels at d >= 4096), `per_cell` random
+    columns, plus the corners."""
+    rng = np.random.default_rng(seed)
+    cols = {0, 1, d // 2 - 1, d // 2, d - 2, d - 1}
+    for piece in range(max(1, d // 1024)):
+        for quarter in range(4):
+            m = rng.integers(quarter * 32, quarter * 32 + 32, per_cell)
+            n = rng.integers(0, 8, per_cell)
+            cols |= set((piece * 1024 + m * 8 + n).tolist())
+    return np.array(sorted(c for c in cols if 0 <= c < d))
+
+
+def _full_size_case(B, w, n_rows, cols, variant):
+    """Full-size run of a config in the launch configuration the benchmark times.  y and dx: sampled rows
+    against the oracle (Eq. 1 and its chain rule).  da, db need every row: the oracle's column form over
+    all T rows, on the columns given (None = every column)."""
     B.wht_affine_set_variant(variant)
     a, b = wl.gen_params(w)
     ad, bd = a.cuda(), b.cuda()
@@ -154,9 +172,8 @@ def _full_size_case(B, w, n_rows, n_cols, variant):
     assert_rows_bf16(to_f64(ys), ref_y, f"{w.name} fwd sampled rows")
     ref_dx, _, _ = oracle.wht_affine_bwd(to_f64(dys), to_f64(xs), a64)
     assert_rows_bf16(to_f64(dxs), ref_dx, f"{w.name} dx sampled rows")
-    # da, db need every row: the oracle's column form, summed over row blocks
-    rng = np.random.default_rng(w.seed + 1)
-    cols = np.array(sorted(set([0, 1, w.d // 2, w.d - 1]) | set(rng.integers(0, w.d, n_cols).tolist())))
+    every = cols is None
+    cols = np.arange(w.d) if every else np.asarray(cols)
     da_ref = np.zeros(cols.size)
     db_ref = np.zeros(cols.size)
     blk = 8192
@@ -166,24 +183,63 @@ def _full_size_case(B, w, n_rows, n_cols, variant):
         db_ref += pb
     da_got = to_f64(da.cpu())[cols]
     db_got = to_f64(db.cpu())[cols]
-    # the bound is 1e-4 * max|g_ref| over the vector; the sampled columns give a lower
-    # estimate of that maximum, which only makes the check stricter
-    assert_grad_vec(da_got, da_ref, f"{w.name} da sampled columns")
-    assert_grad_vec(db_got, db_ref, f"{w.name} db sampled columns")
-    # db over ALL columns against plain column sums in fp64 (cheap at any size)
-    db_all = np.zeros(w.d)
-    for r0 in range(0, w.T, blk):
-        db_all += to_f64(dy[r0:r0 + blk]).sum(axis=0)
-    assert_grad_vec(to_f64(db.cpu()), db_all, f"{w.name} db all columns")
+    # the bound is 1e-4 * max|g_ref| over the vector; a column sample gives a lower estimate of that
+    # maximum, which only makes the check stricter
+    which = "all columns" if every else f"{cols.size} columns"
+    assert_grad_vec(da_got, da_ref, f"{w.name} da {which}")
+    assert_grad_vec(db_got, db_ref, f"{w.name} db {which}")
+    if not every:
+        # db over ALL columns against plain column sums in fp64 (cheap at any size)
+        db_all = np.zeros(w.d)
+        for r0 in range(0, w.T, blk):
+            db_all += to_f64(dy[r0:r0 + blk]).sum(axis=0)
+        assert_grad_vec(to_f64(db.cpu()), db_all, f"{w.name} db all columns")
 
 
 @pytest.mark.parametrize("variant", VARIANTS)
 def test_training_full_size(B, variant):
-    _full_size_case(B, wl.CONFIGS["training"], n_rows=1024, n_cols=96, variant=variant)
+    # the automatic selection (what the benchmark times) is checked on every column of da and db; the
+    # forced families on a spread sample
+    w = wl.CONFIGS["training"]
+    _full_size_case(B, w, n_rows=1024, cols=_spread_columns(w.d, 12, w.seed + 1), variant=variant)
+
+
+def test_training_full_size_every_column(B):
+    _full_size_case(B, wl.CONFIGS["training"], n_rows=1024, cols=None, variant=0)
 
 
 def test_large_full_size(B):
-    _full_size_case(B, wl.CONFIGS["large"], n_rows=256, n_cols=28, variant=0)
+    w = wl.CONFIGS["large"]
+    cols = _spread_columns(w.d, 16, w.seed + 1)  # 8 pieces x 4 lane quarters x 16 = about 500 columns
+    assert cols.size >= 256
+    _full_size_case(B, w, n_rows=256, cols=cols, variant=0)
+
+
+# ------------------------------------------------------------------ the paper's own inference shapes
+
+@pytest.mark.parametrize("d", [1024, 2048])
+def test_paper_prefill_shape(B, d):
+    """The paper's prefill benchmark: batch 1024 x 64 input tokens = 65536 rows, at its two power-of-two
+    model widths (Small d = 1024, Large d = 2048), bf16 rows and parameters; sampled rows against Eq. 1."""
+    B.wht_affine_set_variant(0)
+    w = wl.Workload("paper_prefill", 1024 * 64, d, wl.WHT_BF16, "normal", 10 + d, False, "")
+    a, b = wl.gen_params(w)
+    x = wl.gen_full(w, "x", threads=32)
+    y = B.forward(x.cuda(), a.cuda(), b.cuda())
+    torch.cuda.synchronize()
+    ridx = torch.from_numpy(_sample_rows(w.T, 2048, w.seed))
+    ref = oracle.wht_affine_fwd(to_f64(x[ridx]), to_f64(a), to_f64(b))
+    assert_rows_bf16(to_f64(y[ridx.cuda()].cpu()), ref, f"paper prefill d={d}")
+    B.wht_affine_device_status()
+
+
+@pytest.mark.parametrize("variant", VARIANTS)
+@pytest.mark.parametrize("d", [1024, 2048])
+def test_paper_decode_shape(B, d, variant):
+    """The paper's decode benchmark: batch 2048, one new token per sequence = 2048 rows per call, through
+    wht_affine_fwd_decode; every row against Eq. 1."""
+    w = wl.Workload("paper_decode", 2048, d, wl.WHT_BF16, "normal", 20 + d, False, "")
+    _run_case(B, w, variant, decode=True, bwd=False)
 
 
 # ------------------------------------------------------------------ structure that needs no oracle
@@ -417,6 +473,40 @@ def test_host_pipeline_matches_direct_calls(B):
             assert_rows_bf16(to_f64(dxp), to_f64(dx_ref.cpu()), "chunked backward dx")
             assert_grad_vec(to_f64(dap), to_f64(da_ref.cpu()), "chunked backward da")
             assert_grad_vec(to_f64(dbp), to_f64(db_ref.cpu()), "chunked backward db")
+
+
+def test_host_backward_twice_in_a_row_without_a_sync(B):
+    # Two end-to-end backward calls on different inputs through the SAME staging buffers, no host or
+    # stream synchronisation in between: the second call's copies in must wait for the first call's
+    # kernels, and its kernels for the first call's copies out.  Both results against the oracle.
+    B.wht_affine_set_variant(0)
+    w = wl.CONFIGS["training"].with_rows(6000)
+    a, _ = wl.gen_params(w)
+    sets = []
+    for k in range(2):
+        wk = wl.Workload(w.name, w.T, w.d, w.dtype, w.dist, w.seed + 50 + k, True, "")
+        sets.append((wl.gen_full(wk, "x"), wl.gen_full(wk, "dy")))
+    dev = lambda t: torch.empty_like(t, device="cuda")  # noqa: E731
+    for pipe in (None, B.HostPipe(chunk_rows=1024)):
+        st = {"x": dev(sets[0][0]), "a": dev(a), "dy": dev(sets[0][0]), "dx": dev(sets[0][0]),
+              "da": torch.empty(w.d, device="cuda"), "db": torch.empty(w.d, device="cuda")}
+        ap = a.pin_memory()
+        outs = []
+        for x, dy in sets:
+            xp, dyp = x.pin_memory(), dy.pin_memory()
+            dxp = torch.empty_like(xp).pin_memory()
+            dap, dbp = torch.empty(w.d).pin_memory(), torch.empty(w.d).pin_memory()
+            B.backward_host(dyp, xp, ap, dxp, dap, dbp, st, pipe=pipe, x_resident=False)
+            outs.append((xp, dyp, dxp, dap, dbp))
+        if pipe is not None:
+            pipe.join()
+        torch.cuda.synchronize()
+        for k, (xp, dyp, dxp, dap, dbp) in enumerate(outs):
+            ref_dx, ref_da, ref_db = oracle.wht_affine_bwd(to_f64(dyp), to_f64(xp), to_f64(a))
+            tag = f"host backward call {k} ({'plain' if pipe is None else 'piped'})"
+            assert_rows_bf16(to_f64(dxp), ref_dx, tag + " dx")
+            assert_grad_vec(to_f64(dap), ref_da, tag + " da")
+            assert_grad_vec(to_f64(dbp), ref_db, tag + " db")
 
 
 def test_reduce_grads(B):

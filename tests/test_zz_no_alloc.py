@@ -11,6 +11,7 @@ another test's result in a run that stops at the first failure.
 import pytest
 import torch
 
+import oracle
 from helpers import assert_grad_vec, assert_rows_bf16, assert_rows_fp32, to_f64
 from paper_2603_08343_b200 import workloads as wl
 
@@ -43,12 +44,23 @@ def _both(B, w):
 
 def test_two_calls_in_a_row_match_the_allocating_entry_point(B):
     cases = [
-        wl.Workload("noalloc", 5000, 2048, wl.WHT_BF16_PF32, "normal", 41, True, ""),  # many CTAs: most of the array used
+        wl.Workload("noalloc", 5000, 2048, wl.WHT_BF16_PF32, "normal", 41, True, ""),  # 148 CTAs x 16 KiB of partial sums
         wl.Workload("noalloc", 301, 1024, wl.WHT_BF16, "normal", 42, True, ""),        # fewer, smaller partials over stale data
+        wl.Workload("noalloc", 600, 8192, wl.WHT_F32, "normal", 45, True, ""),         # butterfly family, 64 KiB per CTA: most of the array
+        wl.Workload("noalloc", 300, 4096, wl.WHT_BF16_PF32, "normal", 46, True, ""),
         wl.Workload("noalloc", 64, 256, wl.WHT_F32, "normal", 43, True, ""),
     ]
     for w in cases:
         (ref, got), a, dy = _both(B, w)
+        # against the definition itself (chain rule on Eq. 1), not only against the other entry point
+        x = wl.gen_full(w, "x")
+        o_dx, o_da, o_db = oracle.wht_affine_bwd(to_f64(dy), to_f64(x), to_f64(a))
+        if w.dtype == wl.WHT_F32:
+            assert_rows_fp32(to_f64(got[0]), o_dx, to_f64(a)[None, :] * to_f64(dy), "noalloc dx vs oracle")
+        else:
+            assert_rows_bf16(to_f64(got[0]), o_dx, "noalloc dx vs oracle")
+        assert_grad_vec(to_f64(got[1]), o_da, "noalloc da vs oracle")
+        assert_grad_vec(to_f64(got[2]), o_db, "noalloc db vs oracle")
         if w.dtype == wl.WHT_F32:
             assert_rows_fp32(to_f64(got[0]), to_f64(ref[0]), to_f64(a)[None, :] * to_f64(dy), "noalloc dx")
         else:
@@ -57,6 +69,15 @@ def test_two_calls_in_a_row_match_the_allocating_entry_point(B):
         assert_grad_vec(to_f64(got[2]), to_f64(ref[2]), "noalloc db")
         # same kernels, same launch shape, fixed summation order: the results are in fact identical
         assert all(torch.equal(g, r) for g, r in zip(got, ref))
+
+
+def test_every_width_up_to_8192_fits_the_builtin_array(B):
+    # the header promises that d <= 8192 fits for any T: the scratch need grows with the CTA count, which
+    # stops growing once every SM is full, so a large T gives the maximum
+    for logd in range(3, 14):
+        for dtype in (wl.WHT_F32, wl.WHT_BF16, wl.WHT_BF16_PF32):
+            need = B.wht_affine_bwd_workspace_bytes(1 << 22, 1 << logd, dtype)
+            assert 0 < need <= 16 * 1024 * 1024, f"d={1 << logd} dtype={dtype}: {need} bytes"
 
 
 def test_oversized_problem_is_rejected_without_launching(B):
