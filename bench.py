@@ -38,11 +38,32 @@ from paper_2603_08343_b200 import dp
 from paper_2603_08343_b200 import workloads as wl
 
 METRIC = "wht_affine_tokens_per_s_fwd_bwd"
-# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the dominant kernel,
-# from the one-pass ncu capture at full size quoted in profiles/umma_bwd_training_d2048.txt;
-# keyed by (workload, rows).  Reset to {} when the kernel changes.
-NCU_TRAFFIC_BYTES = {("training", 65536): 537027072 + 228779264}  # umma_bwd_kernel<11,128,3,float,1>, full size
 UNIT = "tokens/s"
+# DRAM bytes of one launch of the dominant kernel come from the ncu capture recorded in this file, in a
+# line "traffic_record: ..." that also names the kernel and a digest of the sources it was built from.
+TRAFFIC_PROFILE = os.path.join("profiles", "umma_bwd_training_d2048.txt")
+
+
+def ncu_traffic(workload: str, rows: int):
+    """(bytes or None, where it comes from): dram__bytes_read.sum + dram__bytes_write.sum of one launch of the
+    dominant kernel, read from the committed ncu summary; None once the kernel's sources have changed since."""
+    from paper_2603_08343_b200 import build as _build
+    path = os.path.join(ROOT, TRAFFIC_PROFILE)
+    try:
+        text = open(path).read()
+    except OSError:
+        return None, f"{TRAFFIC_PROFILE} missing"
+    for line in text.splitlines():
+        if not line.startswith("traffic_record:"):
+            continue
+        rec = dict(kv.split("=", 1) for kv in line.split()[1:])
+        if rec.get("workload") != workload or int(rec.get("rows", -1)) != rows:
+            continue
+        if rec.get("sources_sha256") != _build.source_digest(rec.get("sources", "").split(",")):
+            return None, f"{TRAFFIC_PROFILE}: stale (the sources of {rec.get('kernel')} changed since the capture)"
+        total = int(rec["dram_bytes_read"]) + int(rec["dram_bytes_write"])
+        return total, f"{TRAFFIC_PROFILE}: {rec.get('kernel')}, one ncu pass at {rows} rows, sources unchanged since"
+    return None, f"{TRAFFIC_PROFILE}: no capture recorded for {workload} at {rows} rows"
 
 
 # ----------------------------------------------------------------------------- helpers
@@ -83,18 +104,26 @@ class ClockSampler:
         for line in self.proc.stdout:
             self.lines.append((time.time(), line.strip()))
 
-    def stop(self, t0=None, t1=None):
+    def stop_all(self):
+        """Ends the sampling; returns every (time, line) sample for summarise()."""
         if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+            return []
         time.sleep(0.15)
         self.proc.terminate()
         try:
             self.proc.wait(timeout=5)
         except subprocess.TimeoutExpired:
             self.proc.kill()
+        return list(self.lines)
+
+    @staticmethod
+    def summarise(samples, t0=None, t1=None):
+        """Median SM clock, maximum power and the throttle reasons seen between t0 and t1."""
+        if not samples:
+            return {"sm_mhz": None, "sm_max_mhz": None, "samples": 0, "reasons": ["nvidia-smi unavailable"]}
         sm, mx, reasons, power = [], [], set(), []
-        for ts, line in self.lines:
-            if t0 is not None and not (t0 - 0.05 <= ts <= t1 + 0.15):
+        for ts, line in samples:
+            if t0 is not None and not (t0 + 0.02 <= ts <= t1 + 0.02):
                 continue
             parts = [p.strip() for p in line.split(",")]
             if len(parts) < 9:
@@ -214,8 +243,24 @@ def time_loop(fn, iters: int, warmup: int = 3):
     return t.ms() / iters
 
 
+def graph_of(fn, repeats: int):
+    """CUDA graph of `repeats` back-to-back calls of fn on a side stream (the device time per call without
+    the Python launch path, which at ~10 us per call would otherwise bound a 12 us kernel)."""
+    s = torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=s):
+            for _ in range(repeats):
+                fn()
+    return g, s
+
+
 def section_prefill(B, hbm_peak):
-    """Prefill forward; 16 buffer pairs (1 GiB) are rotated so every call misses L2."""
+    """Prefill forward; 16 buffer pairs (1 GiB) are rotated so every call misses L2.  Timed as a CUDA graph
+    of 64 calls (4 rounds over the buffers) replayed for about a second, and from a plain stream loop."""
     w = wl.CONFIGS["prefill"]
     a, b = (t.cuda() for t in wl.gen_params(w))
     x0 = wl.gen_full(w, "x").cuda()
@@ -234,15 +279,31 @@ def section_prefill(B, hbm_peak):
         state["i"] += 1
         B.wht_copy_rows(xs[i], ys[i], w.T, w.d, w.dtype)
 
-    ms = time_loop(call, 20 * nbuf, warmup=nbuf)
-    ms_copy = time_loop(copy, 20 * nbuf, warmup=nbuf)
-    warm = time_loop(lambda: B.wht_affine_fwd(xs[0], a, b, ys[0], w.T, w.d, w.dtype), 200, warmup=10)
+    def torch_copy():
+        i = state["i"] % nbuf
+        state["i"] += 1
+        ys[i].copy_(xs[i])
+
+    per_graph = 4 * nbuf
+    out = {"T": w.T, "d": w.d, "dtype": "bf16", "l2": "16 rotating buffer pairs (1 GiB)",
+           "timing": f"CUDA graph of {per_graph} calls replayed; stream_loop: plain Python launches"}
     gb = 2 * w.T * w.d * w.io_bytes / 1e9
-    return {"T": w.T, "d": w.d, "dtype": "bf16", "l2": "16 rotating buffer pairs (1 GiB)",
-            "fwd_us": 1e3 * ms, "fwd_tokens_per_s": w.T / (ms * 1e-3), "fwd_GBps": gb / (ms * 1e-3),
-            "fwd_frac_of_measured_peak": gb / (ms * 1e-3) / hbm_peak,
-            "fwd_frac_of_8000": gb / (ms * 1e-3) / 8000.0,
-            "copy_rows_GBps": gb / (ms_copy * 1e-3), "fwd_us_l2_warm": 1e3 * warm}
+    for key, fn in (("fwd", call), ("copy_rows", copy), ("torch_copy", torch_copy)):
+        g, s = graph_of(fn, per_graph)
+        with torch.cuda.stream(s):
+            burst = time_loop(g.replay, 1, warmup=1) / per_graph
+            reps = max(3, int(math.ceil((0.6 if key == "fwd" else 0.15) * 1e3 / (burst * per_graph))))
+            ms = time_loop(g.replay, reps, warmup=1) / per_graph
+        out[f"{key}_us"] = 1e3 * ms
+        out[f"{key}_GBps"] = gb / (ms * 1e-3)
+        if key == "fwd":
+            out["fwd_burst_us"] = 1e3 * burst
+    ms = out["fwd_us"] * 1e-3
+    out.update({"fwd_tokens_per_s": w.T / (ms * 1e-3), "fwd_frac_of_measured_peak": gb / (ms * 1e-3) / hbm_peak,
+                "fwd_frac_of_8000": gb / (ms * 1e-3) / 8000.0})
+    out["fwd_stream_loop_us"] = 1e3 * time_loop(call, 20 * nbuf, warmup=nbuf)
+    out["fwd_us_l2_warm"] = 1e3 * time_loop(lambda: B.wht_affine_fwd(xs[0], a, b, ys[0], w.T, w.d, w.dtype), 200, warmup=10)
+    return out
 
 
 def section_decode(B):
@@ -391,8 +452,28 @@ def section_other_shapes(B, hbm_peak):
     return out
 
 
-def section_fwd_bwd(B, name, hbm_peak, iters):
-    """Forward and backward timed separately on a workload larger than L2."""
+def burst_and_sustained(fn, min_seconds: float, gpu_index: int = 0):
+    """(burst ms, sustained ms, median SM MHz of the sustained loop): 30 launches after a one-second pause,
+    then a loop of at least `min_seconds` of device time."""
+    for _ in range(5):
+        fn()
+    torch.cuda.synchronize()
+    time.sleep(1.0)
+    burst = time_loop(fn, 30, warmup=0)
+    n = max(30, int(math.ceil(min_seconds * 1e3 / burst)))
+    sampler = ClockSampler(gpu_index)
+    sampler.start()
+    time.sleep(0.1)
+    t0 = time.time()
+    ms = time_loop(fn, n, warmup=0)
+    torch.cuda.synchronize()
+    t1 = time.time()
+    clk = ClockSampler.summarise(sampler.stop_all(), t0 + 0.2 * (t1 - t0), t1)
+    return burst, ms, clk["sm_mhz"]
+
+
+def section_fwd_bwd(B, name, hbm_peak, min_seconds):
+    """Forward and backward timed separately on a workload larger than L2: in a burst and sustained."""
     w = wl.CONFIGS[name]
     base_rows = min(w.T, 8192)
     a, b = (t.cuda() for t in wl.gen_params(w))
@@ -405,25 +486,29 @@ def section_fwd_bwd(B, name, hbm_peak, iters):
     y = torch.empty_like(x)
     da = torch.empty(w.d, dtype=torch.float32, device="cuda")
     db = torch.empty_like(da)
-    f_ms = time_loop(lambda: B.wht_affine_fwd(x, a, b, y, w.T, w.d, w.dtype), iters, warmup=10)
-    b_ms = time_loop(lambda: B.wht_affine_bwd(dy, x, a, y, da, db, w.T, w.d, w.dtype), iters, warmup=10)
-    c_ms = time_loop(lambda: B.wht_copy_rows(x, y, w.T, w.d, w.dtype), iters, warmup=10)
-    r_ms = time_loop(lambda: B.wht_affine_fwd_residual(x, a, b, dy, y, w.T, w.d, w.dtype), iters, warmup=10)
     fb = 2 * w.T * w.d * w.io_bytes / 1e9
     bb = 3 * w.T * w.d * w.io_bytes / 1e9
-    res = {"T": w.T, "d": w.d, "rows_drawn": base_rows, "rows_tiled": reps, "iters": iters, "warmup": 10,
-           "fwd_us": 1e3 * f_ms, "fwd_GBps": fb / (f_ms * 1e-3), "fwd_frac_of_measured_peak": fb / (f_ms * 1e-3) / hbm_peak,
-           "fwd_frac_of_8000": fb / (f_ms * 1e-3) / 8000.0, "fwd_tokens_per_s": w.T / (f_ms * 1e-3),
-           "bwd_us": 1e3 * b_ms, "bwd_GBps": bb / (b_ms * 1e-3), "bwd_frac_of_measured_peak": bb / (b_ms * 1e-3) / hbm_peak,
-           "bwd_frac_of_8000": bb / (b_ms * 1e-3) / 8000.0, "bwd_tokens_per_s": w.T / (b_ms * 1e-3),
-           "copy_rows_GBps": fb / (c_ms * 1e-3),
-           # forward fused with the residual add: reads x and the residual stream, writes y (3 row tensors)
-           "fwd_residual_us": 1e3 * r_ms, "fwd_residual_GBps": bb / (r_ms * 1e-3),
-           "fwd_residual_frac_of_measured_peak": bb / (r_ms * 1e-3) / hbm_peak}
+    res = {"T": w.T, "d": w.d, "rows_drawn": base_rows, "rows_tiled": reps,
+           "timing": f"burst: 30 launches after a pause; plain: a loop of >= {min_seconds:g} s"}
+    for which, fn, gb in (("fwd", lambda: B.wht_affine_fwd(x, a, b, y, w.T, w.d, w.dtype), fb),
+                          ("bwd", lambda: B.wht_affine_bwd(dy, x, a, y, da, db, w.T, w.d, w.dtype), bb)):
+        burst, ms, mhz = burst_and_sustained(fn, min_seconds)
+        res.update({f"{which}_us": 1e3 * ms, f"{which}_GBps": gb / (ms * 1e-3),
+                    f"{which}_frac_of_measured_peak": gb / (ms * 1e-3) / hbm_peak,
+                    f"{which}_frac_of_8000": gb / (ms * 1e-3) / 8000.0, f"{which}_tokens_per_s": w.T / (ms * 1e-3),
+                    f"{which}_sm_mhz": mhz, f"{which}_burst_us": 1e3 * burst,
+                    f"{which}_burst_frac_of_measured_peak": gb / (burst * 1e-3) / hbm_peak})
+    iters = 50
+    c_ms = time_loop(lambda: B.wht_copy_rows(x, y, w.T, w.d, w.dtype), iters, warmup=10)
+    r_ms = time_loop(lambda: B.wht_affine_fwd_residual(x, a, b, dy, y, w.T, w.d, w.dtype), iters, warmup=10)
+    res.update({"copy_rows_GBps": fb / (c_ms * 1e-3),
+                # forward fused with the residual add: reads x and the residual stream, writes y (3 row tensors)
+                "fwd_residual_us": 1e3 * r_ms, "fwd_residual_GBps": bb / (r_ms * 1e-3),
+                "fwd_residual_frac_of_measured_peak": bb / (r_ms * 1e-3) / hbm_peak})
     # the dense projection this path replaces, as context: cuBLAS bf16 [T x d] x [d x d]
     if w.dtype != wl.WHT_F32:
         wmat = torch.randn(w.d, w.d, device="cuda", dtype=torch.bfloat16)
-        g_ms = time_loop(lambda: torch.matmul(x, wmat, out=y), max(3, iters // 4))
+        g_ms = time_loop(lambda: torch.matmul(x, wmat, out=y), 12)
         res["dense_gemm_bf16_us"] = 1e3 * g_ms
         res["dense_gemm_tflops"] = 2.0 * w.T * w.d * w.d / (g_ms * 1e-3) / 1e12
     return res
@@ -492,36 +577,56 @@ def run_ours(args, rank: int, world: int, local_rank: int):
                 ev[2].record()
             bucket.all_reduce()  # the path's only exchange; nothing to do on one rank
 
-    for _ in range(max(args.warmup, 3)):
-        step()
-    torch.cuda.synchronize()
-    if world > 1:
-        dist.barrier()
+    def sync_all():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+
+    def max_over_ranks(ms: float) -> float:
+        if world == 1:
+            return ms
+        t = torch.tensor([ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    def timed(fn, n: int):
+        """n calls back to back between two CUDA events (nothing in between, so that each kernel may start
+        while its predecessor drains), barrier + synchronize on both sides, max over ranks; also the
+        wall-clock window for the clock samples."""
+        sync_all()
+        t0 = time.time()
+        with Timer() as t:
+            for _ in range(n):
+                fn()
+        ms = t.ms()
+        torch.cuda.synchronize()
+        t1 = time.time()
+        if world > 1:
+            dist.barrier()
+        return max_over_ranks(ms), (t0, t1)
+
+    def count_for(seconds: float, ms_per_call: float, at_least: int) -> int:
+        return max(at_least, int(math.ceil(seconds * 1e3 / max(ms_per_call, 1e-6))))
+
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
         time.sleep(0.3)
-    torch.cuda.synchronize()
-    # timed region: K steps back to back, one event on either side (nothing between the calls,
-    # so that each kernel may start while its predecessor drains)
-    t_wall0 = time.time()
-    with Timer() as total:
-        for k in range(args.steps):
-            step()
-    total_ms = total.ms()
-    torch.cuda.synchronize()
-    t_wall1 = time.time()
-    if world > 1:
-        dist.barrier()
-        tmax = torch.tensor([total_ms], device="cuda")
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        total_ms = float(tmax.item())
-    clocks_step = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
+    warm = max(args.warmup, 3)
+    for _ in range(warm):
+        step()
+    # 1. burst: K steps straight after the warm-up, the GPU still at its idle clocks and temperature
+    burst_ms, burst_win = timed(step, args.steps)
+    # 2. sustained: the same step repeated for at least --min-seconds of device time (the state a training
+    #    loop is in: the board's power limit has settled the SM clock) ...
+    n_long = count_for(args.min_seconds, burst_ms / args.steps, args.steps)
+    long_ms, long_win = timed(step, n_long)
+    # 3. ... and, with no pause, exactly K steps more: the headline figure (ms_per_step, value)
+    total_ms, head_win = timed(step, args.steps)
+    ms_per_step = total_ms / args.steps
+    value = world * w.T / (ms_per_step * 1e-3)
 
-    # per-call durations for the roofline figure: K launches of one call back to back between
-    # two events (sustained, launches overlapping as they do inside the step), and, for
-    # comparison, the same calls inside the step sequence with an event after every call
-    # (each event adds a few microseconds of idle front-end time to the call before it)
+    # per-call durations for the roofline figure: launches of one call back to back between two events
     def fwd_only():
         i = counter["i"] % nbuf
         counter["i"] += 1
@@ -532,34 +637,70 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         counter["i"] += 1
         B.wht_affine_bwd(dys[i], xs[i], a, dxs[i], da, db, w.T, w.d, w.dtype)
 
-    fwd_b2b_ms = time_loop(fwd_only, args.steps, warmup=3)
-    bwd_b2b_ms = time_loop(bwd_only, args.steps, warmup=3) if w.has_bwd else None
-    ev_steps = min(args.steps, 200)
+    def call_figures(fn, bytes_per_launch):
+        """Burst (after a one-second pause, 30 launches) and sustained (>= --min-seconds) time of one call."""
+        for _ in range(3):
+            fn()
+        sync_all()
+        time.sleep(1.0)
+        n_burst = 30
+        b_ms, b_win = timed(fn, n_burst)
+        n = count_for(args.min_seconds, b_ms / n_burst, n_burst)
+        l_ms, l_win = timed(fn, n)
+        return {"burst_ms": b_ms / n_burst, "burst_launches": n_burst, "burst_win": b_win,
+                "ms": l_ms / n, "launches": n, "win": l_win, "bytes": bytes_per_launch}
+
+    fwd_fig = call_figures(fwd_only, 2 * w.T * w.d * w.io_bytes)
+    bwd_fig = call_figures(bwd_only, 3 * w.T * w.d * w.io_bytes) if w.has_bwd else None
+    # the same calls inside the step sequence with an event after every call, for comparison
+    # (each event adds a few microseconds of idle front-end time to the call before it)
+    ev_steps = min(max(args.steps, 20), 200)
     events = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(ev_steps)]
     for k in range(ev_steps):
         step(events[k])
     torch.cuda.synchronize()
     fwd_ms = [e[0].elapsed_time(e[1]) for e in events]
     bwd_ms = [e[1].elapsed_time(e[2]) for e in events] if w.has_bwd else []
-    clocks = clocks_step
-    ms_per_step = total_ms / args.steps
-    value = world * w.T / (ms_per_step * 1e-3)
+    samples = sampler.stop_all() if rank == 0 else None
+
+    def clocks_in(win):
+        return ClockSampler.summarise(samples, *win) if samples is not None else None
+
+    def call_summary(fig):
+        gbps = fig["bytes"] / 1e9 / (fig["ms"] * 1e-3)
+        gbps_b = fig["bytes"] / 1e9 / (fig["burst_ms"] * 1e-3)
+        ck, ckb = clocks_in(fig["win"]), clocks_in(fig["burst_win"])
+        mhz = ck["sm_mhz"] if ck else None
+        return {"ms": fig["ms"], "launches": fig["launches"], "GBps": gbps, "frac_of_measured_peak": gbps / hbm_peak,
+                "frac_of_nominal_8000": gbps / 8000.0, "tokens_per_s": w.T / (fig["ms"] * 1e-3), "sm_mhz": mhz,
+                "us_x_mhz": fig["ms"] * 1e3 * mhz if mhz else None,
+                "burst": {"ms": fig["burst_ms"], "launches": fig["burst_launches"], "GBps": gbps_b,
+                          "frac_of_measured_peak": gbps_b / hbm_peak, "sm_mhz": ckb["sm_mhz"] if ckb else None}}
+
+    fwd_sum = call_summary(fwd_fig)
+    bwd_sum = call_summary(bwd_fig) if w.has_bwd else None
+    # the clock record of the headline: the sustained loop and the K timed steps that follow it without a pause
+    clocks = clocks_in((long_win[0], head_win[1])) if rank == 0 else None
+    if clocks is not None:
+        clocks["window"] = f"{n_long} steps of the sustained loop + the {args.steps} timed steps, back to back"
+        clocks["burst_steps"] = clocks_in(burst_win)
 
     # roofline of the dominant call: the backward call when there is one
-    if w.has_bwd:
-        dom, dom_ms = "wht_affine_bwd (main kernel + the small second pass)", bwd_b2b_ms
-        bytes_per_launch = 3 * w.T * w.d * w.io_bytes
-    else:
-        dom, dom_ms = "wht_affine_fwd", fwd_b2b_ms
-        bytes_per_launch = 2 * w.T * w.d * w.io_bytes
-    achieved = bytes_per_launch / 1e9 / (dom_ms * 1e-3)
-    traffic = NCU_TRAFFIC_BYTES.get((w.name, w.T))
-    roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": hbm_peak, "unit": "GB/s",
-                "frac": achieved / hbm_peak, "peak_source": peak_src, "traffic": traffic,
-                "algorithmic_bytes_per_launch": bytes_per_launch, "avg_launch_ms": dom_ms,
-                "timing": f"{args.steps} launches back to back between two CUDA events",
-                "frac_of_nominal_8000": achieved / 8000.0}
-    fwd_gbps = 2 * w.T * w.d * w.io_bytes / 1e9 / (fwd_b2b_ms * 1e-3)
+    dom_sum = bwd_sum if w.has_bwd else fwd_sum
+    dom_fig = bwd_fig if w.has_bwd else fwd_fig
+    dom = "wht_affine_bwd (main kernel + the small second pass)" if w.has_bwd else "wht_affine_fwd"
+    traffic, traffic_source = ncu_traffic(w.name, w.T) if w.has_bwd else (None, "no capture recorded for this call")
+    roofline = {"bound": "hbm", "kernel": dom, "achieved": dom_sum["GBps"], "peak": hbm_peak, "unit": "GB/s",
+                "frac": dom_sum["frac_of_measured_peak"], "frac_burst": dom_sum["burst"]["frac_of_measured_peak"],
+                "peak_source": peak_src, "traffic": traffic, "traffic_source": traffic_source,
+                "algorithmic_bytes_per_launch": dom_fig["bytes"], "avg_launch_ms": dom_sum["ms"],
+                "launches": dom_sum["launches"], "avg_launch_ms_burst": dom_sum["burst"]["ms"],
+                "sm_mhz": dom_sum["sm_mhz"], "sm_mhz_burst": dom_sum["burst"]["sm_mhz"], "us_x_mhz": dom_sum["us_x_mhz"],
+                "timing": f"frac: {dom_sum['launches']} launches back to back between two CUDA events (>= "
+                          f"{args.min_seconds:g} s: sustained, the board's power limit settles the SM clock); "
+                          f"frac_burst: {dom_sum['burst']['launches']} launches after a one-second pause",
+                "frac_of_nominal_8000": dom_sum["frac_of_nominal_8000"]}
+    fwd_b2b_ms = fwd_sum["ms"]
 
     # ---- end to end: pinned host buffers in, results back to the host, every step
     e2e = None
@@ -609,22 +750,26 @@ def run_ours(args, rank: int, world: int, local_rank: int):
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+        "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32",  # the arithmetic type; the storage types are in config.storage
         "data": "synthetic",
         "config": {"workload": w.name, "T_per_gpu": w.T, "d": w.d,
                    "storage": {0: "fp32", 1: "bf16 rows, bf16 params", 2: "bf16 rows, fp32 params"}[w.dtype],
                    "step": "wht_affine_fwd + wht_affine_bwd" if w.has_bwd else "wht_affine_fwd",
                    "l2": l2_note, "variant": B.wht_affine_get_variant(),
                    "parallelism": f"dp{world} (rows sharded; all-reduce of da|db only)" if world > 1 else "single GPU"},
-        "fwd": {"ms": fwd_b2b_ms, "GBps": fwd_gbps, "frac_of_measured_peak": fwd_gbps / hbm_peak,
-                "frac_of_nominal_8000": fwd_gbps / 8000.0, "tokens_per_s": w.T / (fwd_b2b_ms * 1e-3),
-                "ms_in_step_with_events": statistics.mean(fwd_ms)},
+        "fwd": dict(fwd_sum, ms_in_step_with_events=statistics.mean(fwd_ms)),
         "roofline": roofline, "e2e": e2e, "gpu_launches": launches_per_step * args.steps, "clocks": clocks,
+        # the same step: straight after the warm-up (burst), and over the long loop the headline follows
+        "burst": {"steps": args.steps, "ms_per_step": burst_ms / args.steps,
+                  "value": world * w.T / (burst_ms / args.steps * 1e-3)},
+        "sustained": {"steps": n_long, "ms_per_step": long_ms / n_long, "seconds": long_ms * 1e-3,
+                      "value": world * w.T / (long_ms / n_long * 1e-3)},
+        "timed_region": f"{warm} warm-up steps, {args.steps} steps (burst), {n_long} steps (sustained, >= "
+                        f"{args.min_seconds:g} s), then without a pause the {args.steps} steps of ms_per_step and value",
     }
     if w.has_bwd:
-        out["bwd"] = {"ms_in_step_with_events": statistics.mean(bwd_ms),
-                      "ms": dom_ms, "GBps": achieved, "frac_of_measured_peak": achieved / hbm_peak,
-                      "frac_of_nominal_8000": achieved / 8000.0, "tokens_per_s": w.T / (dom_ms * 1e-3)}
+        out["bwd"] = dict(bwd_sum, ms_in_step_with_events=statistics.mean(bwd_ms))
 
     # ---- CPU baseline: the oracle as it stands, on a bounded sample of the same workload
     # (a short pilot sizes it: up to 16384 rows per pass, passes until about 12 s of CPU work)
@@ -646,15 +791,42 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         sections["tiny"] = section_tiny(B)
         sections["prefill"] = section_prefill(B, hbm_peak)
         sections["decode"] = section_decode(B)
-        sections["training"] = section_fwd_bwd(B, "training", hbm_peak, 50)
-        sections["large"] = section_fwd_bwd(B, "large", hbm_peak, 50)
+        sections["training"] = section_fwd_bwd(B, "training", hbm_peak, args.min_seconds)
+        sections["large"] = section_fwd_bwd(B, "large", hbm_peak, args.min_seconds)
         sections["paper_shapes"] = section_paper_shapes(B, hbm_peak)
         sections["tensor_parallel_local"] = section_tensor_parallel_local(B, hbm_peak)
         sections["other_shapes"] = section_other_shapes(B, hbm_peak)
         out["sections"] = sections
-    print(json.dumps(out))
+        # the figures the target names, one line each: fraction of the measured copy bandwidth and of the
+        # nominal 8 TB/s ("burst" = 30 launches after a pause, plain = a loop of >= --min-seconds)
+        pc = {}
+        pf = sections["prefill"]
+        pc["prefill_fwd"] = {"us": pf["fwd_us"], "frac": pf["fwd_frac_of_measured_peak"], "frac_8000": pf["fwd_frac_of_8000"]}
+        for name in ("training", "large"):
+            sec = sections[name]
+            for which in ("fwd", "bwd"):
+                pc[f"{name}_{which}"] = {"us": sec[f"{which}_us"], "frac": sec[f"{which}_frac_of_measured_peak"],
+                                         "frac_8000": sec[f"{which}_frac_of_8000"], "sm_mhz": sec[f"{which}_sm_mhz"],
+                                         "burst_us": sec[f"{which}_burst_us"],
+                                         "burst_frac": sec[f"{which}_burst_frac_of_measured_peak"]}
+            pc[f"{name}_dense_gemm_us"] = sec.get("dense_gemm_bf16_us")
+        pc["decode_us_per_call"] = {k: {"graph": v["graph_replay_us_per_call"], "stream_loop": v["stream_loop_us_per_call"]}
+                                    for k, v in sections["decode"].items() if k.startswith("T")}
+        out["roofline"]["per_config"] = pc
+    print(json.dumps(compact(out)))
     if world > 1:
         dist.destroy_process_group()
+
+
+def compact(obj):
+    """Floats to 5 significant digits (the line is long; the driver keeps only its tail)."""
+    if isinstance(obj, float):
+        return float(f"{obj:.5g}")
+    if isinstance(obj, dict):
+        return {k: compact(v) for k, v in obj.items()}
+    if isinstance(obj, (list, tuple)):
+        return [compact(v) for v in obj]
+    return obj
 
 
 def main():
@@ -666,6 +838,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--variant", type=int, default=0)
     ap.add_argument("--no-sections", action="store_true")
+    ap.add_argument("--min-seconds", type=float, default=1.0,
+                    help="device time of the sustained loops (the step loop before the timed steps, and the "
+                         "per-call loops of the roofline figure)")
     ap.add_argument("--rows", type=int, default=0,
                     help="override the workload's row count (small cases for profiler captures; "
                          "not the benchmark configuration)")

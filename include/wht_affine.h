@@ -253,6 +253,26 @@ int wht_affine_set_variant(int variant);
 int wht_affine_get_variant(void);
 
 /*
+ * How g = (a/sqrt(d)) (.) dy enters the second +-1 tensor-core product of the tcgen05 backward
+ * (bf16 rows, 1024 <= d <= 8192; the other kernels ignore the setting):
+ *   0 = as a bf16 pair hi + lo (default): 16-17 significant bits, three products per tile;
+ *       dx is then the fp32-accumulated result rounded once at the store, up to the 2^-17 of the pair;
+ *   1 = rounded to bf16 once ("bf16-operand" mode): two products per tile, a third less
+ *       tensor-core work and less register and shared-memory work, which in long runs under
+ *       the board's power limit is what sets the speed of the backward.  Every one of the 128
+ *       terms of a product then carries a 2^-9 rounding: dx is off by about 1e-3 of a row's typical
+ *       magnitude (the same size as the bf16 rounding of dx itself, and inside the 1e-2 * max|dx_row|
+ *       bound of this library's tests even for spike-dominated rows), but it is no longer the
+ *       correctly rounded fp32 result.  da and db do not pass through g and are bit-identical
+ *       in both modes.
+ * The chain rule on Eq. 1 fixes dx = ((a (.) dy) H)/sqrt(d); the paper says nothing about the
+ * precision of its intermediates beyond "bf16 mixed precision", so both modes are readings of it.
+ * Process-wide; not meant to be changed while calls are in flight.  Unknown mode -> WHT_ERR_BAD_VARIANT.
+ */
+int wht_affine_set_bwd_operand_mode(int mode);
+int wht_affine_get_bwd_operand_mode(void);
+
+/*
  * Bandwidth yardstick with the same access pattern as the forward pass: copies
  * T rows of d elements (element size from dtype) from src to dst.  Used only by
  * the benchmark to report a practical copy ceiling next to the kernels.

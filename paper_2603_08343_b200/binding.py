@@ -22,6 +22,7 @@ EXPORTS = (
     "wht_affine_fwd_grouped", "wht_affine_bwd_grouped", "wht_affine_bwd_grouped_workspace_bytes",
     "wht_affine_fwd_tp", "wht_affine_bwd_tp", "wht_affine_bwd_tp_workspace_bytes",
     "wht_affine_bwd_workspace_bytes", "wht_affine_set_variant", "wht_affine_get_variant",
+    "wht_affine_set_bwd_operand_mode", "wht_affine_get_bwd_operand_mode",
     "wht_copy_rows", "wht_affine_device_status", "wht_affine_last_cuda_error", "wht_affine_status_string",
     "wht_affine_shutdown",
 )
@@ -61,6 +62,8 @@ def _load() -> ctypes.CDLL:
     lib.wht_affine_bwd_workspace_bytes.restype = sz
     lib.wht_affine_set_variant.argtypes = [ci]
     lib.wht_affine_get_variant.argtypes = []
+    lib.wht_affine_set_bwd_operand_mode.argtypes = [ci]
+    lib.wht_affine_get_bwd_operand_mode.argtypes = []
     lib.wht_copy_rows.argtypes = [vp, vp, i64, i32, ci, vp]
     lib.wht_affine_device_status.argtypes = []
     lib.wht_affine_last_cuda_error.argtypes = []
@@ -216,6 +219,15 @@ def wht_affine_set_variant(variant: int) -> None:
 
 def wht_affine_get_variant() -> int:
     return int(_lib.wht_affine_get_variant())
+
+
+def wht_affine_set_bwd_operand_mode(mode: int) -> None:
+    """0: g enters the tcgen05 backward's second product as a bf16 pair hi + lo (default); 1: rounded to bf16."""
+    _check(_lib.wht_affine_set_bwd_operand_mode(mode), "wht_affine_set_bwd_operand_mode")
+
+
+def wht_affine_get_bwd_operand_mode() -> int:
+    return int(_lib.wht_affine_get_bwd_operand_mode())
 
 
 def wht_copy_rows(src, dst, T: int, d: int, dtype: int, stream=None) -> None:

@@ -375,37 +375,4 @@ bfly_bwd_kernel(const TIO* dy, const TIO* x, const TP* __restrict__ a, TIO* dx,
     }
 }
 
-// ---- second pass: da[j] = inv_sqrt_d * sum_p partials[p][0][j], db[j] likewise --
-__global__ void __launch_bounds__(256)
-dadb_finalize_kernel(const float* __restrict__ partials, int nparts, int d, float inv_sqrt_d,
-                     float* __restrict__ da, float* __restrict__ db) {
-    grid_dependency_wait();  // the partials come from the kernel launched just before
-    grid_launch_dependents();
-    const int j = blockIdx.x * blockDim.x + threadIdx.x;
-    if (j >= 2 * d) return;
-    const int which = j / d;
-    const int col = j - which * d;
-    const float* src = partials + static_cast<size_t>(which) * d + col;
-    const size_t stride = static_cast<size_t>(2) * d;
-    float s0 = 0.0f, s1 = 0.0f, s2 = 0.0f, s3 = 0.0f;
-    int p = 0;
-    for (; p + 4 <= nparts; p += 4) {
-        s0 += src[(p + 0) * stride];
-        s1 += src[(p + 1) * stride];
-        s2 += src[(p + 2) * stride];
-        s3 += src[(p + 3) * stride];
-    }
-    for (; p < nparts; ++p) s0 += src[p * stride];
-    const float s = (s0 + s1) + (s2 + s3);
-    if (which == 0) da[col] = s * inv_sqrt_d; else db[col] = s;
-}
-
-// ---- bandwidth yardstick: copy rows with the forward pass's access pattern ----
-__global__ void __launch_bounds__(256)
-copy_rows_kernel(const uint4* src, uint4* dst, long long n16) {
-    const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
-    for (long long i = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; i < n16; i += stride)
-        __stcs(dst + i, __ldcs(src + i));
-}
-
 }  // namespace wht

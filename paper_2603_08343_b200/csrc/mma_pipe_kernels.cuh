@@ -13,8 +13,9 @@
 
 namespace wht {
 
-// set to a non-zero code by a kernel whose bounded wait expired
-__device__ unsigned int g_wht_device_error = 0;
+// set to a non-zero code by a kernel whose bounded wait expired (one word per translation unit of the
+// library; the host reads and clears each of them)
+static __device__ unsigned int g_wht_device_error = 0;
 constexpr unsigned int kDeviceErrWaitExpired = 1;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -308,34 +309,6 @@ mma_bwd_pipe_kernel(const __nv_bfloat16* dy, const __nv_bfloat16* x, const TP* _
         if (++stage == S) { stage = 0; phase ^= 1; }
     }
     bwd_publish_partials<Geo>(da_acc, db_acc, reinterpret_cast<float*>(smem_raw), partials, rg, w, lane);
-}
-
-// ---- second pass of the backward, parallel over slices of the partials -------------
-// block = 32 columns x 32 slices; slice s adds partials s, s+32, ... in order, then
-// the 32 slice sums are added in order: a fixed association, bit-reproducible.
-__global__ void __launch_bounds__(1024)
-dadb_finalize32_kernel(const float* __restrict__ partials, int nparts, int d, float inv_sqrt_d,
-                       float* __restrict__ da, float* __restrict__ db) {
-    __shared__ float red[32][33];
-    grid_dependency_wait();  // the partials come from the kernel launched just before
-    grid_launch_dependents();
-    const int cx = threadIdx.x & 31;
-    const int sl = threadIdx.x >> 5;
-    const int j = blockIdx.x * 32 + cx;  // column in [0, 2d): da columns then db columns
-    const int which = j / d;
-    const int col = j - which * d;
-    const size_t stride = static_cast<size_t>(2) * d;
-    const float* src = partials + static_cast<size_t>(which) * d + col;
-    float s = 0.0f;
-    for (int p = sl; p < nparts; p += 32) s += src[p * stride];
-    red[sl][cx] = s;
-    __syncthreads();
-    if (sl == 0) {
-        float t = 0.0f;
-#pragma unroll
-        for (int k = 0; k < 32; ++k) t += red[k][cx];
-        if (which == 0) da[col] = t * inv_sqrt_d; else db[col] = t;
-    }
 }
 
 }  // namespace wht

@@ -212,6 +212,10 @@ __host__ __device__ constexpr uint32_t umma_idesc(int n) {
 // Instruction-descriptor bit that multiplies by -A instead of A.
 constexpr int kUmmaNegateABit = 13;
 
+// compile-time booleans passed to generic lambdas
+struct TrueTag { static constexpr bool value = true; };
+struct FalseTag { static constexpr bool value = false; };
+
 template <int LOGD, int NCOL_>
 struct UmmaGeo {
     static constexpr int D = 1 << LOGD;
@@ -607,7 +611,13 @@ struct UmmaBwdSmem {
 
 // partials layout: [gridDim.x][2][D] fp32; slot 0: sum_t dy (.) (x H) WITHOUT the
 // 1/sqrt(d) factor (the second pass applies it), slot 1: sum_t dy.
-template <int LOGD, int NCOL, int STAGES, typename TP, bool A_TMEM = false>
+//
+// G_LO = false ("bf16-operand" mode of the backward): g is rounded to bf16 once before the second product
+// instead of being carried as hi + lo, so a tile costs two products instead of three and the lo half of
+// the register work and of the shared-memory writes goes away.  dx then carries the 2^-9 rounding of
+// each of the 128 terms of a product (about 1e-3 of a row's typical dx, far inside the 1e-2 bound, but
+// no longer "one rounding at the store"); da and db do not pass through g and are unchanged.
+template <int LOGD, int NCOL, int STAGES, typename TP, bool A_TMEM = false, bool G_LO = true>
 __global__ void __launch_bounds__(UmmaGeo<LOGD, NCOL>::THREADS, 1)
 umma_bwd_kernel(const __nv_bfloat16* dy, const __nv_bfloat16* x, const TP* __restrict__ a, __nv_bfloat16* dx,
                 float* __restrict__ partials, long long T, float inv_sqrt_d) {
@@ -766,12 +776,14 @@ umma_bwd_kernel(const __nv_bfloat16* dy, const __nv_bfloat16* x, const TP* __res
                     else
                         umma_bf16(tmem_d2 + t * Geo::N, adesc + k * 16, bhi + k * 16, idesc, k > 0);
                 }
+                if constexpr (G_LO) {
 #pragma unroll
-                for (int k = 0; k < 8; ++k) {
-                    if constexpr (A_TMEM)
-                        umma_bf16_a_tmem(tmem_d2 + t * Geo::N, tmem_a + k * 8, blo + k * 16, idesc, 1);
-                    else
-                        umma_bf16(tmem_d2 + t * Geo::N, adesc + k * 16, blo + k * 16, idesc, 1);
+                    for (int k = 0; k < 8; ++k) {
+                        if constexpr (A_TMEM)
+                            umma_bf16_a_tmem(tmem_d2 + t * Geo::N, tmem_a + k * 8, blo + k * 16, idesc, 1);
+                        else
+                            umma_bf16(tmem_d2 + t * Geo::N, adesc + k * 16, blo + k * 16, idesc, 1);
+                    }
                 }
                 umma_commit(d2_full + t);
                 umma_commit(stage_empty + s);
@@ -851,23 +863,29 @@ umma_bwd_kernel(const __nv_bfloat16* dy, const __nv_bfloat16* x, const TP* __res
             long long row0;
             const int nvalid = rows_in_tile(j, row0);
             uint4* const dst0 = reinterpret_cast<uint4*>(dx_thr + row0 * Geo::D);
+            // FULL: every row of the tile exists (all tiles but the last one of a ragged problem): no
+            // per-row test, so the rows stay one straight instruction stream
+            auto store_rows = [&](auto full_tag) {
+                constexpr bool FULL = decltype(full_tag)::value;
 #pragma unroll(ROW_UNROLL)
-            for (int r = 0; r < NROW; ++r) {
-                const int rt = SPLIT ? r : ch * Geo::RPW + r;  // row inside the tile
-                if (rt < nvalid) {                              // uniform over the warp
-                    float w[RE];
-                    row_values(acc, r, w, u);
+                for (int r = 0; r < NROW; ++r) {
+                    const int rt = SPLIT ? r : ch * Geo::RPW + r;  // row inside the tile
+                    if (FULL || rt < nvalid) {                      // uniform over the warp
+                        float w[RE];
+                        row_values(acc, r, w, u);
 #pragma unroll
-                    for (int p = 0; p < PE; ++p) {
-                        uint4 o;
-                        o.x = pack_bf16x2(w[p * 8 + 0], w[p * 8 + 1]);
-                        o.y = pack_bf16x2(w[p * 8 + 2], w[p * 8 + 3]);
-                        o.z = pack_bf16x2(w[p * 8 + 4], w[p * 8 + 5]);
-                        o.w = pack_bf16x2(w[p * 8 + 6], w[p * 8 + 7]);
-                        __stcs(dst0 + rt * (Geo::D / 8) + p * 128, o);
+                        for (int p = 0; p < PE; ++p) {
+                            uint4 o;
+                            o.x = pack_bf16x2(w[p * 8 + 0], w[p * 8 + 1]);
+                            o.y = pack_bf16x2(w[p * 8 + 2], w[p * 8 + 3]);
+                            o.z = pack_bf16x2(w[p * 8 + 4], w[p * 8 + 5]);
+                            o.w = pack_bf16x2(w[p * 8 + 6], w[p * 8 + 7]);
+                            __stcs(dst0 + rt * (Geo::D / 8) + p * 128, o);
+                        }
                     }
                 }
-            }
+            };
+            if (nvalid == Geo::ROWS) store_rows(TrueTag{}); else store_rows(FalseTag{});
             if constexpr (SPLIT) {
                 tc_fence_before();
                 __syncwarp();
@@ -902,13 +920,16 @@ umma_bwd_kernel(const __nv_bfloat16* dy, const __nv_bfloat16* x, const TP* __res
             unsigned char* const cdy = cx + Geo::TILE_BYTES;
             long long row0;
             const int nvalid = rows_in_tile(it, row0);
+            // Rows past T were never copied: their accumulator columns and slot bytes hold
+            // whatever was there before.  They are skipped altogether (uniformly over the
+            // warp); the second product then reads stale columns for them, which nobody stores.
+            // FULL (every row of the tile exists) drops the per-row test.
+            auto tile_rows = [&](auto full_tag) {
+            constexpr bool FULL = decltype(full_tag)::value;
 #pragma unroll(ROW_UNROLL)
             for (int r = 0; r < NROW; ++r) {
                 const int rt = SPLIT ? r : ch * Geo::RPW + r;  // row inside the tile
-                // Rows past T were never copied: their accumulator columns and slot bytes hold
-                // whatever was there before.  They are skipped altogether (uniformly over the
-                // warp); the second product then reads stale columns for them, which nobody stores.
-                if (rt < nvalid) {
+                if (FULL || rt < nvalid) {
                     float v[RE];
                     row_values(acc, r, v, u);
                     thread_stages<RE>(v);  // v = (x H) at this thread's channels, unnormalised
@@ -930,17 +951,28 @@ umma_bwd_kernel(const __nv_bfloat16* dy, const __nv_bfloat16* x, const TP* __res
                     thread_stages<RE>(g);  // the register stages of the second transform
 #pragma unroll
                     for (int p = 0; p < PE; ++p) {
-                        uint4 hi, lo;
-                        split_hi_lo(f2(g[p * 8 + 0], g[p * 8 + 1]), hi.x, lo.x);
-                        split_hi_lo(f2(g[p * 8 + 2], g[p * 8 + 3]), hi.y, lo.y);
-                        split_hi_lo(f2(g[p * 8 + 4], g[p * 8 + 5]), hi.z, lo.z);
-                        split_hi_lo(f2(g[p * 8 + 6], g[p * 8 + 7]), hi.w, lo.w);
                         // the x tile is consumed (D1 is complete); this thread alone read this dy chunk
-                        *reinterpret_cast<uint4*>(cx + (rt * Geo::PIECES + p) * 2048) = hi;
-                        *reinterpret_cast<uint4*>(cdy + (rt * Geo::PIECES + p) * 2048) = lo;
+                        if constexpr (G_LO) {
+                            uint4 hi, lo;
+                            split_hi_lo(f2(g[p * 8 + 0], g[p * 8 + 1]), hi.x, lo.x);
+                            split_hi_lo(f2(g[p * 8 + 2], g[p * 8 + 3]), hi.y, lo.y);
+                            split_hi_lo(f2(g[p * 8 + 4], g[p * 8 + 5]), hi.z, lo.z);
+                            split_hi_lo(f2(g[p * 8 + 6], g[p * 8 + 7]), hi.w, lo.w);
+                            *reinterpret_cast<uint4*>(cx + (rt * Geo::PIECES + p) * 2048) = hi;
+                            *reinterpret_cast<uint4*>(cdy + (rt * Geo::PIECES + p) * 2048) = lo;
+                        } else {
+                            uint4 hi;
+                            hi.x = pack_bf16x2(g[p * 8 + 0], g[p * 8 + 1]);
+                            hi.y = pack_bf16x2(g[p * 8 + 2], g[p * 8 + 3]);
+                            hi.z = pack_bf16x2(g[p * 8 + 4], g[p * 8 + 5]);
+                            hi.w = pack_bf16x2(g[p * 8 + 6], g[p * 8 + 7]);
+                            *reinterpret_cast<uint4*>(cx + (rt * Geo::PIECES + p) * 2048) = hi;
+                        }
                     }
                 }
             }
+            };
+            if (nvalid == Geo::ROWS) tile_rows(TrueTag{}); else tile_rows(FalseTag{});
             if constexpr (SPLIT) {
                 tc_fence_before();
                 __syncwarp();

@@ -579,6 +579,40 @@ def test_outputs_are_the_correctly_rounded_values_almost_everywhere(B, variant):
         assert worst <= 1.0, f"{what} v{variant}: an output is {worst:.2f}x beyond half a bf16 step + {slack:g}*max|row|"
 
 
+# ------------------------------------------------------------------ bf16-operand mode of the tcgen05 backward
+
+@pytest.mark.parametrize("name,rows", [("training", 148 * 8 * 2 + 3), ("large", 148 * 2 * 2 + 1), ("prefill", 148 * 16 + 5)])
+def test_bwd_bf16_operand_mode(B, name, rows):
+    """wht_affine_set_bwd_operand_mode(1): g = (a/sqrt d) (.) dy is rounded to bf16 once before the second
+    +-1 product.  dx must still meet the bound for bf16 storage, 1e-2 * max|dx_row|, on every row of the
+    chain rule of Eq. 1 -- also on the heavy-tailed rows of the Large config, where one spike dominates a
+    row -- and da, db (which never pass through g) must keep the bits of the default mode."""
+    B.wht_affine_set_variant(0)
+    base = wl.CONFIGS[name]
+    w = wl.Workload(base.name, rows, base.d, base.dtype, base.dist, base.seed + 7, True, "")
+    x, dy = wl.gen_full(w, "x"), wl.gen_full(w, "dy")
+    a, _ = wl.gen_params(w)
+    xd, dyd, ad = x.cuda(), dy.cuda(), a.cuda()
+    dx0, da0, db0 = B.backward(dyd, xd, ad)
+    assert B.wht_affine_get_bwd_operand_mode() == 0
+    B.wht_affine_set_bwd_operand_mode(1)
+    try:
+        dx1, da1, db1 = B.backward(dyd, xd, ad)
+        torch.cuda.synchronize()
+    finally:
+        B.wht_affine_set_bwd_operand_mode(0)
+    ref_dx, ref_da, ref_db = oracle.wht_affine_bwd(to_f64(dy), to_f64(x), to_f64(a))
+    worst1 = assert_rows_bf16(to_f64(dx1.cpu()), ref_dx, f"{name} dx, bf16-operand mode")
+    worst0 = assert_rows_bf16(to_f64(dx0.cpu()), ref_dx, f"{name} dx, default mode")
+    assert worst1 <= 0.5, f"{name}: the bf16-operand mode uses {worst1:.2f} of the bound (default {worst0:.2f})"
+    assert torch.equal(da0, da1) and torch.equal(db0, db1)
+    assert_grad_vec(to_f64(da1.cpu()), ref_da, f"{name} da, bf16-operand mode")
+    assert_grad_vec(to_f64(db1.cpu()), ref_db, f"{name} db, bf16-operand mode")
+    with pytest.raises(B.WhtError):
+        B.wht_affine_set_bwd_operand_mode(2)
+    B.wht_affine_device_status()
+
+
 # ------------------------------------------------------------------ grouped (block-diagonal) form
 
 @pytest.mark.parametrize("d,block,dtype,T", [(768, 256, wl.WHT_F32, 70), (768, 256, wl.WHT_BF16, 300),
