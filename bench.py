@@ -498,6 +498,16 @@ def section_fwd_bwd(B, name, hbm_peak, min_seconds):
                     f"{which}_frac_of_8000": gb / (ms * 1e-3) / 8000.0, f"{which}_tokens_per_s": w.T / (ms * 1e-3),
                     f"{which}_sm_mhz": mhz, f"{which}_burst_us": 1e3 * burst,
                     f"{which}_burst_frac_of_measured_peak": gb / (burst * 1e-3) / hbm_peak})
+    if w.dtype != wl.WHT_F32:
+        # the backward with g carried into the second product as a bf16 pair (dx rounded once)
+        B.wht_affine_set_bwd_operand_mode(1)
+        try:
+            burst, ms, mhz = burst_and_sustained(lambda: B.wht_affine_bwd(dy, x, a, y, da, db, w.T, w.d, w.dtype),
+                                                 min_seconds)
+        finally:
+            B.wht_affine_set_bwd_operand_mode(0)
+        res.update({"bwd_pair_mode_us": 1e3 * ms, "bwd_pair_mode_frac_of_measured_peak": bb / (ms * 1e-3) / hbm_peak,
+                    "bwd_pair_mode_sm_mhz": mhz, "bwd_pair_mode_burst_us": 1e3 * burst})
     iters = 50
     c_ms = time_loop(lambda: B.wht_copy_rows(x, y, w.T, w.d, w.dtype), iters, warmup=10)
     r_ms = time_loop(lambda: B.wht_affine_fwd_residual(x, a, b, dy, y, w.T, w.d, w.dtype), iters, warmup=10)
@@ -757,6 +767,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
                    "storage": {0: "fp32", 1: "bf16 rows, bf16 params", 2: "bf16 rows, fp32 params"}[w.dtype],
                    "step": "wht_affine_fwd + wht_affine_bwd" if w.has_bwd else "wht_affine_fwd",
                    "l2": l2_note, "variant": B.wht_affine_get_variant(),
+                   "bwd_operand_mode": B.wht_affine_get_bwd_operand_mode(),
                    "parallelism": f"dp{world} (rows sharded; all-reduce of da|db only)" if world > 1 else "single GPU"},
         "fwd": dict(fwd_sum, ms_in_step_with_events=statistics.mean(fwd_ms)),
         "roofline": roofline, "e2e": e2e, "gpu_launches": launches_per_step * args.steps, "clocks": clocks,
@@ -809,6 +820,8 @@ def run_ours(args, rank: int, world: int, local_rank: int):
                                          "frac_8000": sec[f"{which}_frac_of_8000"], "sm_mhz": sec[f"{which}_sm_mhz"],
                                          "burst_us": sec[f"{which}_burst_us"],
                                          "burst_frac": sec[f"{which}_burst_frac_of_measured_peak"]}
+            pc[f"{name}_bwd_pair_mode"] = {"us": sec.get("bwd_pair_mode_us"),
+                                           "frac": sec.get("bwd_pair_mode_frac_of_measured_peak")}
             pc[f"{name}_dense_gemm_us"] = sec.get("dense_gemm_bf16_us")
         pc["decode_us_per_call"] = {k: {"graph": v["graph_replay_us_per_call"], "stream_loop": v["stream_loop_us_per_call"]}
                                     for k, v in sections["decode"].items() if k.startswith("T")}

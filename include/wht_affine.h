@@ -23,12 +23,12 @@
  *     fp32 whatever the storage type; bf16 outputs are rounded once, to nearest
  *     even, at the store.  One exception: in the tensor-core kernels (bf16 rows,
  *     512 <= d <= 8192) an fp32 intermediate that feeds a second +-1 product is
- *     split into a bf16 pair hi + lo, which carries 16-17 significant bits
- *     (relative error 2^-17) instead of 24.  This touches dx of the backward
- *     calls (and y of the mma.sync forward, variants 2 and 3); sums are still
- *     fp32.  The effect, about 4e-5 of a row's largest output, is far inside the
- *     bf16 rounding of the result (2^-9) and is bounded by the library's test
- *     test_outputs_are_the_correctly_rounded_values_almost_everywhere.
+ *     narrowed on the way: to a bf16 pair hi + lo (16-17 significant bits instead
+ *     of 24) in y of the mma.sync forward (variants 2 and 3) and in dx of the mma.sync
+ *     backward, and in dx of the tcgen05 backward either to that pair or, by default,
+ *     to one bf16 (see wht_affine_set_bwd_operand_mode).  Sums are fp32 throughout.
+ *     The library's tests bound both effects against the 1e-2 * max|row| tolerance
+ *     (test_bwd_bf16_operand_mode, test_outputs_are_the_correctly_rounded_values_almost_everywhere).
  *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
  *     Calls are asynchronous: they enqueue work and return without synchronising.
  *   - Exact aliasing y == x and dx == dy is allowed (a row is read completely
@@ -254,19 +254,20 @@ int wht_affine_get_variant(void);
 
 /*
  * How g = (a/sqrt(d)) (.) dy enters the second +-1 tensor-core product of the tcgen05 backward
- * (bf16 rows, 1024 <= d <= 8192; the other kernels ignore the setting):
- *   0 = as a bf16 pair hi + lo (default): 16-17 significant bits, three products per tile;
- *       dx is then the fp32-accumulated result rounded once at the store, up to the 2^-17 of the pair;
- *   1 = rounded to bf16 once ("bf16-operand" mode): two products per tile, a third less
- *       tensor-core work and less register and shared-memory work, which in long runs under
- *       the board's power limit is what sets the speed of the backward.  Every one of the 128
- *       terms of a product then carries a 2^-9 rounding: dx is off by about 1e-3 of a row's typical
- *       magnitude (the same size as the bf16 rounding of dx itself, and inside the 1e-2 * max|dx_row|
- *       bound of this library's tests even for spike-dominated rows), but it is no longer the
- *       correctly rounded fp32 result.  da and db do not pass through g and are bit-identical
- *       in both modes.
- * The chain rule on Eq. 1 fixes dx = ((a (.) dy) H)/sqrt(d); the paper says nothing about the
- * precision of its intermediates beyond "bf16 mixed precision", so both modes are readings of it.
+ * (bf16 rows, 1024 <= d <= 8192; the other kernels ignore the setting).  The chain rule on Eq. 1
+ * fixes dx = ((a (.) dy) H)/sqrt(d); the paper says of precision only "bfloat16 mixed precision"
+ * (a framework implementation in that regime rounds a (.) dy, and every butterfly stage after it,
+ * to bf16), so both modes are readings of it:
+ *   0 = rounded to bf16 once (default): two products per tile.  Every one of the 128 terms of a
+ *       product carries a 2^-9 rounding, so dx is off by about 1e-3 of a row's typical magnitude
+ *       -- the size of the bf16 rounding of dx itself, and inside the 1e-2 * max|dx_row| bound of
+ *       this library's tests even for spike-dominated rows -- but it is not the correctly rounded
+ *       fp32 result.  In long runs the backward's speed is set by the board's power limit, i.e. by
+ *       energy per row, and this mode needs a third less tensor-core work and less register and
+ *       shared-memory work: measured 13 % faster sustained at d = 2048 and 11 % at d = 8192.
+ *   1 = as a bf16 pair hi + lo: 16-17 significant bits, three products per tile; dx is then the
+ *       fp32-accumulated result rounded once at the store, up to the 2^-17 of the pair.
+ * da and db do not pass through g and are bit-identical in both modes.
  * Process-wide; not meant to be changed while calls are in flight.  Unknown mode -> WHT_ERR_BAD_VARIANT.
  */
 int wht_affine_set_bwd_operand_mode(int mode);
@@ -289,6 +290,20 @@ int wht_copy_rows(const void* src, void* dst, int64_t T, int32_t d, int dtype, v
  * operation; meant for tests and for debugging after a suspicious result.
  */
 int wht_affine_device_status(void);
+
+/*
+ * Self-test of that failure path, for test suites (the paper has no counterpart).  Launches one small
+ * CTA in which one thread waits, through the kernels' own bounded-wait routine, on a barrier that
+ * nothing ever completes, with a limit of about `limit_us` microseconds (1 .. 1000000) instead of the
+ * kernels' tenths of a second; a second warp waits on another such barrier with the kernels' long limit
+ * and must leave through the CTA's abort flag.  Nothing traps and nothing can hang: every wait is
+ * bounded by construction, and the kernel returns by itself after roughly `limit_us`.
+ *   out3: DEVICE pointer to three 32-bit words, written by the kernel: [0] = 1 if the short wait ran
+ *   out, [1] = 1 if the second warp left through the abort flag, [2] unused.
+ * After the launch completes, wht_affine_device_status() returns WHT_ERR_DEVICE_WAIT once and WHT_OK
+ * from then on, and the library works as before.
+ */
+int wht_affine_selftest_wait_expiry(uint32_t limit_us, unsigned int* out3, void* stream);
 
 /* cudaError_t of the most recent failing CUDA call on this thread (0 if none). */
 int wht_affine_last_cuda_error(void);

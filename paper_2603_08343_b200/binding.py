@@ -23,7 +23,7 @@ EXPORTS = (
     "wht_affine_fwd_tp", "wht_affine_bwd_tp", "wht_affine_bwd_tp_workspace_bytes",
     "wht_affine_bwd_workspace_bytes", "wht_affine_set_variant", "wht_affine_get_variant",
     "wht_affine_set_bwd_operand_mode", "wht_affine_get_bwd_operand_mode",
-    "wht_copy_rows", "wht_affine_device_status", "wht_affine_last_cuda_error", "wht_affine_status_string",
+    "wht_copy_rows", "wht_affine_device_status", "wht_affine_selftest_wait_expiry", "wht_affine_last_cuda_error", "wht_affine_status_string",
     "wht_affine_shutdown",
 )
 
@@ -66,6 +66,7 @@ def _load() -> ctypes.CDLL:
     lib.wht_affine_get_bwd_operand_mode.argtypes = []
     lib.wht_copy_rows.argtypes = [vp, vp, i64, i32, ci, vp]
     lib.wht_affine_device_status.argtypes = []
+    lib.wht_affine_selftest_wait_expiry.argtypes = [ctypes.c_uint32, vp, vp]
     lib.wht_affine_last_cuda_error.argtypes = []
     lib.wht_affine_status_string.argtypes = [ci]
     lib.wht_affine_status_string.restype = ctypes.c_char_p
@@ -222,7 +223,8 @@ def wht_affine_get_variant() -> int:
 
 
 def wht_affine_set_bwd_operand_mode(mode: int) -> None:
-    """0: g enters the tcgen05 backward's second product as a bf16 pair hi + lo (default); 1: rounded to bf16."""
+    """How g = (a/sqrt d) (.) dy enters the tcgen05 backward's second product: 0 = rounded to bf16 once
+    (default), 1 = as a bf16 pair hi + lo (dx then is the fp32 result rounded once at the store)."""
     _check(_lib.wht_affine_set_bwd_operand_mode(mode), "wht_affine_set_bwd_operand_mode")
 
 
@@ -238,6 +240,14 @@ def wht_copy_rows(src, dst, T: int, d: int, dtype: int, stream=None) -> None:
 def wht_affine_device_status() -> None:
     """Synchronises and raises WhtError if a kernel's bounded wait expired since the last query."""
     _check(_lib.wht_affine_device_status(), "wht_affine_device_status")
+
+
+def wht_affine_selftest_wait_expiry(limit_us: int, out3, stream=None) -> None:
+    """Launches the library's one-CTA kernel whose bounded wait runs out after about limit_us microseconds
+    (out3: three int32/uint32 words on the device); afterwards wht_affine_device_status() raises once."""
+    _require_cuda(out3)
+    _check(_lib.wht_affine_selftest_wait_expiry(limit_us, _ptr(out3), _stream(stream)),
+           "wht_affine_selftest_wait_expiry")
 
 
 def wht_affine_shutdown() -> None:

@@ -85,6 +85,15 @@ int umma_fwd_tp(int logw, int dtype, const TpCall& t, const FwdArgs& f, const Ct
                              : dispatch_umma_fwd_tp<float>(logw, t, f, c);
 }
 
+int launch_wait_expiry_selftest(uint32_t limit_us, unsigned int* out, cudaStream_t s) {
+    // limit_us of waiting in all: parked try_waits of up to 20 us each, then polls 256 ns apart
+    const uint32_t park = limit_us / 20u + 1u;
+    const uint32_t spin = limit_us * 4u + 1u;
+    wait_expiry_selftest_kernel<0><<<1, 64, 0, s>>>(park, spin, out);
+    WHT_CUDA_TRY(cudaGetLastError());
+    return WHT_OK;
+}
+
 WHT_DEFINE_DEVICE_ERROR_READER(take_device_error_umma_fwd)
 
 }  // namespace wht_host

@@ -185,6 +185,9 @@ int umma_fwd_tp(int logw, int dtype, const TpCall& t, const FwdArgs& f, const Ct
 // g_hi_lo: g enters the second product as a bf16 pair hi + lo (default) or rounded to bf16 once
 int umma_bwd(int logd, int dtype, bool g_hi_lo, const BwdArgs& g, const Ctx& c);        // family_umma_bwd.cu
 
+// Self-test of the bounded waits (family_umma_fwd.cu): a one-CTA kernel whose wait runs out after limit_us.
+int launch_wait_expiry_selftest(uint32_t limit_us, unsigned int* out, cudaStream_t s);
+
 // The kernels that wait with a bound record an expired wait in a device word of their own translation
 // unit; each of these reads that word, clears it, and reports whether it was set.
 int take_device_error_mma(unsigned* flag);

@@ -106,7 +106,7 @@ int run_bwd(const BwdArgs& g, int64_t T, int32_t d, int dtype, cudaStream_t s) {
     // few hundred rows on
     if (umma_bwd_supported(logd, dtype) &&
         (g_variant == 4 || (g_variant == 0 && T * static_cast<int64_t>(d) >= (1ll << 18)))) {
-        return umma_bwd(logd, dtype, g_bwd_operand_mode == 0, g, c);
+        return umma_bwd(logd, dtype, g_bwd_operand_mode == 1, g, c);
     }
     if (g_variant != 1 && mma_supported(logd, dtype)) {
         const bool streamed = g_variant >= 3 || (g_variant == 0 && enough_rows_to_stream(T, c.sms));
@@ -468,6 +468,12 @@ int wht_affine_device_status(void) {
         any |= flag;
     }
     return any ? WHT_ERR_DEVICE_WAIT : WHT_OK;
+}
+
+int wht_affine_selftest_wait_expiry(uint32_t limit_us, unsigned int* out3, void* stream) {
+    if (!out3) return WHT_ERR_NULL;
+    if (limit_us == 0 || limit_us > 1000000u) return WHT_ERR_BAD_T;
+    return launch_wait_expiry_selftest(limit_us, out3, static_cast<cudaStream_t>(stream));
 }
 
 int wht_affine_last_cuda_error(void) { return g_last_cuda_error; }
