@@ -399,7 +399,7 @@ def section_tensor_parallel_local(B, hbm_peak):
     transfer, not the kernel, sets the time).  Bytes: (g+1) blocks forward, (2g+1) backward."""
     from paper_2603_08343_b200 import tp
     out = {}
-    for g, w_, T in ((2, 1024, 65536), (8, 1024, 16384), (8, 256, 65536)):
+    for g, w_, T in ((2, 1024, 65536), (4, 1024, 32768), (8, 1024, 16384), (8, 256, 65536)):
         wk = wl.Workload("tp", T, w_, wl.WHT_BF16_PF32, "normal", 20 + g, True, "")
         base = wl.gen_full(wk.with_rows(4096), "x").cuda()
         xs = [base.roll(s, 0).repeat(T // 4096, 1) for s in range(g)]

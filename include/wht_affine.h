@@ -206,11 +206,13 @@ size_t wht_affine_bwd_grouped_workspace_bytes(int64_t T, int32_t d, int32_t bloc
  * any rank launches (a barrier across ranks on the host or stream), and that no rank overwrites its
  * inputs before every rank's call has completed.  Gradients of a and b need no reduction across the
  * g ranks (each rank owns its channels); across data-parallel replicas they add as usual.
- * Every storage type.  Forward of bf16 rows with 1024 <= w <= 4096 and T*w >= 4 Mi elements: tcgen05
- * kernel (each source block's tile is bulk-copied into shared memory and multiplied by H_128 into one
- * accumulator, negated where the sign is -1); otherwise, and for the backward, butterfly kernels with
- * multi-source loads.  The backward takes caller-owned scratch of at least
- * wht_affine_bwd_tp_workspace_bytes(T, w, g, dtype) bytes and never allocates.
+ * Every storage type.  bf16 rows with 1024 <= w <= 4096: tcgen05 kernels (forward from T*w >= 4 Mi
+ * elements, backward from 256 Ki and g >= 2): each source block's tile is bulk-copied into shared memory
+ * and multiplied by H_128 into one accumulator, negated where the sign is -1; the backward also adds up
+ * +-(a_s/sqrt d) (.) dy_s in registers as the blocks arrive, the rank's own block last.  Otherwise butterfly
+ * kernels with multi-source loads.  The backward takes caller-owned scratch of at least
+ * wht_affine_bwd_tp_workspace_bytes(T, w, g, dtype) bytes and never allocates; it honours
+ * wht_affine_set_bwd_operand_mode.
  * Errors as for the plain calls; g or r out of range -> WHT_ERR_BAD_DIM.
  */
 int wht_affine_fwd_tp(const void* const* x_parts, const void* a, const void* b, void* y,

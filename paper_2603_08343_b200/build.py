@@ -17,7 +17,7 @@ CSRC = os.path.join(HERE, "csrc")
 OBJ_DIR = os.path.join(HERE, "_build")
 LIB_PATH = os.path.join(HERE, "libwht_affine.so")
 SOURCES = ["wht_affine.cu", "family_misc.cu", "family_bfly_fwd.cu", "family_bfly_bwd.cu", "family_tp.cu",
-           "family_mma.cu", "family_umma_fwd.cu", "family_umma_bwd.cu"]
+           "family_mma.cu", "family_umma_fwd.cu", "family_umma_bwd.cu", "family_umma_tp.cu"]
 ARCH = ["-gencode", "arch=compute_100a,code=sm_100a"]
 
 

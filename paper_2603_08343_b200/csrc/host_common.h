@@ -188,11 +188,15 @@ int umma_bwd(int logd, int dtype, bool g_hi_lo, const BwdArgs& g, const Ctx& c);
 // Self-test of the bounded waits (family_umma_fwd.cu): a one-CTA kernel whose wait runs out after limit_us.
 int launch_wait_expiry_selftest(uint32_t limit_us, unsigned int* out, cudaStream_t s);
 
+// g >= 2 ranks, bf16 rows, 1024 <= w <= 4096                                          // family_umma_tp.cu
+int umma_bwd_tp(int logw, int dtype, bool g_hi_lo, const TpCall& t, const BwdArgs& g, const Ctx& c);
+
 // The kernels that wait with a bound record an expired wait in a device word of their own translation
 // unit; each of these reads that word, clears it, and reports whether it was set.
 int take_device_error_mma(unsigned* flag);
 int take_device_error_umma_fwd(unsigned* flag);
 int take_device_error_umma_bwd(unsigned* flag);
+int take_device_error_umma_tp(unsigned* flag);
 
 // Defines one of the three readers above in the translation unit that includes the waiting kernels.
 #define WHT_DEFINE_DEVICE_ERROR_READER(name)                                                         \

@@ -184,6 +184,12 @@ int run_bwd_tp(const TpCall& t, const BwdArgs& g, int64_t T, int32_t w, int dtyp
     int rc = current_device(&c.dev, &c.sms);
     if (rc != WHT_OK) return rc;
     const int logw = log2_of(w);
+    // bf16 rows of 1024 ... 4096 channels per rank on two or more ranks: tcgen05 form (as in the plain
+    // backward it pays from a few hundred rows on)
+    if (dtype != WHT_F32 && logw >= 10 && logw <= 12 && t.g >= 2 &&
+        (g_variant == 4 || (g_variant == 0 && T * static_cast<int64_t>(w) >= (1ll << 18)))) {
+        return umma_bwd_tp(logw, dtype, g_bwd_operand_mode == 1, t, g, c);
+    }
     return bfly_bwd_tp(logw, dtype, t, g, c);
 }
 
@@ -461,7 +467,8 @@ int wht_copy_rows(const void* src, void* dst, int64_t T, int32_t d, int dtype, v
 int wht_affine_device_status(void) {
     // one status word per translation unit that holds waiting kernels: read and clear them all
     unsigned any = 0;
-    for (auto take : {take_device_error_mma, take_device_error_umma_fwd, take_device_error_umma_bwd}) {
+    for (auto take : {take_device_error_mma, take_device_error_umma_fwd, take_device_error_umma_bwd,
+                      take_device_error_umma_tp}) {
         unsigned flag = 0;
         const int rc = take(&flag);
         if (rc != WHT_OK) return rc;

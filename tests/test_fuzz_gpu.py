@@ -99,10 +99,11 @@ def _tp_cases(seed, count):
     return out
 
 
-@pytest.mark.parametrize("seed", [21])
+@pytest.mark.parametrize("seed", [21, 22])
 def test_random_column_sharded_shapes_match_the_oracle(B, seed):
     from paper_2603_08343_b200 import tp
     for case, g, w, T, dtype, variant in _tp_cases(seed, 20):
+        B.wht_affine_set_bwd_operand_mode(case & 1)  # both operand modes of the tcgen05 backward
         d = g * w
         wk = wl.Workload("fuzz-tp", T, d, dtype, "normal", 7000 + 100 * seed + case, True, "")
         x, dy = wl.gen_full(wk, "x"), wl.gen_full(wk, "dy")
@@ -128,3 +129,4 @@ def test_random_column_sharded_shapes_match_the_oracle(B, seed):
         assert _ratio_rows(to_f64(dx), ref_dx, dtype, np.linalg.norm(a64[None, :] * dy64, axis=1)) <= 1.0, what + ": dx"
         assert np.max(np.abs(to_f64(da) - ref_da)) <= 1e-4 * np.max(np.abs(ref_da)), what + ": da"
         assert np.max(np.abs(to_f64(db) - ref_db)) <= 1e-4 * np.max(np.abs(ref_db)), what + ": db"
+    B.wht_affine_set_bwd_operand_mode(0)

@@ -77,6 +77,46 @@ def test_column_sharded_calls_match_the_full_width_oracle(B, g, w, dtype, T, var
     B.wht_affine_set_variant(0)
 
 
+@pytest.mark.parametrize("mode", [0, 1])
+@pytest.mark.parametrize("g,w,T,dtype", [(2, 1024, 148 * 16 * 2 + 5, wl.WHT_BF16_PF32), (4, 1024, 148 * 16 + 3, wl.WHT_BF16),
+                                         (8, 1024, 148 * 16 + 1, wl.WHT_BF16_PF32), (2, 2048, 148 * 8 * 2 + 7, wl.WHT_BF16),
+                                         (4, 2048, 148 * 8 + 4, wl.WHT_BF16_PF32), (2, 4096, 148 * 4 + 3, wl.WHT_BF16_PF32)])
+def test_column_sharded_backward_on_the_tensor_core_many_rows(B, g, w, T, dtype, mode):
+    """The tcgen05 backward of the column-sharded form over several tiles per CTA (the ring and both
+    accumulators wrap, the last tile is ragged), in both operand modes, every rank in turn, against the
+    full-width chain rule of Eq. 1.  Repeating a call must give the same bits (fixed summation order)."""
+    B.wht_affine_set_variant(0)
+    B.wht_affine_set_bwd_operand_mode(mode)
+    try:
+        d = g * w
+        wk = wl.Workload("tp-bwd", T, d, dtype, "normal", 1200 + d + g, True, "")
+        x, dy = wl.gen_full(wk, "x"), wl.gen_full(wk, "dy")
+        a, _ = wl.gen_params(wk)
+        xs = [p.cuda() for p in tp.split_columns(x, g)]
+        dys = [p.cuda() for p in tp.split_columns(dy, g)]
+        as_ = [a[s * w:(s + 1) * w].contiguous().cuda() for s in range(g)]
+        outs = [tp.TpWht(g, r).backward(dys, xs, as_, T, w) for r in range(g)]
+        again = tp.TpWht(g, g - 1).backward(dys, xs, as_, T, w)
+        torch.cuda.synchronize()
+        assert all(torch.equal(u, v) for u, v in zip(outs[g - 1], again))
+        dx = torch.cat([o[0] for o in outs], dim=1).cpu()
+        da, db = torch.cat([o[1] for o in outs]).cpu(), torch.cat([o[2] for o in outs]).cpu()
+        ref_dx, ref_da, ref_db = oracle.wht_affine_bwd(to_f64(dy), to_f64(x), to_f64(a))
+        assert_rows_bf16(to_f64(dx), ref_dx, f"tp dx g={g} w={w} mode={mode}")
+        assert_grad_vec(to_f64(da), ref_da, f"tp da g={g} w={w}")
+        assert_grad_vec(to_f64(db), ref_db, f"tp db g={g} w={w}")
+        # the same bits as the butterfly kernels' reductions is not required; the same values within the bound is:
+        B.wht_affine_set_variant(1)
+        dx_b, da_b, db_b = tp.TpWht(g, 0).backward(dys, xs, as_, T, w)
+        torch.cuda.synchronize()
+        assert_rows_bf16(to_f64(outs[0][0].cpu()), to_f64(dx_b.cpu()), "tcgen05 vs butterfly dx")
+        assert_grad_vec(to_f64(outs[0][1].cpu()), to_f64(da_b.cpu()), "tcgen05 vs butterfly da")
+    finally:
+        B.wht_affine_set_variant(0)
+        B.wht_affine_set_bwd_operand_mode(0)
+    B.wht_affine_device_status()
+
+
 def test_blocks_given_as_addresses_and_repeat_calls_are_bit_identical(B):
     g, w, T, dtype = 4, 512, 257, wl.WHT_BF16_PF32
     wk = wl.Workload("tp", T, g * w, dtype, "normal", 77, True, "")
