@@ -62,7 +62,8 @@ typedef enum {
     WHT_ERR_WORKSPACE = -6,   /* workspace missing, too small, or allocation failed  */
     WHT_ERR_CUDA = -7,        /* a CUDA runtime call failed; see wht_affine_last_cuda_error */
     WHT_ERR_BAD_VARIANT = -8, /* unknown kernel variant id                           */
-    WHT_ERR_DEVICE_WAIT = -9  /* a kernel's bounded wait (copy, product, hand-over) expired */
+    WHT_ERR_DEVICE_WAIT = -9, /* a kernel's bounded wait (copy, product, hand-over) expired */
+    WHT_ERR_GUARD = -10       /* debug build only: a kernel wrote outside an output or scratch buffer */
 } wht_status;
 
 /*
@@ -306,6 +307,26 @@ int wht_affine_device_status(void);
  * from then on, and the library works as before.
  */
 int wht_affine_selftest_wait_expiry(uint32_t limit_us, unsigned int* out3, void* stream);
+
+/*
+ * Debug build (the paper has no counterpart).  The library can be compiled with -DWHT_DEBUG
+ * (python -m paper_2603_08343_b200.build --debug -> libwht_affine_debug.so): the same kernels, but every
+ * compute call then writes its outputs (y; dx, da, db) and its scratch into buffers of the library's own
+ * that carry a 4 KiB guard region filled with a canary byte on either side.  After the kernels have run,
+ * the call synchronises the stream, checks the guards and only then copies the results into the
+ * caller's tensors; a guard that changed makes the call return WHT_ERR_GUARD.  This is the stand-in
+ * for a memory checker where none can be run: an out-of-bounds WRITE next to an output is caught (reads
+ * are not).  Such a build allocates, synchronises and copies on every call -- wht_affine_bwd_noalloc
+ * included -- and is meant for test suites only.
+ *   wht_affine_debug_build()            1 in a debug build, 0 in the regular one.
+ *   wht_affine_debug_selftest_guard(k)  debug build: sets up a guarded buffer, writes its payload and,
+ *                                       for k = 1 / 2, one byte just before / after it (inside the
+ *                                       library's own allocation), and returns the verdict of the check:
+ *                                       WHT_OK for k = 0, WHT_ERR_GUARD for k = 1, 2.  Regular build:
+ *                                       WHT_ERR_BAD_VARIANT.
+ */
+int wht_affine_debug_build(void);
+int wht_affine_debug_selftest_guard(int damage);
 
 /* cudaError_t of the most recent failing CUDA call on this thread (0 if none). */
 int wht_affine_last_cuda_error(void);

@@ -23,7 +23,8 @@ EXPORTS = (
     "wht_affine_fwd_tp", "wht_affine_bwd_tp", "wht_affine_bwd_tp_workspace_bytes",
     "wht_affine_bwd_workspace_bytes", "wht_affine_set_variant", "wht_affine_get_variant",
     "wht_affine_set_bwd_operand_mode", "wht_affine_get_bwd_operand_mode",
-    "wht_copy_rows", "wht_affine_device_status", "wht_affine_selftest_wait_expiry", "wht_affine_last_cuda_error", "wht_affine_status_string",
+    "wht_copy_rows", "wht_affine_device_status", "wht_affine_selftest_wait_expiry",
+    "wht_affine_debug_build", "wht_affine_debug_selftest_guard", "wht_affine_last_cuda_error", "wht_affine_status_string",
     "wht_affine_shutdown",
 )
 
@@ -36,12 +37,15 @@ class WhtError(RuntimeError):
         super().__init__(f"{where}: {msg} (status {status}, cuda error {cuda})")
 
 
-def _load() -> ctypes.CDLL:
-    if not os.path.exists(LIB_PATH):
+def _load(path: str | None = None) -> ctypes.CDLL:
+    """Loads the library (the regular build, or another build of it given by path) and declares the
+    argument types of every export."""
+    path = LIB_PATH if path is None else path
+    if not os.path.exists(path):
         raise ImportError(
-            f"{LIB_PATH} is missing: build it with `python -m paper_2603_08343_b200.build` "
+            f"{path} is missing: build it with `python -m paper_2603_08343_b200.build` "
             "(there is no CPU fallback)")
-    lib = ctypes.CDLL(LIB_PATH)
+    lib = ctypes.CDLL(path)
     vp, i64, i32, ci, sz = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32, ctypes.c_int, ctypes.c_size_t
     lib.wht_affine_fwd.argtypes = [vp, vp, vp, vp, i64, i32, ci, vp]
     lib.wht_affine_fwd_residual.argtypes = [vp, vp, vp, vp, vp, i64, i32, ci, vp]
@@ -71,6 +75,8 @@ def _load() -> ctypes.CDLL:
     lib.wht_affine_status_string.argtypes = [ci]
     lib.wht_affine_status_string.restype = ctypes.c_char_p
     lib.wht_affine_shutdown.argtypes = []
+    lib.wht_affine_debug_build.argtypes = []
+    lib.wht_affine_debug_selftest_guard.argtypes = [ci]
     for name in EXPORTS:
         fn = getattr(lib, name)
         if fn.restype is ctypes.c_int or fn.restype is None:
@@ -84,6 +90,11 @@ _lib = _load()
 def lib() -> ctypes.CDLL:
     """The loaded shared library (for tests that call the C ABI with raw pointers)."""
     return _lib
+
+
+def load_library(path: str) -> ctypes.CDLL:
+    """Another build of the library (the -DWHT_DEBUG one) with the same argument types declared."""
+    return _load(path)
 
 
 def _ptr(t):

@@ -63,46 +63,52 @@ def _run(cmd):
     return proc.stderr
 
 
-def build(force: bool = False, verbose: bool = False, defines: tuple = ()) -> str:
+# only the C ABI file looks at WHT_DEBUG: the debug library links the regular family objects
+DEBUG_SOURCES = ("wht_affine.cu",)
+LIB_DEBUG_PATH = os.path.join(HERE, "libwht_affine_debug.so")
+
+
+def build(force: bool = False, verbose: bool = False, debug: bool = False) -> str:
     """Compile what is missing or older than its sources; return the library's path.
 
-    `verbose` adds -Xptxas -v (registers, spills and shared memory of every kernel, on stderr);
-    `defines` are extra -D flags (a debug build); both rebuild everything.
+    `verbose` adds -Xptxas -v (registers, spills and shared memory of every kernel, on stderr) and
+    rebuilds everything.  `debug` builds libwht_affine_debug.so instead: the same kernels with the C ABI
+    compiled with -DWHT_DEBUG (guard regions around every output and scratch buffer, see the header).
     """
-    force = force or verbose or bool(defines)
+    force = force or verbose
+    lib = LIB_DEBUG_PATH if debug else LIB_PATH
     sources = [os.path.join(CSRC, s) for s in SOURCES]
-    if not force and os.path.exists(LIB_PATH) and \
-            os.path.getmtime(LIB_PATH) >= max(_newest_dependency_mtime(p) for p in sources):
-        return LIB_PATH  # up to date, whether or not the objects are still around
+    if not force and os.path.exists(lib) and \
+            os.path.getmtime(lib) >= max(_newest_dependency_mtime(p) for p in sources):
+        return lib  # up to date, whether or not the objects are still around
     os.makedirs(OBJ_DIR, exist_ok=True)
     nvcc = _nvcc()
-    jobs = []
+    jobs, objs = [], []
     for src in SOURCES:
         path = os.path.join(CSRC, src)
-        obj = os.path.join(OBJ_DIR, src[:-3] + ".o")
+        special = debug and src in DEBUG_SOURCES
+        obj = os.path.join(OBJ_DIR, src[:-3] + ("_debug.o" if special else ".o"))
+        objs.append(obj)
         stale = force or not os.path.exists(obj) or os.path.getmtime(obj) < _newest_dependency_mtime(path)
         if stale:
             cmd = [nvcc, "-std=c++17", "-O3", "-lineinfo", *ARCH, "-Xcompiler", "-fPIC", "-c", path, "-o", obj]
-            cmd += [f"-D{d}" for d in defines]
+            if special:
+                cmd.append("-DWHT_DEBUG")
             if verbose:
                 cmd.insert(1, "-Xptxas=-v")
             jobs.append(cmd)
-    objs = [os.path.join(OBJ_DIR, s[:-3] + ".o") for s in SOURCES]
-    if not jobs and os.path.exists(LIB_PATH) and os.path.getmtime(LIB_PATH) >= max(os.path.getmtime(o) for o in objs):
-        return LIB_PATH
+    if not jobs and os.path.exists(lib) and os.path.getmtime(lib) >= max(os.path.getmtime(o) for o in objs):
+        return lib
     with ThreadPoolExecutor(max_workers=min(len(jobs), os.cpu_count() or 4) or 1) as pool:
         logs = list(pool.map(_run, jobs))
     if verbose:
         sys.stderr.write("".join(logs))
-    _run([nvcc, *ARCH, "-Xcompiler", "-fPIC", "-shared", "-o", LIB_PATH, *objs])
-    if defines:  # a special build must not pass for the regular one on the next call
-        for o in objs:
-            os.utime(o, (0, 0))
-    return LIB_PATH
+    _run([nvcc, *ARCH, "-Xcompiler", "-fPIC", "-shared", "-o", lib, *objs])
+    return lib
 
 
 if __name__ == "__main__":
     if "--digest" in sys.argv:  # python -m paper_2603_08343_b200.build --digest a.cuh,b.cu
         print(source_digest(sys.argv[sys.argv.index("--digest") + 1].split(",")))
     else:
-        print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+        print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, debug="--debug" in sys.argv))

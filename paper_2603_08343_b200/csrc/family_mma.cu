@@ -8,6 +8,12 @@ using namespace wht;
 
 namespace {
 
+// CTAs along x: enough to fill the device, shared out over the channel groups of the block-diagonal form
+int grid_x(const Ctx& c, int rows_per_cta, int per_sm) {
+    const int grid = capped_grid(ceil_div(c.T, rows_per_cta), c.sms, per_sm);
+    return c.groups > 1 ? (grid / c.groups > 0 ? grid / c.groups : 1) : grid;
+}
+
 template <int LOGD, int TB, int RG, typename TP>
 int launch_mma_fwd(const FwdArgs& f, const Ctx& c) {
     using Geo = MmaGeo<LOGD, TB, RG>;
@@ -15,11 +21,11 @@ int launch_mma_fwd(const FwdArgs& f, const Ctx& c) {
     auto kernel = mma_fwd_kernel<LOGD, TB, RG, TP>;
     const int per_sm = resident_ctas(kernel, Geo::THREADS, Geo::SMEM_FWD, c.dev, occ);
     if (per_sm <= 0) return occupancy_fail();
-    const int grid = capped_grid(ceil_div(c.T, RG), c.sms, per_sm);
-    launch_overlapped(kernel, grid, Geo::THREADS, Geo::SMEM_FWD, c.stream,
+    const int grid = grid_x(c, RG, per_sm);
+    launch_overlapped(kernel, dim3(grid, c.groups), Geo::THREADS, Geo::SMEM_FWD, c.stream,
                       static_cast<const __nv_bfloat16*>(f.x), static_cast<const TP*>(f.a), static_cast<const TP*>(f.b),
                       static_cast<const __nv_bfloat16*>(f.resid), static_cast<__nv_bfloat16*>(f.y),
-                      static_cast<long long>(c.T), inv_sqrt(Geo::D));
+                      static_cast<long long>(c.T), static_cast<long long>(c.ld ? c.ld : Geo::D), inv_sqrt(Geo::D));
     WHT_CUDA_TRY(cudaGetLastError());
     return WHT_OK;
 }
@@ -31,12 +37,12 @@ int launch_mma_bwd(const BwdArgs& g, const Ctx& c) {
     auto kernel = mma_bwd_kernel<LOGD, TB, RG, TP>;
     const int per_sm = resident_ctas(kernel, Geo::THREADS, Geo::SMEM_BWD, c.dev, occ);
     if (per_sm <= 0) return occupancy_fail();
-    const int grid = capped_grid(ceil_div(c.T, RG), c.sms, per_sm);
+    const int grid = grid_x(c, RG, per_sm);
     return run_bwd_with_grid(g, c, grid, Geo::D, [&](int n) {
-        kernel<<<n, Geo::THREADS, Geo::SMEM_BWD, c.stream>>>(
+        kernel<<<dim3(n, c.groups), Geo::THREADS, Geo::SMEM_BWD, c.stream>>>(
             static_cast<const __nv_bfloat16*>(g.dy), static_cast<const __nv_bfloat16*>(g.x),
             static_cast<const TP*>(g.a), static_cast<__nv_bfloat16*>(g.dx), static_cast<float*>(g.ws),
-            static_cast<long long>(c.T), inv_sqrt(Geo::D));
+            static_cast<long long>(c.T), static_cast<long long>(c.ld ? c.ld : Geo::D), inv_sqrt(Geo::D));
     });
 }
 
@@ -47,11 +53,11 @@ int launch_mma_fwd_pipe(const FwdArgs& f, const Ctx& c) {
     auto kernel = mma_fwd_pipe_kernel<LOGD, TB, RG, S, MINB, TP>;
     const int per_sm = resident_ctas(kernel, Geo::THREADS, Geo::SMEM, c.dev, occ);
     if (per_sm <= 0) return occupancy_fail();
-    const int grid = capped_grid(ceil_div(c.T, RG), c.sms, per_sm);
-    kernel<<<grid, Geo::THREADS, Geo::SMEM, c.stream>>>(
+    const int grid = grid_x(c, RG, per_sm);
+    kernel<<<dim3(grid, c.groups), Geo::THREADS, Geo::SMEM, c.stream>>>(
         static_cast<const __nv_bfloat16*>(f.x), static_cast<const TP*>(f.a), static_cast<const TP*>(f.b),
         static_cast<const __nv_bfloat16*>(f.resid), static_cast<__nv_bfloat16*>(f.y), static_cast<long long>(c.T),
-        inv_sqrt(Geo::D));
+        static_cast<long long>(c.ld ? c.ld : Geo::D), inv_sqrt(Geo::D));
     WHT_CUDA_TRY(cudaGetLastError());
     return WHT_OK;
 }
@@ -63,12 +69,12 @@ int launch_mma_bwd_pipe(const BwdArgs& g, const Ctx& c) {
     auto kernel = mma_bwd_pipe_kernel<LOGD, TB, RG, S, MINB, TP>;
     const int per_sm = resident_ctas(kernel, Geo::THREADS, Geo::SMEM, c.dev, occ);
     if (per_sm <= 0) return occupancy_fail();
-    const int grid = capped_grid(ceil_div(c.T, RG), c.sms, per_sm);
+    const int grid = grid_x(c, RG, per_sm);
     return run_bwd_with_grid(g, c, grid, Geo::D, [&](int n) {
-        kernel<<<n, Geo::THREADS, Geo::SMEM, c.stream>>>(
+        kernel<<<dim3(n, c.groups), Geo::THREADS, Geo::SMEM, c.stream>>>(
             static_cast<const __nv_bfloat16*>(g.dy), static_cast<const __nv_bfloat16*>(g.x),
             static_cast<const TP*>(g.a), static_cast<__nv_bfloat16*>(g.dx), static_cast<float*>(g.ws),
-            static_cast<long long>(c.T), inv_sqrt(Geo::D));
+            static_cast<long long>(c.T), static_cast<long long>(c.ld ? c.ld : Geo::D), inv_sqrt(Geo::D));
     });
 }
 
@@ -79,6 +85,7 @@ template <typename TP>
 int dispatch_mma_fwd(int logd, bool few_rows, bool streamed, const FwdArgs& f, const Ctx& c) {
     if (few_rows) {
         switch (logd) {
+            case 8: return launch_mma_fwd<8, 0, 8, TP>(f, c);
             case 9: return launch_mma_fwd<9, 1, 4, TP>(f, c);
             case 10: return launch_mma_fwd<10, 1, 2, TP>(f, c);
             case 11: return launch_mma_fwd<11, 2, 2, TP>(f, c);
@@ -88,6 +95,7 @@ int dispatch_mma_fwd(int logd, bool few_rows, bool streamed, const FwdArgs& f, c
         }
     } else if (!streamed) {
         switch (logd) {
+            case 8: return launch_mma_fwd<8, 0, 8, TP>(f, c);
             case 9: return launch_mma_fwd<9, 1, 4, TP>(f, c);
             case 10: return launch_mma_fwd<10, 2, 4, TP>(f, c);
             case 11: return launch_mma_fwd<11, 3, 4, TP>(f, c);
@@ -96,6 +104,7 @@ int dispatch_mma_fwd(int logd, bool few_rows, bool streamed, const FwdArgs& f, c
         }
     } else {
         switch (logd) {
+            case 8: return launch_mma_fwd_pipe<8, 0, 8, 4, 4, TP>(f, c);
             case 9: return launch_mma_fwd_pipe<9, 1, 8, 4, 2, TP>(f, c);
             case 10: return launch_mma_fwd_pipe<10, 2, 8, 4, 3, TP>(f, c);
             case 11: return launch_mma_fwd_pipe<11, 3, 8, 3, 2, TP>(f, c);
@@ -110,6 +119,7 @@ template <typename TP>
 int dispatch_mma_bwd(int logd, bool streamed, const BwdArgs& g, const Ctx& c) {
     if (!streamed) {
         switch (logd) {
+            case 8: return launch_mma_bwd<8, 0, 8, TP>(g, c);
             case 9: return launch_mma_bwd<9, 1, 8, TP>(g, c);
             case 10: return launch_mma_bwd<10, 2, 8, TP>(g, c);
             case 11: return launch_mma_bwd<11, 2, 4, TP>(g, c);
@@ -118,6 +128,7 @@ int dispatch_mma_bwd(int logd, bool streamed, const BwdArgs& g, const Ctx& c) {
         }
     } else {
         switch (logd) {
+            case 8: return launch_mma_bwd_pipe<8, 0, 8, 4, 3, TP>(g, c);
             case 9: return launch_mma_bwd_pipe<9, 1, 8, 4, 2, TP>(g, c);
             case 10: return launch_mma_bwd_pipe<10, 2, 8, 3, 2, TP>(g, c);
             case 11: return launch_mma_bwd_pipe<11, 2, 4, 2, 2, TP>(g, c);

@@ -91,7 +91,7 @@ struct MmaGeo {
     static constexpr int D = 1 << LOGD;
     static constexpr int NT = 1 << TB;         // chunks of 8 elements per thread
     static constexpr int WB = LOGD - 8 - TB;   // stages that cross warps
-    static_assert(TB >= 1 && WB >= 0 && WB <= TB, "unsupported split of the row");
+    static_assert(TB >= 0 && WB >= 0 && WB <= TB, "unsupported split of the row");
     static constexpr int W = 1 << WB;          // warps per row
     static constexpr int NREST = NT / W;
     static constexpr int RG = RG_;             // rows in flight per CTA
@@ -152,8 +152,10 @@ struct MmaXform {
         }
     }
 
-    // fp32 butterflies on bit 2 (h) and on chunk-slot bits 1..TB-1
+    // fp32 butterflies on bit 2 (h) and on chunk-slot bits 1..TB-1.  A row of one chunk per thread
+    // (d = 256) has no bit 8 for pass 2, which takes bit 2 instead: nothing to do here.
     static __device__ __forceinline__ void mid_stages(F2 (&m)[NT][2][2]) {
+        if constexpr (NT == 1) return;
 #pragma unroll
         for (int t = 0; t < NT; ++t) {
             bfly2(m[t][0][0], m[t][1][0]);
@@ -174,9 +176,25 @@ struct MmaXform {
         }
     }
 
-    // pass 2 on bits {5,6,7} and chunk-slot bit 0; the result is in load layout
+    // pass 2 on bits {5,6,7} and chunk-slot bit 0; the result is in load layout.  With one chunk per
+    // thread (d = 256) the fourth bit is bit 2 instead: the register select of the B fragment is h, and the
+    // two halves of the accumulator fragment are h = 0 and h = 1 of the output.
     static __device__ __forceinline__ void pass2(const F2 (&m)[NT][2][2], F2 (&v)[NT][4],
                                                  const uint32_t (&hf)[4]) {
+        if constexpr (NT == 1) {
+#pragma unroll
+            for (int p = 0; p < 2; ++p) {
+                uint32_t b0h, b0l, b1h, b1l;
+                split_hi_lo(m[0][0][p], b0h, b0l);
+                split_hi_lo(m[0][1][p], b1h, b1l);
+                F2 d01 = f2(0.0f, 0.0f), d23 = f2(0.0f, 0.0f);
+                mma_bf16_m16n8k16(d01, d23, hf, b0h, b1h);
+                mma_bf16_m16n8k16(d01, d23, hf, b0l, b1l);
+                v[0][p] = d01;
+                v[0][2 + p] = d23;
+            }
+            return;
+        }
 #pragma unroll
         for (int u = 0; u < NT / 2; ++u) {
 #pragma unroll
@@ -311,7 +329,8 @@ template <class Geo>
 __device__ __forceinline__ void bwd_publish_partials(const F2 (&da_acc)[Geo::NT][4], const F2 (&db_acc)[Geo::NT][4],
                                                      float* fold, float* __restrict__ partials, int rg, int w,
                                                      int lane) {
-    float* out = partials + static_cast<size_t>(blockIdx.x) * 2 * Geo::D;
+    // block-diagonal form: the partials of channel group blockIdx.y follow those of the group before
+    float* out = partials + (static_cast<size_t>(blockIdx.y) * gridDim.x + blockIdx.x) * 2 * Geo::D;
 #pragma unroll
     for (int which = 0; which < 2; ++which) {
         __syncthreads();
@@ -337,7 +356,9 @@ __device__ __forceinline__ void bwd_publish_partials(const F2 (&da_acc)[Geo::NT]
 template <int LOGD, int TB, int RG, typename TP>
 __global__ void __launch_bounds__(MmaGeo<LOGD, TB, RG>::THREADS)
 mma_fwd_kernel(const __nv_bfloat16* x, const TP* __restrict__ a, const TP* __restrict__ b,
-               const __nv_bfloat16* resid, __nv_bfloat16* y, long long T, float inv_sqrt_d) {
+               const __nv_bfloat16* resid, __nv_bfloat16* y, long long T, long long ld, float inv_sqrt_d) {
+    // ld: elements between consecutive rows (>= D).  Block-diagonal form: blockIdx.y picks the channel
+    // group [y*D, (y+1)*D) of rows ld wide.
     using Geo = MmaGeo<LOGD, TB, RG>;
     using X = MmaXform<Geo>;
     constexpr int NT = Geo::NT;
@@ -350,6 +371,11 @@ mma_fwd_kernel(const __nv_bfloat16* x, const TP* __restrict__ a, const TP* __res
     uint32_t hf[4];
     make_h16_fragment(hf, lane);
     const F2 rs2 = f2(inv_sqrt_d, inv_sqrt_d);
+    {
+        const long long goff = static_cast<long long>(blockIdx.y) * Geo::D;
+        x += goff; y += goff; a += goff; b += goff;
+        if (resid != nullptr) resid += goff;
+    }
     grid_dependency_wait();
     grid_launch_dependents();
 
@@ -371,7 +397,7 @@ mma_fwd_kernel(const __nv_bfloat16* x, const TP* __restrict__ a, const TP* __res
     int parity = 0;
     const long long stride = static_cast<long long>(gridDim.x) * RG;
     for (long long row = static_cast<long long>(blockIdx.x) * RG + rg; row < T; row += stride) {
-        const uint4* src = reinterpret_cast<const uint4*>(x + row * Geo::D);
+        const uint4* src = reinterpret_cast<const uint4*>(x + row * ld);
         uint4 raw[NT];
 #pragma unroll
         for (int t = 0; t < NT; ++t) raw[t] = __ldcs(src + chunk_of<Geo, false>(w, t) * 32 + lane);
@@ -379,7 +405,7 @@ mma_fwd_kernel(const __nv_bfloat16* x, const TP* __restrict__ a, const TP* __res
         if (resid != nullptr) {  // the residual chunks too, ahead of the transform
 #pragma unroll
             for (int idx = 0; idx < NT; ++idx)
-                res[idx] = __ldcs(reinterpret_cast<const uint4*>(resid + row * Geo::D) +
+                res[idx] = __ldcs(reinterpret_cast<const uint4*>(resid + row * ld) +
                                   chunk_of<Geo, true>(w, idx) * 32 + lane);
         }
         F2 m[NT][2][2];
@@ -389,7 +415,7 @@ mma_fwd_kernel(const __nv_bfloat16* x, const TP* __restrict__ a, const TP* __res
         X::pass2(m, v, hf);
         X::exchange_and_top(v, xbuf + parity * Geo::XCHG_ONE, w, lane, 1 + rg);
         parity ^= 1;
-        uint4* dst = reinterpret_cast<uint4*>(y + row * Geo::D);
+        uint4* dst = reinterpret_cast<uint4*>(y + row * ld);
 #pragma unroll
         for (int idx = 0; idx < NT; ++idx) {
             const int c = chunk_of<Geo, true>(w, idx);
@@ -416,7 +442,7 @@ mma_fwd_kernel(const __nv_bfloat16* x, const TP* __restrict__ a, const TP* __res
 template <int LOGD, int TB, int RG, typename TP>
 __global__ void __launch_bounds__(MmaGeo<LOGD, TB, RG>::THREADS)
 mma_bwd_kernel(const __nv_bfloat16* dy, const __nv_bfloat16* x, const TP* __restrict__ a,
-               __nv_bfloat16* dx, float* __restrict__ partials, long long T, float inv_sqrt_d) {
+               __nv_bfloat16* dx, float* __restrict__ partials, long long T, long long ld, float inv_sqrt_d) {
     using Geo = MmaGeo<LOGD, TB, RG>;
     using X = MmaXform<Geo>;
     constexpr int NT = Geo::NT;
@@ -429,6 +455,10 @@ mma_bwd_kernel(const __nv_bfloat16* dy, const __nv_bfloat16* x, const TP* __rest
     uint32_t hf[4];
     make_h16_fragment(hf, lane);
     const F2 rs2 = f2(inv_sqrt_d, inv_sqrt_d);
+    {
+        const long long goff = static_cast<long long>(blockIdx.y) * Geo::D;
+        dy += goff; x += goff; dx += goff; a += goff;
+    }
 
     F2 da_acc[NT][4], db_acc[NT][4];
 #pragma unroll
@@ -439,8 +469,8 @@ mma_bwd_kernel(const __nv_bfloat16* dy, const __nv_bfloat16* x, const TP* __rest
 
     const long long stride = static_cast<long long>(gridDim.x) * RG;
     for (long long row = static_cast<long long>(blockIdx.x) * RG + rg; row < T; row += stride) {
-        const uint4* xsrc = reinterpret_cast<const uint4*>(x + row * Geo::D);
-        const uint4* dysrc = reinterpret_cast<const uint4*>(dy + row * Geo::D);
+        const uint4* xsrc = reinterpret_cast<const uint4*>(x + row * ld);
+        const uint4* dysrc = reinterpret_cast<const uint4*>(dy + row * ld);
         uint4 raw[NT], rawdy[NT];
 #pragma unroll
         for (int t = 0; t < NT; ++t) raw[t] = __ldcs(xsrc + chunk_of<Geo, false>(w, t) * 32 + lane);
@@ -468,7 +498,7 @@ mma_bwd_kernel(const __nv_bfloat16* dy, const __nv_bfloat16* x, const TP* __rest
         X::mid_stages(m);
         X::pass2(m, v, hf);
         X::exchange_and_top(v, xbuf + Geo::XCHG_ONE, w, lane, 1 + rg);
-        uint4* dst = reinterpret_cast<uint4*>(dx + row * Geo::D);
+        uint4* dst = reinterpret_cast<uint4*>(dx + row * ld);
 #pragma unroll
         for (int idx = 0; idx < NT; ++idx)
             bwd_store_chunk(v[idx], dst + chunk_of<Geo, false>(w, idx) * 32 + lane);

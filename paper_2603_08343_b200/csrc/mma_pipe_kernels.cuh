@@ -125,7 +125,7 @@ __device__ __forceinline__ void read_staged8(const float* base, int c, int lane,
 template <int LOGD, int TB, int RG, int S, int MINB, typename TP>
 __global__ void __launch_bounds__(MmaGeo<LOGD, TB, RG>::THREADS, MINB)
 mma_fwd_pipe_kernel(const __nv_bfloat16* x, const TP* __restrict__ a, const TP* __restrict__ b,
-                    const __nv_bfloat16* resid, __nv_bfloat16* y, long long T, float inv_sqrt_d) {
+                    const __nv_bfloat16* resid, __nv_bfloat16* y, long long T, long long ld, float inv_sqrt_d) {
     using Geo = PipeGeo<LOGD, TB, RG, S, false>;
     using X = MmaXform<Geo>;
     constexpr int NT = Geo::NT;
@@ -141,6 +141,11 @@ mma_fwd_pipe_kernel(const __nv_bfloat16* x, const TP* __restrict__ a, const TP* 
 
     float* pa = reinterpret_cast<float*>(smem_raw + Geo::PARAM_OFFSET);
     float* pb = pa + Geo::D;
+    {   // block-diagonal form: blockIdx.y picks the channel group [y*D, (y+1)*D) of rows ld wide
+        const long long goff = static_cast<long long>(blockIdx.y) * Geo::D;
+        x += goff; y += goff; a += goff; b += goff;
+        if (resid != nullptr) resid += goff;
+    }
 
     if (elected) {
 #pragma unroll
@@ -158,7 +163,7 @@ mma_fwd_pipe_kernel(const __nv_bfloat16* x, const TP* __restrict__ a, const TP* 
     const long long first = static_cast<long long>(blockIdx.x) * RG + rg;
     auto issue = [&](int s, long long r) {
         mbar_expect_tx(full + s, Geo::ROW_BYTES);
-        bulk_load(ring + s * Geo::STAGE_BYTES, x + r * Geo::D, Geo::ROW_BYTES, full + s);
+        bulk_load(ring + s * Geo::STAGE_BYTES, x + r * ld, Geo::ROW_BYTES, full + s);
     };
     if (elected) {
 #pragma unroll
@@ -194,7 +199,7 @@ mma_fwd_pipe_kernel(const __nv_bfloat16* x, const TP* __restrict__ a, const TP* 
             // its pass 1: the stage is free
             if (elected && next_row < T) issue(stage, next_row);
         }
-        uint4* dst = reinterpret_cast<uint4*>(y + row * Geo::D);
+        uint4* dst = reinterpret_cast<uint4*>(y + row * ld);
 #pragma unroll
         for (int idx = 0; idx < NT; ++idx) {
             const int c = chunk_of<Geo, true>(w, idx);
@@ -202,7 +207,7 @@ mma_fwd_pipe_kernel(const __nv_bfloat16* x, const TP* __restrict__ a, const TP* 
             read_staged8(pa, c, lane, as);
             read_staged8(pb, c, lane, bs);
             if (resid != nullptr) {
-                const uint4 r = __ldcs(reinterpret_cast<const uint4*>(resid + row * Geo::D) + c * 32 + lane);
+                const uint4 r = __ldcs(reinterpret_cast<const uint4*>(resid + row * ld) + c * 32 + lane);
                 fwd_store_chunk_res(v[idx], as, bs, r, dst + c * 32 + lane);
             } else {
                 fwd_store_chunk(v[idx], as, bs, dst + c * 32 + lane);
@@ -216,7 +221,7 @@ mma_fwd_pipe_kernel(const __nv_bfloat16* x, const TP* __restrict__ a, const TP* 
 template <int LOGD, int TB, int RG, int S, int MINB, typename TP>
 __global__ void __launch_bounds__(MmaGeo<LOGD, TB, RG>::THREADS, MINB)
 mma_bwd_pipe_kernel(const __nv_bfloat16* dy, const __nv_bfloat16* x, const TP* __restrict__ a,
-                    __nv_bfloat16* dx, float* __restrict__ partials, long long T, float inv_sqrt_d) {
+                    __nv_bfloat16* dx, float* __restrict__ partials, long long T, long long ld, float inv_sqrt_d) {
     using Geo = PipeGeo<LOGD, TB, RG, S, true>;
     using X = MmaXform<Geo>;
     constexpr int NT = Geo::NT;
@@ -231,6 +236,10 @@ mma_bwd_pipe_kernel(const __nv_bfloat16* dy, const __nv_bfloat16* x, const TP* _
     const bool elected = (w == 0 && lane == 0);
 
     float* pa = reinterpret_cast<float*>(smem_raw + Geo::PARAM_OFFSET);
+    {
+        const long long goff = static_cast<long long>(blockIdx.y) * Geo::D;
+        dy += goff; x += goff; dx += goff; a += goff;
+    }
 
     if (elected) {
 #pragma unroll
@@ -254,8 +263,8 @@ mma_bwd_pipe_kernel(const __nv_bfloat16* dy, const __nv_bfloat16* x, const TP* _
     const long long first = static_cast<long long>(blockIdx.x) * RG + rg;
     auto issue = [&](int s, long long r) {
         mbar_expect_tx(full + s, Geo::STAGE_BYTES);
-        bulk_load(ring + s * Geo::STAGE_BYTES, x + r * Geo::D, Geo::ROW_BYTES, full + s);
-        bulk_load(ring + s * Geo::STAGE_BYTES + Geo::ROW_BYTES, dy + r * Geo::D, Geo::ROW_BYTES, full + s);
+        bulk_load(ring + s * Geo::STAGE_BYTES, x + r * ld, Geo::ROW_BYTES, full + s);
+        bulk_load(ring + s * Geo::STAGE_BYTES + Geo::ROW_BYTES, dy + r * ld, Geo::ROW_BYTES, full + s);
     };
     if (elected) {
 #pragma unroll
@@ -302,7 +311,7 @@ mma_bwd_pipe_kernel(const __nv_bfloat16* dy, const __nv_bfloat16* x, const TP* _
         if constexpr (Geo::WB > 0) {
             if (elected && next_row < T) issue(stage, next_row);
         }
-        uint4* dst = reinterpret_cast<uint4*>(dx + row * Geo::D);
+        uint4* dst = reinterpret_cast<uint4*>(dx + row * ld);
 #pragma unroll
         for (int idx = 0; idx < NT; ++idx)
             bwd_store_chunk(v[idx], dst + chunk_of<Geo, false>(w, idx) * 32 + lane);

@@ -57,6 +57,58 @@ int current_device(int* dev, int* sms) {
 bool is_pow2(int32_t d) { return d > 0 && (d & (d - 1)) == 0; }
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+size_t elem_bytes(int dtype) { return dtype == WHT_F32 ? 4 : 2; }
+
+#ifdef WHT_DEBUG
+// Debug build (-DWHT_DEBUG): every output and scratch buffer of a compute call is replaced by a device
+// buffer of the library's own with a guard region on either side, filled with a canary byte.  After the
+// kernels have run the stream is synchronised, the guards are read back and compared, and only then is
+// the payload copied into the caller's tensor.  A kernel that writes outside its output shows up as
+// WHT_ERR_GUARD instead of as silent corruption of a neighbouring tensor.  Slow by design (allocation,
+// synchronisation and a copy per call); the kernels themselves are the ones of the regular build.
+constexpr size_t kGuardBytes = 4096;
+constexpr unsigned char kCanary = 0xA5;
+
+class GuardedBuffer {
+  public:
+    GuardedBuffer() = default;
+    GuardedBuffer(const GuardedBuffer&) = delete;
+    GuardedBuffer& operator=(const GuardedBuffer&) = delete;
+    ~GuardedBuffer() { if (base_) cudaFree(base_); }
+
+    int init(size_t bytes, cudaStream_t s) {
+        bytes_ = bytes;
+        padded_ = (bytes + 15) / 16 * 16;
+        if (cudaMalloc(&base_, padded_ + 2 * kGuardBytes) != cudaSuccess) return cuda_fail(cudaGetLastError());
+        WHT_CUDA_TRY(cudaMemsetAsync(base_, kCanary, kGuardBytes, s));
+        WHT_CUDA_TRY(cudaMemsetAsync(static_cast<unsigned char*>(base_) + kGuardBytes + padded_, kCanary, kGuardBytes, s));
+        return WHT_OK;
+    }
+    void* data() const { return static_cast<unsigned char*>(base_) + kGuardBytes; }
+
+    // Waits for the stream, checks both guards, then hands the payload to `user` (none for scratch).
+    int finish(void* user, cudaStream_t s) {
+        WHT_CUDA_TRY(cudaStreamSynchronize(s));
+        unsigned char host[2][kGuardBytes];
+        WHT_CUDA_TRY(cudaMemcpy(host[0], base_, kGuardBytes, cudaMemcpyDeviceToHost));
+        WHT_CUDA_TRY(cudaMemcpy(host[1], static_cast<unsigned char*>(base_) + kGuardBytes + padded_, kGuardBytes,
+                                cudaMemcpyDeviceToHost));
+        for (int side = 0; side < 2; ++side)
+            for (size_t i = 0; i < kGuardBytes; ++i)
+                if (host[side][i] != kCanary) return WHT_ERR_GUARD;
+        if (user && bytes_ > 0) {
+            WHT_CUDA_TRY(cudaMemcpyAsync(user, data(), bytes_, cudaMemcpyDeviceToDevice, s));
+            WHT_CUDA_TRY(cudaStreamSynchronize(s));
+        }
+        return WHT_OK;
+    }
+
+  private:
+    void* base_ = nullptr;
+    size_t bytes_ = 0, padded_ = 0;
+};
+#endif
+
 int check_common(int64_t T, int32_t d, int dtype) {
     if (dtype != WHT_F32 && dtype != WHT_BF16 && dtype != WHT_BF16_PF32) return WHT_ERR_BAD_DTYPE;
     if (!is_pow2(d) || d < 8 || d > 32768) return WHT_ERR_BAD_DIM;
@@ -67,7 +119,11 @@ int check_common(int64_t T, int32_t d, int dtype) {
 bool umma_fwd_supported(int logd, int dtype) { return dtype != WHT_F32 && logd >= 10 && logd <= 13; }
 bool umma_bwd_supported(int logd, int dtype) { return dtype != WHT_F32 && logd >= 10 && logd <= 13; }
 
-bool mma_supported(int logd, int dtype) { return dtype != WHT_F32 && logd >= 9 && logd <= 13; }
+// d = 256 (two chained H_16 passes, one chunk per thread) serves the block-diagonal form and forced
+// variants; plain calls at d = 256 stay on the butterfly kernels, which keep such a row in registers too
+bool mma_supported(int logd, int dtype, bool with_256) {
+    return dtype != WHT_F32 && logd >= (with_256 ? 8 : 9) && logd <= 13;
+}
 
 // The persistent tcgen05 kernels win once there are a few hundred 32 KiB tiles (measured
 // cross-over against the direct-load kernels, CUDA-graph replay, d = 1024 ... 8192).
@@ -80,16 +136,20 @@ bool enough_work_for_tiles(int64_t T, int32_t d) {
 bool enough_rows_to_stream(int64_t T, int sms) { return T >= static_cast<int64_t>(sms) * 32; }
 
 // ------------------------------------------------------------------ selection
-int run_fwd(const FwdArgs& f, int64_t T, int32_t d, int dtype, cudaStream_t s, bool decode) {
+// `groups` > 1: block-diagonal form, d is the block width and the rows are groups * d elements apart
+// (the tcgen05 kernels copy whole tiles of contiguous rows and do not apply).
+int select_fwd(const FwdArgs& f, int64_t T, int32_t d, int dtype, cudaStream_t s, bool decode, int groups) {
     Ctx c{T, 0, 0, s};
     int rc = current_device(&c.dev, &c.sms);
     if (rc != WHT_OK) return rc;
+    c.groups = groups;
+    if (groups > 1) c.ld = static_cast<int64_t>(groups) * d;
     const int logd = log2_of(d);
-    if (umma_fwd_supported(logd, dtype) &&
+    if (groups == 1 && umma_fwd_supported(logd, dtype) &&
         (g_variant == 4 || (g_variant == 0 && enough_work_for_tiles(T, d)))) {
         return umma_fwd(logd, dtype, f, c);
     }
-    if (g_variant != 1 && mma_supported(logd, dtype)) {
+    if (g_variant != 1 && mma_supported(logd, dtype, groups > 1 || g_variant >= 2)) {
         const bool streamed = g_variant >= 3 || (g_variant == 0 && !decode && enough_rows_to_stream(T, c.sms));
         const bool few_rows = !streamed && (decode || (g_variant == 0 && T < static_cast<int64_t>(c.sms) * 4));
         return mma_fwd(logd, dtype, few_rows, streamed, f, c);
@@ -97,22 +157,87 @@ int run_fwd(const FwdArgs& f, int64_t T, int32_t d, int dtype, cudaStream_t s, b
     return bfly_fwd(logd, dtype, f, c);
 }
 
-int run_bwd(const BwdArgs& g, int64_t T, int32_t d, int dtype, cudaStream_t s) {
+int select_bwd(const BwdArgs& g, int64_t T, int32_t d, int dtype, cudaStream_t s, int groups) {
     Ctx c{T, 0, 0, s};
     int rc = current_device(&c.dev, &c.sms);
     if (rc != WHT_OK) return rc;
+    c.groups = groups;
+    if (groups > 1) c.ld = static_cast<int64_t>(groups) * d;
     const int logd = log2_of(d);
     // the backward is the heavier kernel: the tcgen05 form was never slower than the others from a
     // few hundred rows on
-    if (umma_bwd_supported(logd, dtype) &&
+    if (groups == 1 && umma_bwd_supported(logd, dtype) &&
         (g_variant == 4 || (g_variant == 0 && T * static_cast<int64_t>(d) >= (1ll << 18)))) {
         return umma_bwd(logd, dtype, g_bwd_operand_mode == 1, g, c);
     }
-    if (g_variant != 1 && mma_supported(logd, dtype)) {
+    if (g_variant != 1 && mma_supported(logd, dtype, groups > 1 || g_variant >= 2)) {
         const bool streamed = g_variant >= 3 || (g_variant == 0 && enough_rows_to_stream(T, c.sms));
         return mma_bwd(logd, dtype, streamed, g, c);
     }
     return bfly_bwd(logd, dtype, g, c);
+}
+
+// What the entry points call.  Regular build: the selection above.  Debug build: the same with every
+// output (and the scratch) replaced by a guarded buffer and checked after the call.
+int run_fwd(FwdArgs f, int64_t T, int32_t d, int dtype, cudaStream_t s, bool decode, int groups = 1) {
+#ifdef WHT_DEBUG
+    GuardedBuffer gy;
+    int rc = gy.init(static_cast<size_t>(T) * groups * d * elem_bytes(dtype), s);
+    if (rc != WHT_OK) return rc;
+    void* const user_y = f.y;
+    f.y = gy.data();
+    rc = select_fwd(f, T, d, dtype, s, decode, groups);
+    const int rg = gy.finish(rc == WHT_OK ? user_y : nullptr, s);
+    return rc != WHT_OK ? rc : rg;
+#else
+    return select_fwd(f, T, d, dtype, s, decode, groups);
+#endif
+}
+
+#ifdef WHT_DEBUG
+// Guarded stand-ins for dx, da, db and the scratch of a backward call; `launch` runs the real selection.
+template <typename Launch>
+int guarded_bwd(BwdArgs g, size_t dx_bytes, size_t vec_bytes, size_t need, cudaStream_t s, Launch launch) {
+    if (need > 0 && (g.ws == nullptr || g.ws_bytes < need)) return WHT_ERR_WORKSPACE;
+    GuardedBuffer gdx, gda, gdb, gws;
+    int rc = gdx.init(dx_bytes, s);
+    if (rc == WHT_OK) rc = gda.init(vec_bytes, s);
+    if (rc == WHT_OK) rc = gdb.init(vec_bytes, s);
+    if (rc == WHT_OK) rc = gws.init(need, s);
+    if (rc != WHT_OK) return rc;
+    void* const user_dx = g.dx;
+    float* const user_da = g.da;
+    float* const user_db = g.db;
+    g.dx = gdx.data();
+    g.da = static_cast<float*>(gda.data());
+    g.db = static_cast<float*>(gdb.data());
+    g.ws = gws.data();
+    g.ws_bytes = need;
+    rc = launch(g);
+    const bool ok = rc == WHT_OK;
+    const int r1 = gdx.finish(ok ? user_dx : nullptr, s);
+    const int r2 = gda.finish(ok ? user_da : nullptr, s);
+    const int r3 = gdb.finish(ok ? user_db : nullptr, s);
+    const int r4 = gws.finish(nullptr, s);
+    if (!ok) return rc;
+    return r1 != WHT_OK ? r1 : r2 != WHT_OK ? r2 : r3 != WHT_OK ? r3 : r4;
+}
+#endif
+
+int run_bwd(const BwdArgs& g, int64_t T, int32_t d, int dtype, cudaStream_t s, int groups = 1) {
+#ifdef WHT_DEBUG
+    if (!g.query_only) {
+        size_t need = 0;
+        BwdArgs q{nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, 0, true, &need};
+        int rc = select_bwd(q, T, d, dtype, s, groups);
+        if (rc != WHT_OK) return rc;
+        *g.need = need;
+        return guarded_bwd(g, static_cast<size_t>(T) * groups * d * elem_bytes(dtype),
+                           static_cast<size_t>(groups) * d * sizeof(float), need, s,
+                           [&](const BwdArgs& h) { return select_bwd(h, T, d, dtype, s, groups); });
+    }
+#endif
+    return select_bwd(g, T, d, dtype, s, groups);
 }
 
 int check_fwd_args(const void* x, const void* a, const void* b, void* y, int64_t T, int32_t d, int dtype) {
@@ -179,7 +304,7 @@ unsigned tp_neg_mask(int g, int r) {
     return m;
 }
 
-int run_bwd_tp(const TpCall& t, const BwdArgs& g, int64_t T, int32_t w, int dtype, cudaStream_t s) {
+int select_bwd_tp(const TpCall& t, const BwdArgs& g, int64_t T, int32_t w, int dtype, cudaStream_t s) {
     Ctx c{T, 0, 0, s};
     int rc = current_device(&c.dev, &c.sms);
     if (rc != WHT_OK) return rc;
@@ -191,6 +316,21 @@ int run_bwd_tp(const TpCall& t, const BwdArgs& g, int64_t T, int32_t w, int dtyp
         return umma_bwd_tp(logw, dtype, g_bwd_operand_mode == 1, t, g, c);
     }
     return bfly_bwd_tp(logw, dtype, t, g, c);
+}
+
+int run_bwd_tp(const TpCall& t, const BwdArgs& g, int64_t T, int32_t w, int dtype, cudaStream_t s) {
+#ifdef WHT_DEBUG
+    if (!g.query_only) {
+        size_t need = 0;
+        BwdArgs q{nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, 0, true, &need};
+        int rc = select_bwd_tp(t, q, T, w, dtype, s);
+        if (rc != WHT_OK) return rc;
+        *g.need = need;
+        return guarded_bwd(g, static_cast<size_t>(T) * w * elem_bytes(dtype), static_cast<size_t>(w) * sizeof(float),
+                           need, s, [&](const BwdArgs& h) { return select_bwd_tp(t, h, T, w, dtype, s); });
+    }
+#endif
+    return select_bwd_tp(t, g, T, w, dtype, s);
 }
 
 int query_bwd_bytes(int64_t T, int32_t d, int dtype, size_t* need) {
@@ -324,14 +464,7 @@ int wht_affine_fwd_grouped(const void* x, const void* a, const void* b, void* y,
     if (T > 0 && (!x || !y)) return WHT_ERR_NULL;
     if (!aligned16(x) || !aligned16(a) || !aligned16(b) || !aligned16(y)) return WHT_ERR_MISALIGNED;
     if (T == 0) return WHT_OK;
-    Ctx c{T, 0, 0, static_cast<cudaStream_t>(stream)};
-    c.ld = d;
-    rc = current_device(&c.dev, &c.sms);
-    if (rc != WHT_OK) return rc;
-    c.groups = d / block;
-    const int logb = log2_of(block);
-    const FwdArgs f{x, a, b, y};
-    return bfly_fwd(logb, dtype, f, c);
+    return run_fwd(FwdArgs{x, a, b, y}, T, block, dtype, static_cast<cudaStream_t>(stream), false, d / block);
 }
 
 int wht_affine_bwd_grouped(const void* dy, const void* x, const void* a, void* dx, float* da, float* db, int64_t T,
@@ -344,25 +477,16 @@ int wht_affine_bwd_grouped(const void* dy, const void* x, const void* a, void* d
     if (!aligned16(dy) || !aligned16(x) || !aligned16(a) || !aligned16(dx) || !aligned16(da) || !aligned16(db) ||
         !aligned16(workspace))
         return WHT_ERR_MISALIGNED;
-    Ctx c{T, 0, 0, static_cast<cudaStream_t>(stream)};
-    c.ld = d;
-    rc = current_device(&c.dev, &c.sms);
-    if (rc != WHT_OK) return rc;
-    c.groups = d / block;
-    const int logb = log2_of(block);
     size_t need = 0;
     const BwdArgs q{dy, x, a, dx, da, db, workspace, workspace_bytes, false, &need};
-    return bfly_bwd(logb, dtype, q, c);
+    return run_bwd(q, T, block, dtype, static_cast<cudaStream_t>(stream), d / block);
 }
 
 size_t wht_affine_bwd_grouped_workspace_bytes(int64_t T, int32_t d, int32_t block, int dtype) {
     if (check_grouped(T, d, block, dtype) != WHT_OK) return 0;
-    Ctx c{T, 0, 0, nullptr};
-    if (current_device(&c.dev, &c.sms) != WHT_OK) return 0;
-    c.groups = d / block;
     size_t need = 0;
     BwdArgs q{nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, 0, true, &need};
-    return bfly_bwd(log2_of(block), dtype, q, c) == WHT_OK ? need : 0;
+    return run_bwd(q, T, block, dtype, nullptr, d / block) == WHT_OK ? need : 0;
 }
 
 // ---- column-sharded (tensor-parallel) form: see the header.
@@ -383,14 +507,22 @@ int wht_affine_fwd_tp(const void* const* x_parts, const void* a, const void* b, 
     Ctx c{T, 0, 0, static_cast<cudaStream_t>(stream)};
     rc = current_device(&c.dev, &c.sms);
     if (rc != WHT_OK) return rc;
-    const FwdArgs f{nullptr, a, b, y};
+    FwdArgs f{nullptr, a, b, y};
     const int logw = log2_of(w);
     // bf16 rows of 1024 ... 4096 channels per rank with enough rows for 32 KiB tiles: tcgen05 form
-    if (dtype != WHT_F32 && logw >= 10 && logw <= 12 && (g_variant == 0 || g_variant == 4) &&
-        (g_variant == 4 || enough_work_for_tiles(T, w))) {
-        return umma_fwd_tp(logw, dtype, t, f, c);
-    }
-    return bfly_fwd_tp(logw, dtype, t, f, c);
+    const bool tensor_core = dtype != WHT_F32 && logw >= 10 && logw <= 12 && (g_variant == 0 || g_variant == 4) &&
+                             (g_variant == 4 || enough_work_for_tiles(T, w));
+#ifdef WHT_DEBUG
+    GuardedBuffer gy;
+    rc = gy.init(static_cast<size_t>(T) * w * elem_bytes(dtype), c.stream);
+    if (rc != WHT_OK) return rc;
+    f.y = gy.data();
+    rc = tensor_core ? umma_fwd_tp(logw, dtype, t, f, c) : bfly_fwd_tp(logw, dtype, t, f, c);
+    const int rg = gy.finish(rc == WHT_OK ? y : nullptr, c.stream);
+    return rc != WHT_OK ? rc : rg;
+#else
+    return tensor_core ? umma_fwd_tp(logw, dtype, t, f, c) : bfly_fwd_tp(logw, dtype, t, f, c);
+#endif
 }
 
 size_t wht_affine_bwd_tp_workspace_bytes(int64_t T, int32_t w, int32_t g, int dtype) {
@@ -483,6 +615,32 @@ int wht_affine_selftest_wait_expiry(uint32_t limit_us, unsigned int* out3, void*
     return launch_wait_expiry_selftest(limit_us, out3, static_cast<cudaStream_t>(stream));
 }
 
+int wht_affine_debug_build(void) {
+#ifdef WHT_DEBUG
+    return 1;
+#else
+    return 0;
+#endif
+}
+
+int wht_affine_debug_selftest_guard(int damage) {
+#ifdef WHT_DEBUG
+    if (damage < 0 || damage > 2) return WHT_ERR_BAD_VARIANT;
+    GuardedBuffer g;
+    int rc = g.init(1000, nullptr);
+    if (rc != WHT_OK) return rc;
+    unsigned char* payload = static_cast<unsigned char*>(g.data());
+    WHT_CUDA_TRY(cudaMemset(payload, 0, 1000));  // what a well-behaved kernel does
+    // one byte just outside the payload, on either side: inside the library's own allocation
+    if (damage == 1) WHT_CUDA_TRY(cudaMemset(payload - 1, 0, 1));
+    if (damage == 2) WHT_CUDA_TRY(cudaMemset(payload + 1008, 0, 1));
+    return g.finish(nullptr, nullptr);
+#else
+    (void)damage;
+    return WHT_ERR_BAD_VARIANT;
+#endif
+}
+
 int wht_affine_last_cuda_error(void) { return g_last_cuda_error; }
 
 const char* wht_affine_status_string(int status) {
@@ -498,6 +656,8 @@ const char* wht_affine_status_string(int status) {
         case WHT_ERR_BAD_VARIANT: return "WHT_ERR_BAD_VARIANT: unknown kernel variant";
         case WHT_ERR_DEVICE_WAIT:
             return "WHT_ERR_DEVICE_WAIT: a kernel gave up waiting for an async copy; that launch's results are invalid";
+        case WHT_ERR_GUARD:
+            return "WHT_ERR_GUARD: debug build: a kernel wrote outside an output or scratch buffer";
         default: return "unknown wht_status";
     }
 }

@@ -621,11 +621,14 @@ def test_bwd_bf16_operand_mode(B, name, rows):
 
 # ------------------------------------------------------------------ grouped (block-diagonal) form
 
+@pytest.mark.parametrize("variant", [0, 1, 3])
 @pytest.mark.parametrize("d,block,dtype,T", [(768, 256, wl.WHT_F32, 70), (768, 256, wl.WHT_BF16, 300),
                                              (1536, 512, wl.WHT_BF16_PF32, 129), (3072, 1024, wl.WHT_BF16, 33),
-                                             (96, 32, wl.WHT_F32, 1000), (1024, 1024, wl.WHT_BF16, 40)])
-def test_grouped_form(B, d, block, dtype, T):
-    B.wht_affine_set_variant(0)
+                                             (96, 32, wl.WHT_F32, 1000), (1024, 1024, wl.WHT_BF16, 40),
+                                             (768, 256, wl.WHT_BF16_PF32, 148 * 32 + 77), (1536, 512, wl.WHT_BF16, 148 * 32 + 5),
+                                             (512, 256, wl.WHT_BF16, 3), (6144, 2048, wl.WHT_BF16_PF32, 21)])
+def test_grouped_form(B, d, block, dtype, T, variant):
+    B.wht_affine_set_variant(variant)
     w = wl.Workload("grp", T, block, dtype, "normal", 800 + d, True, "")  # generators take a power of two:
     G = d // block                                                          # draw G blocks side by side
     x = torch.cat([wl.gen_full(wl.Workload("grp", T, block, dtype, "normal", 800 + d + g, True, ""), "x")
@@ -655,13 +658,12 @@ def test_grouped_form(B, d, block, dtype, T):
         assert_rows_bf16(to_f64(dx.cpu()), ref_dx, "grouped dx")
     assert_grad_vec(to_f64(da.cpu()), ref_da, "grouped da")
     assert_grad_vec(to_f64(db.cpu()), ref_db, "grouped db")
-    if G == 1:  # one group is the plain call (butterfly family)
-        B.wht_affine_set_variant(1)
+    if G == 1:  # one group is the plain call
         assert torch.equal(y, B.forward(xd, ad, bd))
-        B.wht_affine_set_variant(0)
     with pytest.raises(B.WhtError) as err:
         B.wht_affine_fwd_grouped(xd, ad, bd, y, T, d, 48, dtype)
     assert err.value.status == -2
+    B.wht_affine_set_variant(0)
 
 
 def test_autograd_wrapper(B):
