@@ -107,8 +107,49 @@ def build(force: bool = False, verbose: bool = False, debug: bool = False) -> st
     return lib
 
 
+def ptxas_summary() -> str:
+    """Rebuilds everything with -Xptxas -v and returns one line per kernel: registers per thread, spill
+    bytes, static shared memory (what the compiler reports; nothing is disassembled)."""
+    import io
+    from contextlib import redirect_stderr
+    buf = io.StringIO()
+    with redirect_stderr(buf):
+        build(verbose=True)
+    text = buf.getvalue()
+    try:
+        demangled = subprocess.run(["c++filt"], input=text, capture_output=True, text=True).stdout or text
+    except OSError:
+        demangled = text
+    rows, name, spill = [], None, (0, 0)
+    for line in demangled.splitlines():
+        m = re.search(r"Compiling entry function '(.+)' for", line)
+        if m:
+            name = m.group(1)
+            continue
+        m = re.search(r"(\d+) bytes stack frame, (\d+) bytes spill stores, (\d+) bytes spill loads", line)
+        if m:
+            spill = (int(m.group(2)), int(m.group(3)))
+            continue
+        m = re.search(r"Used (\d+) registers", line)
+        if m and name:
+            smem = re.search(r"(\d+) bytes smem", line)
+            short = re.sub(r"\(.*$", "", name).replace("void ", "").replace("wht::", "")
+            rows.append((short, int(m.group(1)), spill[0], spill[1], int(smem.group(1)) if smem else 0))
+            name, spill = None, (0, 0)
+    rows.sort()
+    out = ["kernel | registers/thread | spill stores B | spill loads B | static smem B",
+           "---|---|---|---|---"]
+    out += [f"{n} | {r} | {ss} | {sl} | {sm}" for n, r, ss, sl, sm in rows]
+    worst = [r for r in rows if r[2] or r[3]]
+    out.append("")
+    out.append(f"{len(rows)} kernels; with spills: " + (", ".join(f"{n} ({ss}/{sl} B)" for n, _, ss, sl, _ in worst) or "none"))
+    return "\n".join(out)
+
+
 if __name__ == "__main__":
-    if "--digest" in sys.argv:  # python -m paper_2603_08343_b200.build --digest a.cuh,b.cu
+    if "--ptxas-summary" in sys.argv:
+        print(ptxas_summary())
+    elif "--digest" in sys.argv:  # python -m paper_2603_08343_b200.build --digest a.cuh,b.cu
         print(source_digest(sys.argv[sys.argv.index("--digest") + 1].split(",")))
     else:
         print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, debug="--debug" in sys.argv))

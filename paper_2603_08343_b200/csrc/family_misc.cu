@@ -6,11 +6,13 @@ namespace wht_host {
 
 using namespace wht;
 
-int launch_finalize(const float* parts, int nparts, int d, float scale, float* da, float* db, cudaStream_t s) {
+int launch_finalize(const float* parts, int nparts, int d, float scale, float* da, float* db, cudaStream_t s,
+                    int groups) {
     if (d >= 32) {
-        launch_overlapped(dadb_finalize32_kernel, 2 * d / 32, 1024, 0, s, parts, nparts, d, scale, da, db);
+        launch_overlapped(dadb_finalize32_kernel, dim3(2 * d / 32, groups), 1024, 0, s, parts, nparts, d, scale, da, db);
     } else {
-        launch_overlapped(dadb_finalize_kernel, (2 * d + 255) / 256, 256, 0, s, parts, nparts, d, scale, da, db);
+        launch_overlapped(dadb_finalize_kernel, dim3((2 * d + 255) / 256, groups), 256, 0, s, parts, nparts, d, scale,
+                          da, db);
     }
     WHT_CUDA_TRY(cudaGetLastError());
     return WHT_OK;

@@ -149,12 +149,14 @@ int prepare_umma(Kernel kernel, int smem, int dev, int* cache) {
 }
 
 // ---- family_misc.cu: second pass of the backward, gradient sums, copy yardstick
-// da = scale * (sum of the partials' first slots), db = sum of their second slots
-int launch_finalize(const float* parts, int nparts, int d, float scale, float* da, float* db, cudaStream_t s);
+// da = scale * (sum of the partials' first slots), db = sum of their second slots; `groups` channel groups
+// of d channels each (block-diagonal form), group k's partials, da and db following those of group k - 1
+int launch_finalize(const float* parts, int nparts, int d, float scale, float* da, float* db, cudaStream_t s,
+                    int groups = 1);
 int launch_copy_rows(const void* src, void* dst, long long n16, int sms, cudaStream_t s);
 
 // Common tail of every backward launcher: size the scratch, check it, launch, then the second pass
-// (one per channel group; `grid` is the CTA count per group).
+// (`grid` is the CTA count per channel group).
 template <typename Launch>
 int run_bwd_with_grid(const BwdArgs& g, const Ctx& c, int grid, int d, Launch launch, float scale = 0.0f) {
     *g.need = static_cast<size_t>(grid) * c.groups * 2 * d * sizeof(float);
@@ -164,13 +166,8 @@ int run_bwd_with_grid(const BwdArgs& g, const Ctx& c, int grid, int d, Launch la
         launch(grid);
         WHT_CUDA_TRY(cudaGetLastError());
     }
-    for (int grp = 0; grp < c.groups; ++grp) {
-        const int rc = launch_finalize(static_cast<const float*>(g.ws) + static_cast<size_t>(grp) * grid * 2 * d, grid, d,
-                                       scale > 0.0f ? scale : inv_sqrt(d), g.da + static_cast<size_t>(grp) * d,
-                                       g.db + static_cast<size_t>(grp) * d, c.stream);
-        if (rc != WHT_OK) return rc;
-    }
-    return WHT_OK;
+    return launch_finalize(static_cast<const float*>(g.ws), grid, d, scale > 0.0f ? scale : inv_sqrt(d), g.da, g.db,
+                           c.stream, c.groups);
 }
 
 // ---- one dispatch function per family and direction (dtype: a wht_dtype; log2 of the width)

@@ -14,6 +14,11 @@ dadb_finalize32_kernel(const float* __restrict__ partials, int nparts, int d, fl
     __shared__ float red[32][33];
     grid_dependency_wait();  // the partials come from the kernel launched just before
     grid_launch_dependents();
+    {   // block-diagonal form: blockIdx.y is the channel group; its partials, da and db follow the group before
+        partials += static_cast<size_t>(blockIdx.y) * nparts * 2 * d;
+        da += static_cast<size_t>(blockIdx.y) * d;
+        db += static_cast<size_t>(blockIdx.y) * d;
+    }
     const int cx = threadIdx.x & 31;
     const int sl = threadIdx.x >> 5;
     const int j = blockIdx.x * 32 + cx;  // column in [0, 2d): da columns then db columns
@@ -39,6 +44,9 @@ dadb_finalize_kernel(const float* __restrict__ partials, int nparts, int d, floa
                      float* __restrict__ da, float* __restrict__ db) {
     grid_dependency_wait();  // the partials come from the kernel launched just before
     grid_launch_dependents();
+    partials += static_cast<size_t>(blockIdx.y) * nparts * 2 * d;  // channel group, as above
+    da += static_cast<size_t>(blockIdx.y) * d;
+    db += static_cast<size_t>(blockIdx.y) * d;
     const int j = blockIdx.x * blockDim.x + threadIdx.x;
     if (j >= 2 * d) return;
     const int which = j / d;

@@ -119,11 +119,8 @@ int check_common(int64_t T, int32_t d, int dtype) {
 bool umma_fwd_supported(int logd, int dtype) { return dtype != WHT_F32 && logd >= 10 && logd <= 13; }
 bool umma_bwd_supported(int logd, int dtype) { return dtype != WHT_F32 && logd >= 10 && logd <= 13; }
 
-// d = 256 (two chained H_16 passes, one chunk per thread) serves the block-diagonal form and forced
-// variants; plain calls at d = 256 stay on the butterfly kernels, which keep such a row in registers too
-bool mma_supported(int logd, int dtype, bool with_256) {
-    return dtype != WHT_F32 && logd >= (with_256 ? 8 : 9) && logd <= 13;
-}
+// bf16 rows of 256 ... 8192 elements (d = 256: two chained H_16 passes on one chunk per thread)
+bool mma_supported(int logd, int dtype) { return dtype != WHT_F32 && logd >= 8 && logd <= 13; }
 
 // The persistent tcgen05 kernels win once there are a few hundred 32 KiB tiles (measured
 // cross-over against the direct-load kernels, CUDA-graph replay, d = 1024 ... 8192).
@@ -149,8 +146,10 @@ int select_fwd(const FwdArgs& f, int64_t T, int32_t d, int dtype, cudaStream_t s
         (g_variant == 4 || (g_variant == 0 && enough_work_for_tiles(T, d)))) {
         return umma_fwd(logd, dtype, f, c);
     }
-    if (g_variant != 1 && mma_supported(logd, dtype, groups > 1 || g_variant >= 2)) {
-        const bool streamed = g_variant >= 3 || (g_variant == 0 && !decode && enough_rows_to_stream(T, c.sms));
+    if (g_variant != 1 && mma_supported(logd, dtype)) {
+        // rows of 256 or 512 elements: the direct-load kernels (which request a warp's next row ahead) beat
+        // the streamed ones at every size (measured)
+        const bool streamed = g_variant >= 3 || (g_variant == 0 && !decode && logd >= 10 && enough_rows_to_stream(T, c.sms));
         const bool few_rows = !streamed && (decode || (g_variant == 0 && T < static_cast<int64_t>(c.sms) * 4));
         return mma_fwd(logd, dtype, few_rows, streamed, f, c);
     }
@@ -170,8 +169,9 @@ int select_bwd(const BwdArgs& g, int64_t T, int32_t d, int dtype, cudaStream_t s
         (g_variant == 4 || (g_variant == 0 && T * static_cast<int64_t>(d) >= (1ll << 18)))) {
         return umma_bwd(logd, dtype, g_bwd_operand_mode == 1, g, c);
     }
-    if (g_variant != 1 && mma_supported(logd, dtype, groups > 1 || g_variant >= 2)) {
-        const bool streamed = g_variant >= 3 || (g_variant == 0 && enough_rows_to_stream(T, c.sms));
+    if (g_variant != 1 && mma_supported(logd, dtype)) {
+        // d = 256: direct loads (measured); wider rows are streamed once there are enough of them
+        const bool streamed = g_variant >= 3 || (g_variant == 0 && logd >= 9 && enough_rows_to_stream(T, c.sms));
         return mma_bwd(logd, dtype, streamed, g, c);
     }
     return bfly_bwd(logd, dtype, g, c);
