@@ -316,6 +316,8 @@ def section_decode(B):
         y = torch.empty_like(x)
         fn = lambda: B.wht_affine_fwd_decode(x, a, b, y, w.T, w.d, w.dtype)  # noqa: E731
         loop_us = 1e3 * time_loop(fn, 2000, warmup=20)
+        # the same call with its arguments marshalled once (binding.prepare): what a decode loop would use
+        prepared_us = 1e3 * time_loop(B.prepare("wht_affine_fwd_decode", x, a, b, y, w.T, w.d, w.dtype), 4000, warmup=20)
         # CUDA-graph replay of 50 back-to-back calls: per-call device time without launch overhead
         s = torch.cuda.Stream()
         with torch.cuda.stream(s):
@@ -327,7 +329,8 @@ def section_decode(B):
                 for _ in range(50):
                     B.wht_affine_fwd_decode(x, a, b, y, w.T, w.d, w.dtype)
             graph_us = 1e3 * time_loop(g.replay, 40, warmup=3) / 50
-        out[f"T{T}"] = {"stream_loop_us_per_call": loop_us, "graph_replay_us_per_call": graph_us}
+        out[f"T{T}"] = {"stream_loop_us_per_call": loop_us, "prepared_stream_loop_us_per_call": prepared_us,
+                        "graph_replay_us_per_call": graph_us}
     out["d"] = w0.d
     return out
 
@@ -823,7 +826,8 @@ def run_ours(args, rank: int, world: int, local_rank: int):
             pc[f"{name}_bwd_pair_mode"] = {"us": sec.get("bwd_pair_mode_us"),
                                            "frac": sec.get("bwd_pair_mode_frac_of_measured_peak")}
             pc[f"{name}_dense_gemm_us"] = sec.get("dense_gemm_bf16_us")
-        pc["decode_us_per_call"] = {k: {"graph": v["graph_replay_us_per_call"], "stream_loop": v["stream_loop_us_per_call"]}
+        pc["decode_us_per_call"] = {k: {"graph": v["graph_replay_us_per_call"], "stream_loop": v["stream_loop_us_per_call"],
+                                        "prepared_stream_loop": v["prepared_stream_loop_us_per_call"]}
                                     for k, v in sections["decode"].items() if k.startswith("T")}
         out["roofline"]["per_config"] = pc
     print(json.dumps(compact(out)))

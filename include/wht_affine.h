@@ -238,18 +238,20 @@ int wht_affine_reduce_grads(const float* parts, int32_t n, int32_t d, float* da,
 size_t wht_affine_bwd_workspace_bytes(int64_t T, int32_t d, int dtype);
 
 /*
- * Kernel family used by the three compute calls (for A/B measurements):
- *   0 = automatic (default): for bf16 rows, the tcgen05 kernels when 1024 <= d <= 8192
- *       and there is enough work for their 32 KiB tiles (forward: T*d >= 4 Mi elements,
- *       8 Mi at d = 8192; backward: T*d >= 256 Ki), else the mma.sync kernels
- *       for 512 <= d <= 8192 (rows streamed through a shared-memory ring when there
- *       are many, loaded directly when there are few); butterfly otherwise;
+ * Kernel family used by the compute calls (for A/B measurements):
+ *   0 = automatic (default).  bf16 rows: the tcgen05 kernels when 1024 <= d <= 8192 and there is
+ *       enough work for their 32 KiB tiles (forward: T*d >= 4 Mi elements, 8 Mi at d = 8192;
+ *       backward: T*d >= 256 Ki); else the mma.sync kernels for 256 <= d <= 8192 (rows loaded
+ *       directly when they are few or narrow, streamed through a shared-memory ring otherwise);
+ *       butterfly otherwise and for fp32 rows;
  *   1 = butterfly (registers + warp shuffles + shared memory), every d and dtype;
  *   2 = mma.sync tensor-core assisted with direct row loads;
  *   3 = mma.sync tensor-core assisted with streamed rows;
- *   4 = tcgen05: rows copied into shared memory as they are and multiplied by H_128
- *       on the tensor core (accumulators in tensor memory), the rest in registers.
- * A variant that does not support the requested (d, dtype) falls back (4 -> 3 -> 1).
+ *   4 = tcgen05: rows copied into shared memory as they are and multiplied by H_128 on the
+ *       tensor core (accumulators in tensor memory), the rest in registers;
+ *   5 = as 4, the backward with half-size products (H_64, two accumulators side by side in the
+ *       lanes of tensor memory, one more register stage) where d <= 4096.
+ * A variant that does not support the requested (d, dtype) falls back (5 -> 4 -> 3 -> 1).
  * Process-wide; not meant to be changed while calls are in flight.
  */
 int wht_affine_set_variant(int variant);

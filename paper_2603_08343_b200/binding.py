@@ -138,6 +138,38 @@ def wht_affine_fwd_decode(x, a, b, y, T: int, d: int, dtype: int, stream=None) -
            "wht_affine_fwd_decode")
 
 
+class PreparedCall:
+    """One call of the C ABI with its arguments marshalled once.
+
+    The plain wrappers look up the current stream, check every tensor and box every pointer on each call,
+    about 7 us of Python per call -- several times the device time of a decode-sized forward.  A loop that
+    repeats the same call on the same buffers (one decode step after another) prepares it once and then
+    pays one foreign call per launch.  The tensors must stay alive and in place; the stream is fixed at
+    preparation time.
+    """
+    __slots__ = ("_fn", "_args", "_where", "_keep")
+
+    def __init__(self, fn, args, where, keep):
+        self._fn, self._args, self._where, self._keep = fn, args, where, keep
+
+    def __call__(self) -> None:
+        rc = self._fn(*self._args)
+        if rc != 0:
+            raise WhtError(rc, self._where)
+
+
+def prepare(name: str, *args, stream=None) -> PreparedCall:
+    """Prepares `name(*args, stream)` of the C ABI: tensors become device pointers, integers stay.
+    E.g. prepare("wht_affine_fwd_decode", x, a, b, y, T, d, dtype)."""
+    if name not in EXPORTS:
+        raise ValueError(f"{name} is not an entry point of the library")
+    tensors = [t for t in args if isinstance(t, torch.Tensor)]
+    _require_cuda(*tensors)
+    marshalled = [_ptr(t) if isinstance(t, torch.Tensor) else t for t in args]
+    marshalled.append(_stream(stream))
+    return PreparedCall(getattr(_lib, name), tuple(marshalled), name, tensors)
+
+
 def wht_affine_bwd(dy, x, a, dx, da, db, T: int, d: int, dtype: int, stream=None) -> None:
     _require_cuda(dy, x, a, dx, da, db)
     _check(_lib.wht_affine_bwd(_ptr(dy), _ptr(x), _ptr(a), _ptr(dx), _ptr(da), _ptr(db), T, d, dtype,

@@ -180,7 +180,8 @@ int mma_bwd(int logd, int dtype, bool streamed, const BwdArgs& g, const Ctx& c);
 int umma_fwd(int logd, int dtype, const FwdArgs& f, const Ctx& c);                      // family_umma_fwd.cu
 int umma_fwd_tp(int logw, int dtype, const TpCall& t, const FwdArgs& f, const Ctx& c);
 // g_hi_lo: g enters the second product as a bf16 pair hi + lo (default) or rounded to bf16 once
-int umma_bwd(int logd, int dtype, bool g_hi_lo, const BwdArgs& g, const Ctx& c);        // family_umma_bwd.cu
+// half_size: products with H_64 instead of H_128 (d <= 4096; wider rows take the full-size kernel)
+int umma_bwd(int logd, int dtype, bool g_hi_lo, bool half_size, const BwdArgs& g, const Ctx& c);  // family_umma_bwd.cu
 
 // Self-test of the bounded waits (family_umma_fwd.cu): a one-CTA kernel whose wait runs out after limit_us.
 int launch_wait_expiry_selftest(uint32_t limit_us, unsigned int* out, cudaStream_t s);

@@ -143,7 +143,7 @@ int select_fwd(const FwdArgs& f, int64_t T, int32_t d, int dtype, cudaStream_t s
     if (groups > 1) c.ld = static_cast<int64_t>(groups) * d;
     const int logd = log2_of(d);
     if (groups == 1 && umma_fwd_supported(logd, dtype) &&
-        (g_variant == 4 || (g_variant == 0 && enough_work_for_tiles(T, d)))) {
+        (g_variant >= 4 || (g_variant == 0 && enough_work_for_tiles(T, d)))) {
         return umma_fwd(logd, dtype, f, c);
     }
     if (g_variant != 1 && mma_supported(logd, dtype)) {
@@ -166,8 +166,10 @@ int select_bwd(const BwdArgs& g, int64_t T, int32_t d, int dtype, cudaStream_t s
     // the backward is the heavier kernel: the tcgen05 form was never slower than the others from a
     // few hundred rows on
     if (groups == 1 && umma_bwd_supported(logd, dtype) &&
-        (g_variant == 4 || (g_variant == 0 && T * static_cast<int64_t>(d) >= (1ll << 18)))) {
-        return umma_bwd(logd, dtype, g_bwd_operand_mode == 1, g, c);
+        (g_variant >= 4 || (g_variant == 0 && T * static_cast<int64_t>(d) >= (1ll << 18)))) {
+        // half-size products: measured 2-4 % faster in long runs at d = 1024 and 2048, 1 % slower at 4096
+        const bool half_size = g_variant == 5 || (g_variant == 0 && logd <= 11);
+        return umma_bwd(logd, dtype, g_bwd_operand_mode == 1, half_size, g, c);
     }
     if (g_variant != 1 && mma_supported(logd, dtype)) {
         // d = 256: direct loads (measured); wider rows are streamed once there are enough of them
@@ -312,7 +314,7 @@ int select_bwd_tp(const TpCall& t, const BwdArgs& g, int64_t T, int32_t w, int d
     // bf16 rows of 1024 ... 4096 channels per rank on two or more ranks: tcgen05 form (as in the plain
     // backward it pays from a few hundred rows on)
     if (dtype != WHT_F32 && logw >= 10 && logw <= 12 && t.g >= 2 &&
-        (g_variant == 4 || (g_variant == 0 && T * static_cast<int64_t>(w) >= (1ll << 18)))) {
+        (g_variant >= 4 || (g_variant == 0 && T * static_cast<int64_t>(w) >= (1ll << 18)))) {
         return umma_bwd_tp(logw, dtype, g_bwd_operand_mode == 1, t, g, c);
     }
     return bfly_bwd_tp(logw, dtype, t, g, c);
@@ -510,8 +512,8 @@ int wht_affine_fwd_tp(const void* const* x_parts, const void* a, const void* b, 
     FwdArgs f{nullptr, a, b, y};
     const int logw = log2_of(w);
     // bf16 rows of 1024 ... 4096 channels per rank with enough rows for 32 KiB tiles: tcgen05 form
-    const bool tensor_core = dtype != WHT_F32 && logw >= 10 && logw <= 12 && (g_variant == 0 || g_variant == 4) &&
-                             (g_variant == 4 || enough_work_for_tiles(T, w));
+    const bool tensor_core = dtype != WHT_F32 && logw >= 10 && logw <= 12 && (g_variant == 0 || g_variant >= 4) &&
+                             (g_variant >= 4 || enough_work_for_tiles(T, w));
 #ifdef WHT_DEBUG
     GuardedBuffer gy;
     rc = gy.init(static_cast<size_t>(T) * w * elem_bytes(dtype), c.stream);
@@ -567,7 +569,7 @@ int wht_affine_reduce_grads(const float* parts, int32_t n, int32_t d, float* da,
 }
 
 int wht_affine_set_variant(int variant) {
-    if (variant < 0 || variant > 4) return WHT_ERR_BAD_VARIANT;
+    if (variant < 0 || variant > 5) return WHT_ERR_BAD_VARIANT;
     g_variant = variant;
     return WHT_OK;
 }

@@ -48,7 +48,7 @@ CASES = [(256, wl.WHT_F32, 64), (8, wl.WHT_F32, 1031), (64, wl.WHT_BF16, 257), (
          (4096, wl.WHT_BF16, 37), (8192, wl.WHT_BF16_PF32, 21), (16384, wl.WHT_F32, 5), (32768, wl.WHT_BF16, 3)]
 
 
-@pytest.mark.parametrize("variant", [0, 1, 2, 3, 4])
+@pytest.mark.parametrize("variant", [0, 1, 2, 3, 4, 5])
 def test_small_parity_cases_through_the_guarded_build(libs, variant):
     B, dbg = libs
     B.wht_affine_set_variant(variant)

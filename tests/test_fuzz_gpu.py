@@ -39,7 +39,7 @@ def _cases(seed, count):
         logd = rng.choice([3, 5, 8, 9, 10, 10, 11, 11, 12, 12, 13, 13, 14])
         d = 1 << logd
         dtype = rng.choice([wl.WHT_F32, wl.WHT_BF16, wl.WHT_BF16_PF32, wl.WHT_BF16_PF32, wl.WHT_BF16])
-        variant = rng.choice([0, 0, 1, 2, 3, 4, 4])
+        variant = rng.choice([0, 0, 1, 2, 3, 4, 5])
         max_rows = max(1, min(6000, (1 << 25) // (d * d // 64 + 1)))  # keeps the dense oracle to a fraction of a second
         if 10 <= logd <= 13 and rng.random() < 0.5:
             tile = 128 // (8 * (d // 1024))

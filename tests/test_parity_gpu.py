@@ -17,7 +17,9 @@ from paper_2603_08343_b200 import workloads as wl
 
 pytestmark = pytest.mark.gpu
 
-VARIANTS = [1, 2, 3, 4]  # butterfly; mma.sync with direct loads; with streamed rows; tcgen05 (each falls back where unsupported)
+# butterfly; mma.sync with direct loads; with streamed rows; tcgen05; tcgen05 with half-size products in the
+# backward (each falls back where unsupported)
+VARIANTS = [1, 2, 3, 4, 5]
 
 
 @pytest.fixture(scope="module")
@@ -113,6 +115,25 @@ def test_prefill_full(B, variant):
 def test_decode(B, T, variant):
     w = wl.CONFIGS["decode"].with_rows(T)
     _run_case(B, w, variant, decode=True, bwd=False)
+
+
+def test_prepared_call_equals_the_plain_wrapper(B):
+    B.wht_affine_set_variant(0)
+    w = wl.CONFIGS["decode"].with_rows(8)
+    x = wl.gen_full(w, "x").cuda()
+    a, b = (t.cuda() for t in wl.gen_params(w))
+    y1 = B.forward(x, a, b, decode=True)
+    y2 = torch.zeros_like(x)
+    call = B.prepare("wht_affine_fwd_decode", x, a, b, y2, w.T, w.d, w.dtype)
+    call()
+    call()
+    torch.cuda.synchronize()
+    assert torch.equal(y1, y2)
+    bad = B.prepare("wht_affine_fwd_decode", x, a, b, y2, w.T, 100, w.dtype)  # errors surface at the call
+    with pytest.raises(B.WhtError):
+        bad()
+    with pytest.raises(ValueError):
+        B.prepare("no_such_call", x)
 
 
 def test_decode_equals_fwd_bitwise(B):
@@ -357,6 +378,7 @@ def test_tcgen05_kernels_on_many_rows(B):
                         (4096, wl.WHT_BF16, 148 * 4 * 3 + 1), (8192, wl.WHT_BF16_PF32, 148 * 2 * 3 + 1)]:
         w = wl.Workload("tc5", T, d, dtype, "normal", 400 + d, True, "")
         _run_case(B, w, 4)
+        _run_case(B, w, 5)
     B.wht_affine_device_status()
 
 
@@ -546,7 +568,7 @@ def _round_to_bf16_bits(v64: np.ndarray) -> np.ndarray:
     return (u >> 16).astype(np.uint16)
 
 
-@pytest.mark.parametrize("variant", [0, 3, 4])
+@pytest.mark.parametrize("variant", [0, 3, 4, 5])
 def test_outputs_are_the_correctly_rounded_values_almost_everywhere(B, variant):
     # fp32 accumulation then ONE rounding: the stored bf16 must be the nearest bf16 of the exact
     # result except where the fp32 error (~1e-7 relative to the row scale) straddles a rounding
@@ -586,13 +608,14 @@ def test_outputs_are_the_correctly_rounded_values_almost_everywhere(B, variant):
 # ------------------------------------------------------------------ bf16-operand mode of the tcgen05 backward
 
 @pytest.mark.parametrize("name,rows", [("training", 148 * 8 * 2 + 3), ("large", 148 * 2 * 2 + 1), ("prefill", 148 * 16 + 5)])
-def test_bwd_bf16_operand_mode(B, name, rows):
+@pytest.mark.parametrize("variant", [4, 5])
+def test_bwd_bf16_operand_mode(B, name, rows, variant):
     """The two settings of wht_affine_set_bwd_operand_mode.  In the default one g = (a/sqrt d) (.) dy is
     rounded to bf16 once before the second +-1 product; with mode 1 it is carried as a bf16 pair.  In both,
     dx must meet the bound for bf16 storage, 1e-2 * max|dx_row|, on every row of the chain rule of Eq. 1
     -- also on the heavy-tailed rows of the Large config, where one spike dominates a row -- with half
     of the bound to spare, and da, db (which never pass through g) must have the same bits in both."""
-    B.wht_affine_set_variant(0)
+    B.wht_affine_set_variant(variant)
     base = wl.CONFIGS[name]
     w = wl.Workload(base.name, rows, base.d, base.dtype, base.dist, base.seed + 7, True, "")
     x, dy = wl.gen_full(w, "x"), wl.gen_full(w, "dy")
@@ -616,6 +639,7 @@ def test_bwd_bf16_operand_mode(B, name, rows):
     assert_grad_vec(to_f64(db0.cpu()), ref_db, f"{name} db")
     with pytest.raises(B.WhtError):
         B.wht_affine_set_bwd_operand_mode(2)
+    B.wht_affine_set_variant(0)
     B.wht_affine_device_status()
 
 
