@@ -41,7 +41,7 @@ METRIC = "wht_affine_tokens_per_s_fwd_bwd"
 UNIT = "tokens/s"
 # DRAM bytes of one launch of the dominant kernel come from the ncu capture recorded in this file, in a
 # line "traffic_record: ..." that also names the kernel and a digest of the sources it was built from.
-TRAFFIC_PROFILE = os.path.join("profiles", "umma_bwd_training_d2048.txt")
+TRAFFIC_PROFILE = os.path.join("profiles", "umma64_bwd_training_d2048.txt")
 
 
 def ncu_traffic(workload: str, rows: int):
