@@ -396,58 +396,56 @@ mma_fwd_kernel(const __nv_bfloat16* x, const TP* __restrict__ a, const TP* __res
 
     int parity = 0;
     const long long stride = static_cast<long long>(gridDim.x) * RG;
-    // Requesting the warp's next row before this one is transformed was measured and does not pay in the
-    // forward (d = 256: 5 % slower, d = 512: the same); the hook stays for the backward's use of it.
-    constexpr bool PREFETCH = false;
+    // Narrow rows (one or two 128-bit loads per lane and row) put little data in flight per warp, and the
+    // registers allow only ~40 warps per SM: a warp requests U of its rows before it transforms the first.
+    constexpr int U = (Geo::WB == 0 && NT <= 2) ? 4 / NT : 1;
     auto load_row = [&](long long r, uint4 (&dst)[NT]) {
         const uint4* src = reinterpret_cast<const uint4*>(x + r * ld);
 #pragma unroll
         for (int t = 0; t < NT; ++t) dst[t] = __ldcs(src + chunk_of<Geo, false>(w, t) * 32 + lane);
     };
-    uint4 ahead[NT];
-    const long long first = static_cast<long long>(blockIdx.x) * RG + rg;
-    if (PREFETCH && first < T) load_row(first, ahead);
-    for (long long row = first; row < T; row += stride) {
-        uint4 raw[NT];
-        if constexpr (PREFETCH) {
+    for (long long row0 = static_cast<long long>(blockIdx.x) * RG + rg; row0 < T; row0 += U * stride) {
+        uint4 raws[U][NT];
 #pragma unroll
-            for (int t = 0; t < NT; ++t) raw[t] = ahead[t];
-            if (row + stride < T) load_row(row + stride, ahead);
-        } else {
-            load_row(row, raw);
-        }
-        uint4 res[NT];
-        if (resid != nullptr) {  // the residual chunks too, ahead of the transform
+        for (int u = 0; u < U; ++u)
+            if (row0 + u * stride < T) load_row(row0 + u * stride, raws[u]);  // uniform over the warp
 #pragma unroll
-            for (int idx = 0; idx < NT; ++idx)
-                res[idx] = __ldcs(reinterpret_cast<const uint4*>(resid + row * ld) +
-                                  chunk_of<Geo, true>(w, idx) * 32 + lane);
-        }
-        F2 m[NT][2][2];
-        F2 v[NT][4];
-        X::pass1_raw(raw, m, hf);
-        X::mid_stages(m);
-        X::pass2(m, v, hf);
-        X::exchange_and_top(v, xbuf + parity * Geo::XCHG_ONE, w, lane, 1 + rg);
-        parity ^= 1;
-        uint4* dst = reinterpret_cast<uint4*>(y + row * ld);
+        for (int u = 0; u < U; ++u) {
+            const long long row = row0 + u * stride;
+            if (row >= T) break;
+            uint4 res[NT];
+            if (resid != nullptr) {  // the residual chunks too, ahead of the transform
 #pragma unroll
-        for (int idx = 0; idx < NT; ++idx) {
-            const int c = chunk_of<Geo, true>(w, idx);
-            F2 as[4], bs[4];
-            if constexpr (PRELOAD) {
-#pragma unroll
-                for (int j = 0; j < 4; ++j) { as[j] = pas[idx][j]; bs[j] = pbs[idx][j]; }
-            } else {
-                load_params8(a + (c * 32 + lane) * 8, as);
-                load_params8(b + (c * 32 + lane) * 8, bs);
-#pragma unroll
-                for (int j = 0; j < 4; ++j) as[j] = mul2(as[j], rs2);
+                for (int idx = 0; idx < NT; ++idx)
+                    res[idx] = __ldcs(reinterpret_cast<const uint4*>(resid + row * ld) +
+                                      chunk_of<Geo, true>(w, idx) * 32 + lane);
             }
-            if (resid != nullptr) {
-                fwd_store_chunk_res(v[idx], as, bs, res[idx], dst + c * 32 + lane);
-            } else {
-                fwd_store_chunk(v[idx], as, bs, dst + c * 32 + lane);
+            F2 m[NT][2][2];
+            F2 v[NT][4];
+            X::pass1_raw(raws[u], m, hf);
+            X::mid_stages(m);
+            X::pass2(m, v, hf);
+            X::exchange_and_top(v, xbuf + parity * Geo::XCHG_ONE, w, lane, 1 + rg);
+            parity ^= 1;
+            uint4* dst = reinterpret_cast<uint4*>(y + row * ld);
+#pragma unroll
+            for (int idx = 0; idx < NT; ++idx) {
+                const int c = chunk_of<Geo, true>(w, idx);
+                F2 as[4], bs[4];
+                if constexpr (PRELOAD) {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) { as[j] = pas[idx][j]; bs[j] = pbs[idx][j]; }
+                } else {
+                    load_params8(a + (c * 32 + lane) * 8, as);
+                    load_params8(b + (c * 32 + lane) * 8, bs);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) as[j] = mul2(as[j], rs2);
+                }
+                if (resid != nullptr) {
+                    fwd_store_chunk_res(v[idx], as, bs, res[idx], dst + c * 32 + lane);
+                } else {
+                    fwd_store_chunk(v[idx], as, bs, dst + c * 32 + lane);
+                }
             }
         }
     }
@@ -483,9 +481,10 @@ mma_bwd_kernel(const __nv_bfloat16* dy, const __nv_bfloat16* x, const TP* __rest
     }
 
     const long long stride = static_cast<long long>(gridDim.x) * RG;
-    // d = 512 (two 128-bit loads per tensor, thread and row): the warp's next row is requested before this one
-    // is transformed, measured 7 % faster; at d = 256 the extra registers cost more than the loads in flight gain
-    constexpr bool PREFETCH = NT == 2;
+    // A warp may request U of its rows (x and dy) before it transforms the first.  Measured: with two tensors
+    // and the column sums in registers this costs occupancy and loses at every narrow width (d = 256: 0.885 ->
+    // 0.73 of the copy rate, d = 512: 0.84 -> 0.61), unlike in the forward; so U = 1, the hook stays.
+    constexpr int U = 1;
     auto load_rows = [&](long long r, uint4 (&dx_)[NT], uint4 (&ddy)[NT]) {
         const uint4* xsrc = reinterpret_cast<const uint4*>(x + r * ld);
         const uint4* dysrc = reinterpret_cast<const uint4*>(dy + r * ld);
@@ -494,44 +493,42 @@ mma_bwd_kernel(const __nv_bfloat16* dy, const __nv_bfloat16* x, const TP* __rest
 #pragma unroll
         for (int t = 0; t < NT; ++t) ddy[t] = __ldcs(dysrc + chunk_of<Geo, true>(w, t) * 32 + lane);
     };
-    uint4 ahead_x[NT], ahead_dy[NT];
-    const long long first = static_cast<long long>(blockIdx.x) * RG + rg;
-    if (PREFETCH && first < T) load_rows(first, ahead_x, ahead_dy);
-    for (long long row = first; row < T; row += stride) {
-        uint4 raw[NT], rawdy[NT];
-        if constexpr (PREFETCH) {
+    for (long long row0 = static_cast<long long>(blockIdx.x) * RG + rg; row0 < T; row0 += U * stride) {
+        uint4 raws[U][NT], rawdys[U][NT];
 #pragma unroll
-            for (int t = 0; t < NT; ++t) { raw[t] = ahead_x[t]; rawdy[t] = ahead_dy[t]; }
-            if (row + stride < T) load_rows(row + stride, ahead_x, ahead_dy);
-        } else {
-            load_rows(row, raw, rawdy);
+        for (int u = 0; u < U; ++u)
+            if (row0 + u * stride < T) load_rows(row0 + u * stride, raws[u], rawdys[u]);  // uniform over the warp
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const long long row = row0 + u * stride;
+            if (row >= T) break;
+            F2 m[NT][2][2];
+            F2 v[NT][4];
+            // u = x H, delivered in layout B
+            X::pass1_raw(raws[u], m, hf);
+            X::mid_stages(m);
+            X::pass2(m, v, hf);
+            X::exchange_and_top(v, xbuf, w, lane, 1 + rg);
+            // da, db partial sums and g = a (.) dy, all in layout B
+#pragma unroll
+            for (int idx = 0; idx < NT; ++idx) {
+                const int c = chunk_of<Geo, true>(w, idx);
+                F2 as[4];
+                load_params8(a + (c * 32 + lane) * 8, as);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) as[j] = mul2(as[j], rs2);
+                bwd_mid_chunk(v[idx], rawdys[u][idx], as, da_acc[idx], db_acc[idx]);
+            }
+            // dx = (g H)/sqrt(d): layout B in, layout A out
+            X::pass1_f32(v, m, hf);
+            X::mid_stages(m);
+            X::pass2(m, v, hf);
+            X::exchange_and_top(v, xbuf + Geo::XCHG_ONE, w, lane, 1 + rg);
+            uint4* dst = reinterpret_cast<uint4*>(dx + row * ld);
+#pragma unroll
+            for (int idx = 0; idx < NT; ++idx)
+                bwd_store_chunk(v[idx], dst + chunk_of<Geo, false>(w, idx) * 32 + lane);
         }
-        F2 m[NT][2][2];
-        F2 v[NT][4];
-        // u = x H, delivered in layout B
-        X::pass1_raw(raw, m, hf);
-        X::mid_stages(m);
-        X::pass2(m, v, hf);
-        X::exchange_and_top(v, xbuf, w, lane, 1 + rg);
-        // da, db partial sums and g = a (.) dy, all in layout B
-#pragma unroll
-        for (int idx = 0; idx < NT; ++idx) {
-            const int c = chunk_of<Geo, true>(w, idx);
-            F2 as[4];
-            load_params8(a + (c * 32 + lane) * 8, as);
-#pragma unroll
-            for (int j = 0; j < 4; ++j) as[j] = mul2(as[j], rs2);
-            bwd_mid_chunk(v[idx], rawdy[idx], as, da_acc[idx], db_acc[idx]);
-        }
-        // dx = (g H)/sqrt(d): layout B in, layout A out
-        X::pass1_f32(v, m, hf);
-        X::mid_stages(m);
-        X::pass2(m, v, hf);
-        X::exchange_and_top(v, xbuf + Geo::XCHG_ONE, w, lane, 1 + rg);
-        uint4* dst = reinterpret_cast<uint4*>(dx + row * ld);
-#pragma unroll
-        for (int idx = 0; idx < NT; ++idx)
-            bwd_store_chunk(v[idx], dst + chunk_of<Geo, false>(w, idx) * 32 + lane);
     }
     bwd_publish_partials<Geo>(da_acc, db_acc, smem, partials, rg, w, lane);
 }

@@ -594,15 +594,20 @@ umma_fwd_kernel(const __nv_bfloat16* x, const TP* __restrict__ a, const TP* __re
                 __syncwarp();
                 if (lane == 0) mbar_arrive(acc_empty + t);  // the accumulator is in registers now
 
+                // this thread's 16-byte chunk of piece 0 of its first row of the tile; FULL (every row of the
+                // tile exists: all tiles but the last of a ragged problem) drops the per-row test
+                const long long row_first = tile * Geo::ROWS + ch * Geo::RPW;
+                uint4* const dst_first = reinterpret_cast<uint4*>(y + row_first * Geo::D + m * 8);
+                auto rows_out = [&](auto full_tag) {
+                constexpr bool FULL = decltype(full_tag)::value;
 #pragma unroll
                 for (int rl = 0; rl < Geo::RPW; ++rl) {
-                    const long long row = tile * Geo::ROWS + ch * Geo::RPW + rl;
                     float v[Geo::R];
 #pragma unroll
                     for (int i = 0; i < Geo::R; ++i) v[i] = u[rl * Geo::R + i];
                     thread_stages<Geo::R>(v);
-                    if (row < T) {
-                        uint4* dst = reinterpret_cast<uint4*>(y + row * Geo::D + m * 8);
+                    if (FULL || row_first + rl < T) {
+                        uint4* dst = dst_first + rl * (Geo::D / 8);
 #pragma unroll
                         for (int p = 0; p < Geo::PIECES; ++p) {
                             F2 w[4];
@@ -627,6 +632,8 @@ umma_fwd_kernel(const __nv_bfloat16* x, const TP* __restrict__ a, const TP* __re
                         }
                     }
                 }
+                };
+                if ((tile + 1) * Geo::ROWS <= T) rows_out(TrueTag{}); else rows_out(FalseTag{});
             }
         }
     }

@@ -5,8 +5,8 @@
 //     dx_r = ( (sum_s H_g[r][s] (a_s (.) dy_s)) H_w ) / sqrt(d)
 //
 // The x side is what the column-sharded forward does: the tile of EVERY rank's x block is copied into
-// a ring slot (this GPU's memory or a peer mapping; plain bulk copies of one CTA for itself, never
-// multicast) and multiplied by H_128 into ONE accumulator, with the instruction descriptor's negate-A
+// a ring slot (this GPU's memory or a peer mapping; plain bulk copies that one CTA
+// issues for itself alone) and multiplied by H_128 into ONE accumulator, with the instruction descriptor's negate-A
 // bit where the sign is -1, so the signed sum is the tensor core's fp32 accumulation of exact +-1
 // products.  The dy side cannot be summed that way (every block has its own a_s), so each slot also
 // carries the block's dy tile and the epilogue threads accumulate sum_s +- (a_s/sqrt d) (.) dy_s in

@@ -130,3 +130,61 @@ def test_random_column_sharded_shapes_match_the_oracle(B, seed):
         assert np.max(np.abs(to_f64(da) - ref_da)) <= 1e-4 * np.max(np.abs(ref_da)), what + ": da"
         assert np.max(np.abs(to_f64(db) - ref_db)) <= 1e-4 * np.max(np.abs(ref_db)), what + ": db"
     B.wht_affine_set_bwd_operand_mode(0)
+
+
+def _grouped_cases(seed, count):
+    rng = random.Random(seed)
+    out = []
+    for case in range(count):
+        groups = rng.choice([2, 3, 3, 5, 6, 7])
+        logb = rng.choice([3, 5, 7, 8, 8, 9, 9, 10, 11])
+        block = 1 << logb
+        dtype = rng.choice([wl.WHT_F32, wl.WHT_BF16, wl.WHT_BF16_PF32, wl.WHT_BF16_PF32])
+        variant = rng.choice([0, 0, 1, 2, 3])
+        d = groups * block
+        max_rows = max(1, min(5000, (1 << 24) // (d * d // 64 + 1)))
+        out.append((case, groups, block, rng.randint(1, max_rows), dtype, variant))
+    return out
+
+
+@pytest.mark.parametrize("seed", [31])
+def test_random_block_diagonal_shapes_match_the_oracle(B, seed):
+    """The grouped form (d = groups * block, every block transformed on its own) over random group counts,
+    block widths, storage types and kernel families, against its plain block-diagonal definition."""
+    for case, groups, block, T, dtype, variant in _grouped_cases(seed, 24):
+        d = groups * block
+        gen = torch.Generator().manual_seed(9000 + 100 * seed + case)
+        io = torch.float32 if dtype == wl.WHT_F32 else torch.bfloat16
+        pt = torch.bfloat16 if dtype == wl.WHT_BF16 else torch.float32
+        x = torch.randn(T, d, generator=gen).to(io)
+        dy = torch.randn(T, d, generator=gen).to(io)
+        a = (torch.rand(d, generator=gen) + 0.5).to(pt)
+        b = (torch.randn(d, generator=gen) * 0.1).to(pt)
+        B.wht_affine_set_variant(variant)
+        xd, dyd, ad, bd = x.cuda(), dy.cuda(), a.cuda(), b.cuda()
+        y = torch.empty_like(xd)
+        B.wht_affine_fwd_grouped(xd, ad, bd, y, T, d, block, dtype)
+        ws = torch.empty(max(B.wht_affine_bwd_grouped_workspace_bytes(T, d, block, dtype), 16), dtype=torch.uint8, device="cuda")
+        dx = torch.empty_like(xd)
+        da, db = torch.empty(d, device="cuda"), torch.empty(d, device="cuda")
+        B.wht_affine_bwd_grouped(dyd, xd, ad, dx, da, db, T, d, block, dtype, ws)
+        torch.cuda.synchronize()
+        x64, dy64, a64, b64 = to_f64(x), to_f64(dy), to_f64(a), to_f64(b)
+        ref_y = oracle.wht_affine_fwd_grouped(x64, a64, b64, block)
+        ref_dx, ref_da, ref_db = oracle.wht_affine_bwd_grouped(dy64, x64, a64, block)
+        what = f"groups={groups} block={block} T={T} dtype={dtype} variant={variant}"
+        # the fp32 bound is per transform input: here the norm of the row's block, the smallest over the blocks
+        blocks_x = np.linalg.norm(x64.reshape(T, groups, block), axis=2).min(axis=1)
+        blocks_g = np.linalg.norm((a64[None, :] * dy64).reshape(T, groups, block), axis=2).min(axis=1)
+        if dtype == wl.WHT_F32:
+            # per block the error is bounded by 1e-5 of ITS norm; the largest block norm bounds the row's maximum
+            nx = np.linalg.norm(x64.reshape(T, groups, block), axis=2).max(axis=1)
+            ng = np.linalg.norm((a64[None, :] * dy64).reshape(T, groups, block), axis=2).max(axis=1)
+            assert _ratio_rows(to_f64(y.cpu()), ref_y, dtype, nx) <= 1.0, what + ": y"
+            assert _ratio_rows(to_f64(dx.cpu()), ref_dx, dtype, ng) <= 1.0, what + ": dx"
+        else:
+            assert _ratio_rows(to_f64(y.cpu()), ref_y, dtype, blocks_x) <= 1.0, what + ": y"
+            assert _ratio_rows(to_f64(dx.cpu()), ref_dx, dtype, blocks_g) <= 1.0, what + ": dx"
+        assert np.max(np.abs(to_f64(da.cpu()) - ref_da)) <= 1e-4 * np.max(np.abs(ref_da)), what + ": da"
+        assert np.max(np.abs(to_f64(db.cpu()) - ref_db)) <= 1e-4 * np.max(np.abs(ref_db)), what + ": db"
+    B.wht_affine_set_variant(0)

@@ -459,6 +459,22 @@ def test_fwd_residual_many_rows(B):
     B.wht_affine_device_status()
 
 
+def test_fwd_residual_training_full_size(B):
+    # the fused residual forward in the launch configuration the benchmark times (65536 x 2048), sampled rows
+    # against y = resid + Eq. 1
+    B.wht_affine_set_variant(0)
+    w = wl.CONFIGS["training"]
+    a, b = wl.gen_params(w)
+    x = wl.gen_full(w, "x", threads=32)
+    r = wl.gen_full(w, "dy", threads=32)  # the second seeded tensor serves as the residual stream
+    y = B.forward(x.cuda(), a.cuda(), b.cuda(), resid=r.cuda())
+    torch.cuda.synchronize()
+    ridx = torch.from_numpy(_sample_rows(w.T, 1024, w.seed + 9))
+    ref = oracle.wht_affine_fwd_residual(to_f64(x[ridx]), to_f64(a), to_f64(b), to_f64(r[ridx]))
+    assert_rows_bf16(to_f64(y[ridx.cuda()].cpu()), ref, "residual forward, training size")
+    B.wht_affine_device_status()
+
+
 def test_host_pipeline_matches_direct_calls(B):
     # end-to-end helpers: pinned host -> device -> C ABI -> pinned host, rows moving in chunks on two
     # copy streams; same results as the plain device-resident calls
