@@ -66,21 +66,13 @@ dadb_finalize_kernel(const float* __restrict__ partials, int nparts, int d, floa
     if (which == 0) da[col] = s * inv_sqrt_d; else db[col] = s;
 }
 
-// ---- bandwidth yardstick: a plain streaming copy (what the forward's traffic costs with no arithmetic) ----
-// Four 128-bit loads per thread are in flight before the first store: 64 KiB per SM with 8 CTAs of 256 threads.
+// ---- bandwidth yardstick: copy rows with the forward pass's access pattern ----
+// (four loads in flight per thread were tried: the same at the Training size, 5 % slower at the Prefill size)
 __global__ void __launch_bounds__(256)
 copy_rows_kernel(const uint4* src, uint4* dst, long long n16) {
     const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
-    long long i = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x;
-    for (; i + 3 * stride < n16; i += 4 * stride) {
-        const uint4 q0 = __ldcs(src + i), q1 = __ldcs(src + i + stride), q2 = __ldcs(src + i + 2 * stride),
-                    q3 = __ldcs(src + i + 3 * stride);
-        __stcs(dst + i, q0);
-        __stcs(dst + i + stride, q1);
-        __stcs(dst + i + 2 * stride, q2);
-        __stcs(dst + i + 3 * stride, q3);
-    }
-    for (; i < n16; i += stride) __stcs(dst + i, __ldcs(src + i));
+    for (long long i = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; i < n16; i += stride)
+        __stcs(dst + i, __ldcs(src + i));
 }
 
 }  // namespace wht

@@ -320,11 +320,15 @@ __device__ __forceinline__ void thread_stages(float (&v)[R]) {
 }
 
 // ---- forward ---------------------------------------------------------------------------
-template <int LOGD, int NCOL, int STAGES, typename TP, bool RES = false>
+// LEAN: a footprint small enough for TWO CTAs per SM (H_128 in tensor memory instead of shared memory, one
+// accumulator, 256 tensor-memory columns), so that the CTAs of the NEXT launch in the stream can take their
+// places and set themselves up while this launch still runs (programmatic dependent launch); for calls of a
+// few tiles per CTA, where launch and set-up are a visible share of the time.
+template <int LOGD, int NCOL, int STAGES, typename TP, bool RES = false, bool LEAN = false>
 struct UmmaFwdSmem {
     using Geo = UmmaGeo<LOGD, NCOL>;
-    static constexpr int ACC = 512 / NCOL > 4 ? 4 : 512 / NCOL;          // accumulator buffers in TMEM
-    static constexpr int TMEM_COLS = ACC * NCOL <= 256 ? 256 : 512;
+    static constexpr int ACC = LEAN ? 1 : (512 / NCOL > 4 ? 4 : 512 / NCOL);  // accumulator buffers in TMEM
+    static constexpr int TMEM_COLS = (ACC * NCOL + (LEAN ? 64 : 0)) <= 256 ? 256 : 512;
     // a and b live in registers while a row's share of them is small.  At d = 8192 the plain
     // forward splits the channels between its two warp groups instead (SPLIT); with a residual,
     // whose chunks need registers too, a and b are staged in shared memory as fp32 from d = 4096 on
@@ -332,7 +336,7 @@ struct UmmaFwdSmem {
     static constexpr bool SPLIT = Geo::R > 32 && !RES;
     static constexpr bool PARAMS_IN_SMEM = RES && Geo::R >= 32;
     static constexpr int OFF_H = 0;
-    static constexpr int OFF_RING = Geo::H_BYTES;
+    static constexpr int OFF_RING = LEAN ? 0 : Geo::H_BYTES;
     static constexpr int OFF_PARAMS = OFF_RING + STAGES * Geo::TILE_BYTES;
     static constexpr int PARAM_BYTES = PARAMS_IN_SMEM ? 2 * Geo::D * 4 : 0;
     static constexpr int OFF_BARS = OFF_PARAMS + PARAM_BYTES;
@@ -369,7 +373,7 @@ __device__ __forceinline__ void stage_params_umma(const TP* __restrict__ src, fl
 // and multiplied by H_128 into the SAME accumulator, with the instruction descriptor's negate-A bit
 // set for the blocks whose sign is -1: the signed sum happens in the tensor core's fp32 accumulation
 // of exact +-1 products, and the epilogue is the ordinary one.  inv_sqrt_d is then 1/sqrt(nsrc * D).
-template <int LOGD, int NCOL, int STAGES, typename TP, bool RES, bool MULTI = false>
+template <int LOGD, int NCOL, int STAGES, typename TP, bool RES, bool MULTI = false, bool LEAN = false>
 __global__ void __launch_bounds__(UmmaGeo<LOGD, NCOL>::THREADS, 1)
 umma_fwd_kernel(const __nv_bfloat16* x, const TP* __restrict__ a, const TP* __restrict__ b,
                 const __nv_bfloat16* resid, __nv_bfloat16* y, long long T, float inv_sqrt_d,
@@ -378,8 +382,9 @@ umma_fwd_kernel(const __nv_bfloat16* x, const TP* __restrict__ a, const TP* __re
     static_assert(!(RES && MULTI), "the column-sharded form has no fused residual");
     const int nsrc = MULTI ? nsrc_arg : 1;
     using Geo = UmmaGeo<LOGD, NCOL>;
-    using L = UmmaFwdSmem<LOGD, NCOL, STAGES, TP, RES>;
+    using L = UmmaFwdSmem<LOGD, NCOL, STAGES, TP, RES, LEAN>;
     constexpr int ACC = L::ACC;
+    static_assert(!LEAN || !L::PARAMS_IN_SMEM, "the lean form keeps a and b in registers");
     extern __shared__ __align__(1024) unsigned char umma_smem[];
     unsigned char* const smem_raw = umma_smem;
     unsigned char* ring = smem_raw + L::OFF_RING;
@@ -415,8 +420,10 @@ umma_fwd_kernel(const __nv_bfloat16* x, const TP* __restrict__ a, const TP* __re
             asm volatile("bar.arrive 2, %0;" ::"r"(Geo::THREADS) : "memory");
         }
     } else {
-        write_h128(smem_raw + L::OFF_H, tid - 32, Geo::THREADS - 32);
-        fence_async_smem();  // H_128 was written by ordinary stores and is read by the tensor core
+        if constexpr (!LEAN) {
+            write_h128(smem_raw + L::OFF_H, tid - 32, Geo::THREADS - 32);
+            fence_async_smem();  // H_128 was written by ordinary stores and is read by the tensor core
+        }
         if (warp == 1) {
             tmem_alloc(tmem_slot, L::TMEM_COLS);
             tmem_relinquish();
@@ -425,6 +432,14 @@ umma_fwd_kernel(const __nv_bfloat16* x, const TP* __restrict__ a, const TP* __re
         named_barrier(2, Geo::THREADS);
         tc_fence_after();
         tmem_base = *tmem_slot;
+        if constexpr (LEAN) {  // H_128 into the 64 columns after the accumulator, one row per lane
+            if (warp >= 2 && warp < 6)
+                write_h128_row_tmem(tmem_base + ACC * Geo::N + (static_cast<uint32_t>((warp & 3) * 32) << 16),
+                                    (warp & 3) * 32 + lane);
+            tc_fence_before();
+            named_barrier(3, Geo::THREADS - 32);  // everybody but the producer warp
+            tc_fence_after();
+        }
     }
     // everything above touched only this CTA's own shared and tensor memory
     grid_dependency_wait();
@@ -480,8 +495,13 @@ umma_fwd_kernel(const __nv_bfloat16* x, const TP* __restrict__ a, const TP* __re
                     const uint64_t bdesc = umma_smem_desc(smem_u32(ring + s * Geo::TILE_BYTES));
                     const uint32_t idesc_s = MULTI ? (idesc | (((neg_mask >> src) & 1u) << kUmmaNegateABit)) : idesc;
 #pragma unroll
-                    for (int k = 0; k < 8; ++k)  // K = 16 per instruction: 256 bytes further in both operands
-                        umma_bf16(tmem_base + t * Geo::N, adesc + k * 16, bdesc + k * 16, idesc_s, (src | k) != 0);
+                    for (int k = 0; k < 8; ++k) {  // K = 16 per instruction: 256 bytes further in both operands
+                        if constexpr (LEAN)
+                            umma_bf16_a_tmem(tmem_base + t * Geo::N, tmem_base + ACC * Geo::N + k * 8, bdesc + k * 16,
+                                             idesc_s, (src | k) != 0);
+                        else
+                            umma_bf16(tmem_base + t * Geo::N, adesc + k * 16, bdesc + k * 16, idesc_s, (src | k) != 0);
+                    }
                     if (src == nsrc - 1) umma_commit(acc_full + t);
                     umma_commit(empty + s);
                 }
