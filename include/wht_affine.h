@@ -243,10 +243,12 @@ size_t wht_affine_bwd_workspace_bytes(int64_t T, int32_t d, int dtype);
  *       enough work for their 32 KiB tiles (forward: T*d >= 4 Mi elements, 8 Mi at d = 8192;
  *       backward: T*d >= 256 Ki); else the mma.sync kernels for 256 <= d <= 8192 (rows loaded
  *       directly when they are few or narrow, streamed through a shared-memory ring otherwise);
- *       butterfly otherwise and for fp32 rows;
+ *       butterfly otherwise.  fp32 rows: the streamed mma.sync kernels once T >= 32 rows per SM
+ *       (forward: 1024 <= d <= 8192, backward: 256 <= d <= 4096), each
+ *       fp32 operand of a pass carried as three bf16 terms, i.e. exactly; butterfly otherwise;
  *   1 = butterfly (registers + warp shuffles + shared memory), every d and dtype;
- *   2 = mma.sync tensor-core assisted with direct row loads;
- *   3 = mma.sync tensor-core assisted with streamed rows;
+ *   2 = mma.sync tensor-core assisted with direct row loads (256 <= d <= 8192, every dtype);
+ *   3 = mma.sync tensor-core assisted with streamed rows (the same range);
  *   4 = tcgen05: rows copied into shared memory as they are and multiplied by H_128 on the
  *       tensor core (accumulators in tensor memory), the rest in registers;
  *   5 = as 4, the backward with half-size products (H_64, two accumulators side by side in the

@@ -82,6 +82,35 @@ __device__ __forceinline__ void split_hi_lo(F2 v, uint32_t& hi, uint32_t& lo) {
     lo = pack_bf16x2(sub2(v, unpack_bf16x2(hi)));
 }
 
+// fp32 pair -> three bf16x2 terms hi + mid + lo: 24 significant bits, i.e. the fp32 value itself (up to
+// the exponent range of bf16, which is fp32's).
+__device__ __forceinline__ void split_hi_mid_lo(F2 v, uint32_t& hi, uint32_t& mid, uint32_t& lo) {
+    hi = pack_bf16x2(v);
+    const F2 r = sub2(v, unpack_bf16x2(hi));
+    mid = pack_bf16x2(r);
+    lo = pack_bf16x2(sub2(r, unpack_bf16x2(mid)));
+}
+
+// d += H_16 * [b0; b1] with the fp32 operands carried as NS bf16 terms each (NS mma into one accumulator):
+// NS = 2 carries 16-17 significant bits, NS = 3 all 24.
+template <int NS>
+__device__ __forceinline__ void mma_split(F2& d01, F2& d23, const uint32_t (&hf)[4], F2 b0, F2 b1) {
+    if constexpr (NS == 2) {
+        uint32_t b0h, b0l, b1h, b1l;
+        split_hi_lo(b0, b0h, b0l);
+        split_hi_lo(b1, b1h, b1l);
+        mma_bf16_m16n8k16(d01, d23, hf, b0h, b1h);
+        mma_bf16_m16n8k16(d01, d23, hf, b0l, b1l);
+    } else {
+        uint32_t b0h, b0m, b0l, b1h, b1m, b1l;
+        split_hi_mid_lo(b0, b0h, b0m, b0l);
+        split_hi_mid_lo(b1, b1h, b1m, b1l);
+        mma_bf16_m16n8k16(d01, d23, hf, b0h, b1h);
+        mma_bf16_m16n8k16(d01, d23, hf, b0m, b1m);
+        mma_bf16_m16n8k16(d01, d23, hf, b0l, b1l);
+    }
+}
+
 __device__ __forceinline__ void named_barrier(int id, int threads) {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
@@ -120,7 +149,8 @@ __device__ __forceinline__ int chunk_of(int w, int idx) {
 // Thread-local views of a row slice:
 //   m[t][h][p]  (after pass 1)  pair r = (x, y) <-> index bit 5, p <-> bit 1, h <-> bit 2
 //   v[t][j]     (load layout)   pair (x, y) = elements 2j, 2j+1 of chunk slot t
-template <class Geo>
+//   NS: bf16 terms an fp32 operand of a pass is carried as (2 for bf16 rows, 3 for fp32 rows)
+template <class Geo, int NS = 2>
 struct MmaXform {
     static constexpr int NT = Geo::NT;
 
@@ -142,12 +172,8 @@ struct MmaXform {
         for (int t = 0; t < NT; ++t) {
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
-                uint32_t b0h, b0l, b1h, b1l;
-                split_hi_lo(v[t][2 * h + 0], b0h, b0l);
-                split_hi_lo(v[t][2 * h + 1], b1h, b1l);
                 m[t][h][0] = m[t][h][1] = f2(0.0f, 0.0f);
-                mma_bf16_m16n8k16(m[t][h][0], m[t][h][1], hf, b0h, b1h);
-                mma_bf16_m16n8k16(m[t][h][0], m[t][h][1], hf, b0l, b1l);
+                mma_split<NS>(m[t][h][0], m[t][h][1], hf, v[t][2 * h + 0], v[t][2 * h + 1]);
             }
         }
     }
@@ -184,12 +210,8 @@ struct MmaXform {
         if constexpr (NT == 1) {
 #pragma unroll
             for (int p = 0; p < 2; ++p) {
-                uint32_t b0h, b0l, b1h, b1l;
-                split_hi_lo(m[0][0][p], b0h, b0l);
-                split_hi_lo(m[0][1][p], b1h, b1l);
                 F2 d01 = f2(0.0f, 0.0f), d23 = f2(0.0f, 0.0f);
-                mma_bf16_m16n8k16(d01, d23, hf, b0h, b1h);
-                mma_bf16_m16n8k16(d01, d23, hf, b0l, b1l);
+                mma_split<NS>(d01, d23, hf, m[0][0][p], m[0][1][p]);
                 v[0][p] = d01;
                 v[0][2 + p] = d23;
             }
@@ -201,12 +223,8 @@ struct MmaXform {
             for (int h = 0; h < 2; ++h) {
 #pragma unroll
                 for (int p = 0; p < 2; ++p) {
-                    uint32_t b0h, b0l, b1h, b1l;
-                    split_hi_lo(m[2 * u][h][p], b0h, b0l);
-                    split_hi_lo(m[2 * u + 1][h][p], b1h, b1l);
                     F2 d01 = f2(0.0f, 0.0f), d23 = f2(0.0f, 0.0f);
-                    mma_bf16_m16n8k16(d01, d23, hf, b0h, b1h);
-                    mma_bf16_m16n8k16(d01, d23, hf, b0l, b1l);
+                    mma_split<NS>(d01, d23, hf, m[2 * u][h][p], m[2 * u + 1][h][p]);
                     v[2 * u][2 * h + p] = d01;
                     v[2 * u + 1][2 * h + p] = d23;
                 }
@@ -274,52 +292,102 @@ __device__ __forceinline__ void load_params8(const __nv_bfloat16* __restrict__ p
     v[2] = unpack_bf16x2(q.z); v[3] = unpack_bf16x2(q.w);
 }
 
+// Eight contiguous row elements of one thread ("chunk"), as stored: how the direct-load kernels read and
+// write rows of either storage type.  `pairs` are the fp32 values as four packed pairs (elements 2j, 2j+1).
+template <typename TIO> struct MmaRowIO;
+template <> struct MmaRowIO<__nv_bfloat16> {
+    using Raw = uint4;
+    static constexpr bool kStoredBf16 = true;
+    static __device__ __forceinline__ Raw load(const __nv_bfloat16* row, int chunk) {
+        return __ldcs(reinterpret_cast<const uint4*>(row) + chunk);
+    }
+    static __device__ __forceinline__ Raw staged(const unsigned char* row, int chunk) {  // row in shared memory
+        return reinterpret_cast<const uint4*>(row)[chunk];
+    }
+    static __device__ __forceinline__ void pairs(const Raw& r, F2 (&v)[4]) {
+        v[0] = unpack_bf16x2(r.x); v[1] = unpack_bf16x2(r.y); v[2] = unpack_bf16x2(r.z); v[3] = unpack_bf16x2(r.w);
+    }
+    static __device__ __forceinline__ void store(__nv_bfloat16* row, int chunk, const F2 (&v)[4]) {
+        uint4 o;
+        o.x = pack_bf16x2(v[0]); o.y = pack_bf16x2(v[1]); o.z = pack_bf16x2(v[2]); o.w = pack_bf16x2(v[3]);
+        __stcs(reinterpret_cast<uint4*>(row) + chunk, o);
+    }
+};
+template <> struct MmaRowIO<float> {
+    struct Raw { float4 a, b; };
+    static constexpr bool kStoredBf16 = false;
+    static __device__ __forceinline__ Raw load(const float* row, int chunk) {
+        Raw r;
+        r.a = __ldcs(reinterpret_cast<const float4*>(row) + 2 * chunk);
+        r.b = __ldcs(reinterpret_cast<const float4*>(row) + 2 * chunk + 1);
+        return r;
+    }
+    static __device__ __forceinline__ Raw staged(const unsigned char* row, int chunk) {
+        // lanes 32 bytes apart: lanes l and l + 4 of a quarter-warp would meet in the same banks, so every
+        // other group of four lanes fetches its two halves in the opposite order
+        const int sw = (chunk >> 2) & 1;
+        const float4 p = reinterpret_cast<const float4*>(row)[2 * chunk + sw];
+        const float4 q = reinterpret_cast<const float4*>(row)[2 * chunk + (sw ^ 1)];
+        Raw r;
+        r.a = sw ? q : p;
+        r.b = sw ? p : q;
+        return r;
+    }
+    static __device__ __forceinline__ void pairs(const Raw& r, F2 (&v)[4]) {
+        v[0] = f2(r.a.x, r.a.y); v[1] = f2(r.a.z, r.a.w); v[2] = f2(r.b.x, r.b.y); v[3] = f2(r.b.z, r.b.w);
+    }
+    static __device__ __forceinline__ void store(float* row, int chunk, const F2 (&v)[4]) {
+        __stcs(reinterpret_cast<float4*>(row) + 2 * chunk, make_float4(v[0].x, v[0].y, v[1].x, v[1].y));
+        __stcs(reinterpret_cast<float4*>(row) + 2 * chunk + 1, make_float4(v[2].x, v[2].y, v[3].x, v[3].y));
+    }
+};
+
 // In every helper below `as` is a / sqrt(d): the normalisation rides on the scale
 // vector, so the forward epilogue is one fma and the backward needs no final scale
 // (H is linear: ((a/sqrt(d)) (.) dy) H = ((a (.) dy) H)/sqrt(d)).
 
-// y chunk = as (.) v + b, rounded to bf16 and stored (128-bit, streaming)
+// y chunk = as (.) v + b, rounded to the stored type once and stored (128-bit, streaming)
+template <typename TIO>
 __device__ __forceinline__ void fwd_store_chunk(const F2 (&v)[4], const F2 (&as)[4], const F2 (&bs)[4],
-                                                uint4* dst) {
-    uint4 o;
-    o.x = pack_bf16x2(fma2(v[0], as[0], bs[0]));
-    o.y = pack_bf16x2(fma2(v[1], as[1], bs[1]));
-    o.z = pack_bf16x2(fma2(v[2], as[2], bs[2]));
-    o.w = pack_bf16x2(fma2(v[3], as[3], bs[3]));
-    __stcs(dst, o);
+                                                TIO* row, int chunk) {
+    F2 o[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) o[j] = fma2(v[j], as[j], bs[j]);
+    MmaRowIO<TIO>::store(row, chunk, o);
 }
 // y chunk = r + (as (.) v + b) with r the 8 stored residual values `res`: the sum is taken in
-// fp32 and rounded to bf16 once
+// fp32 and rounded to the stored type once
+template <typename TIO>
+__device__ __forceinline__ void fwd_store_chunk_res(const F2 (&v)[4], const F2 (&as)[4], const F2 (&bs)[4],
+                                                    const typename MmaRowIO<TIO>::Raw& res, TIO* row, int chunk) {
+    F2 o[4], r[4];
+    MmaRowIO<TIO>::pairs(res, r);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) o[j] = add2(fma2(v[j], as[j], bs[j]), r[j]);
+    MmaRowIO<TIO>::store(row, chunk, o);
+}
+
+// the same for a bf16 chunk given by its address
+__device__ __forceinline__ void fwd_store_chunk(const F2 (&v)[4], const F2 (&as)[4], const F2 (&bs)[4], uint4* dst) {
+    fwd_store_chunk<__nv_bfloat16>(v, as, bs, reinterpret_cast<__nv_bfloat16*>(dst), 0);
+}
 __device__ __forceinline__ void fwd_store_chunk_res(const F2 (&v)[4], const F2 (&as)[4], const F2 (&bs)[4],
                                                     const uint4& res, uint4* dst) {
-    uint4 o;
-    o.x = pack_bf16x2(add2(fma2(v[0], as[0], bs[0]), unpack_bf16x2(res.x)));
-    o.y = pack_bf16x2(add2(fma2(v[1], as[1], bs[1]), unpack_bf16x2(res.y)));
-    o.z = pack_bf16x2(add2(fma2(v[2], as[2], bs[2]), unpack_bf16x2(res.z)));
-    o.w = pack_bf16x2(add2(fma2(v[3], as[3], bs[3]), unpack_bf16x2(res.w)));
-    __stcs(dst, o);
+    fwd_store_chunk_res<__nv_bfloat16>(v, as, bs, res, reinterpret_cast<__nv_bfloat16*>(dst), 0);
 }
 
 // backward, between the two transforms, one chunk: da += dy (.) u, db += dy, v <- as (.) dy
-__device__ __forceinline__ void bwd_mid_chunk(F2 (&v)[4], const uint4& rawdy, const F2 (&as)[4],
-                                              F2 (&da_acc)[4], F2 (&db_acc)[4]) {
-    const uint32_t w[4] = {rawdy.x, rawdy.y, rawdy.z, rawdy.w};
+template <typename TIO>
+__device__ __forceinline__ void bwd_mid_chunk(F2 (&v)[4], const typename MmaRowIO<TIO>::Raw& rawdy,
+                                              const F2 (&as)[4], F2 (&da_acc)[4], F2 (&db_acc)[4]) {
+    F2 dyv[4];
+    MmaRowIO<TIO>::pairs(rawdy, dyv);
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
-        const F2 dyv = unpack_bf16x2(w[j]);
-        da_acc[j] = fma2(dyv, v[j], da_acc[j]);
-        db_acc[j] = add2(db_acc[j], dyv);
-        v[j] = mul2(as[j], dyv);
+        da_acc[j] = fma2(dyv[j], v[j], da_acc[j]);
+        db_acc[j] = add2(db_acc[j], dyv[j]);
+        v[j] = mul2(as[j], dyv[j]);
     }
-}
-
-__device__ __forceinline__ void bwd_store_chunk(const F2 (&v)[4], uint4* dst) {
-    uint4 o;
-    o.x = pack_bf16x2(v[0]);
-    o.y = pack_bf16x2(v[1]);
-    o.z = pack_bf16x2(v[2]);
-    o.w = pack_bf16x2(v[3]);
-    __stcs(dst, o);
 }
 
 // Fold the RG row groups' partial sums of one CTA in a fixed order and publish them.
@@ -353,14 +421,18 @@ __device__ __forceinline__ void bwd_publish_partials(const F2 (&da_acc)[Geo::NT]
 }
 
 // ---- forward, rows loaded straight from global memory (few rows / decode) ----------
-template <int LOGD, int TB, int RG, typename TP>
+//   TIO: storage type of the rows.  bf16 rows enter the first pass as they are (exact) and later passes as
+//   two bf16 terms; fp32 rows enter every pass as three, so that no pass rounds below fp32.
+template <int LOGD, int TB, int RG, typename TP, typename TIO = __nv_bfloat16>
 __global__ void __launch_bounds__(MmaGeo<LOGD, TB, RG>::THREADS)
-mma_fwd_kernel(const __nv_bfloat16* x, const TP* __restrict__ a, const TP* __restrict__ b,
-               const __nv_bfloat16* resid, __nv_bfloat16* y, long long T, long long ld, float inv_sqrt_d) {
+mma_fwd_kernel(const TIO* x, const TP* __restrict__ a, const TP* __restrict__ b,
+               const TIO* resid, TIO* y, long long T, long long ld, float inv_sqrt_d) {
     // ld: elements between consecutive rows (>= D).  Block-diagonal form: blockIdx.y picks the channel
     // group [y*D, (y+1)*D) of rows ld wide.
     using Geo = MmaGeo<LOGD, TB, RG>;
-    using X = MmaXform<Geo>;
+    using IO = MmaRowIO<TIO>;
+    using Raw = typename IO::Raw;
+    using X = MmaXform<Geo, IO::kStoredBf16 ? 2 : 3>;
     constexpr int NT = Geo::NT;
     extern __shared__ __align__(16) float smem[];
     const int lane = threadIdx.x & 31;
@@ -399,13 +471,12 @@ mma_fwd_kernel(const __nv_bfloat16* x, const TP* __restrict__ a, const TP* __res
     // Narrow rows (one or two 128-bit loads per lane and row) put little data in flight per warp, and the
     // registers allow only ~40 warps per SM: a warp requests U of its rows before it transforms the first.
     constexpr int U = (Geo::WB == 0 && NT <= 2) ? 4 / NT : 1;
-    auto load_row = [&](long long r, uint4 (&dst)[NT]) {
-        const uint4* src = reinterpret_cast<const uint4*>(x + r * ld);
+    auto load_row = [&](long long r, Raw (&dst)[NT]) {
 #pragma unroll
-        for (int t = 0; t < NT; ++t) dst[t] = __ldcs(src + chunk_of<Geo, false>(w, t) * 32 + lane);
+        for (int t = 0; t < NT; ++t) dst[t] = IO::load(x + r * ld, chunk_of<Geo, false>(w, t) * 32 + lane);
     };
     for (long long row0 = static_cast<long long>(blockIdx.x) * RG + rg; row0 < T; row0 += U * stride) {
-        uint4 raws[U][NT];
+        Raw raws[U][NT];
 #pragma unroll
         for (int u = 0; u < U; ++u)
             if (row0 + u * stride < T) load_row(row0 + u * stride, raws[u]);  // uniform over the warp
@@ -413,21 +484,26 @@ mma_fwd_kernel(const __nv_bfloat16* x, const TP* __restrict__ a, const TP* __res
         for (int u = 0; u < U; ++u) {
             const long long row = row0 + u * stride;
             if (row >= T) break;
-            uint4 res[NT];
+            Raw res[NT];
             if (resid != nullptr) {  // the residual chunks too, ahead of the transform
 #pragma unroll
                 for (int idx = 0; idx < NT; ++idx)
-                    res[idx] = __ldcs(reinterpret_cast<const uint4*>(resid + row * ld) +
-                                      chunk_of<Geo, true>(w, idx) * 32 + lane);
+                    res[idx] = IO::load(resid + row * ld, chunk_of<Geo, true>(w, idx) * 32 + lane);
             }
             F2 m[NT][2][2];
             F2 v[NT][4];
-            X::pass1_raw(raws[u], m, hf);
+            if constexpr (IO::kStoredBf16) {
+                X::pass1_raw(raws[u], m, hf);
+            } else {
+#pragma unroll
+                for (int t = 0; t < NT; ++t) IO::pairs(raws[u][t], v[t]);
+                X::pass1_f32(v, m, hf);
+            }
             X::mid_stages(m);
             X::pass2(m, v, hf);
             X::exchange_and_top(v, xbuf + parity * Geo::XCHG_ONE, w, lane, 1 + rg);
             parity ^= 1;
-            uint4* dst = reinterpret_cast<uint4*>(y + row * ld);
+            TIO* dst = y + row * ld;
 #pragma unroll
             for (int idx = 0; idx < NT; ++idx) {
                 const int c = chunk_of<Geo, true>(w, idx);
@@ -442,9 +518,9 @@ mma_fwd_kernel(const __nv_bfloat16* x, const TP* __restrict__ a, const TP* __res
                     for (int j = 0; j < 4; ++j) as[j] = mul2(as[j], rs2);
                 }
                 if (resid != nullptr) {
-                    fwd_store_chunk_res(v[idx], as, bs, res[idx], dst + c * 32 + lane);
+                    fwd_store_chunk_res<TIO>(v[idx], as, bs, res[idx], dst, c * 32 + lane);
                 } else {
-                    fwd_store_chunk(v[idx], as, bs, dst + c * 32 + lane);
+                    fwd_store_chunk<TIO>(v[idx], as, bs, dst, c * 32 + lane);
                 }
             }
         }
@@ -452,12 +528,14 @@ mma_fwd_kernel(const __nv_bfloat16* x, const TP* __restrict__ a, const TP* __res
 }
 
 // ---- backward, rows loaded straight from global memory ------------------------------
-template <int LOGD, int TB, int RG, typename TP>
+template <int LOGD, int TB, int RG, typename TP, typename TIO = __nv_bfloat16>
 __global__ void __launch_bounds__(MmaGeo<LOGD, TB, RG>::THREADS)
-mma_bwd_kernel(const __nv_bfloat16* dy, const __nv_bfloat16* x, const TP* __restrict__ a,
-               __nv_bfloat16* dx, float* __restrict__ partials, long long T, long long ld, float inv_sqrt_d) {
+mma_bwd_kernel(const TIO* dy, const TIO* x, const TP* __restrict__ a,
+               TIO* dx, float* __restrict__ partials, long long T, long long ld, float inv_sqrt_d) {
     using Geo = MmaGeo<LOGD, TB, RG>;
-    using X = MmaXform<Geo>;
+    using IO = MmaRowIO<TIO>;
+    using Raw = typename IO::Raw;
+    using X = MmaXform<Geo, IO::kStoredBf16 ? 2 : 3>;
     constexpr int NT = Geo::NT;
     extern __shared__ __align__(16) float smem[];
     const int lane = threadIdx.x & 31;
@@ -485,16 +563,14 @@ mma_bwd_kernel(const __nv_bfloat16* dy, const __nv_bfloat16* x, const TP* __rest
     // and the column sums in registers this costs occupancy and loses at every narrow width (d = 256: 0.885 ->
     // 0.73 of the copy rate, d = 512: 0.84 -> 0.61), unlike in the forward; so U = 1, the hook stays.
     constexpr int U = 1;
-    auto load_rows = [&](long long r, uint4 (&dx_)[NT], uint4 (&ddy)[NT]) {
-        const uint4* xsrc = reinterpret_cast<const uint4*>(x + r * ld);
-        const uint4* dysrc = reinterpret_cast<const uint4*>(dy + r * ld);
+    auto load_rows = [&](long long r, Raw (&dx_)[NT], Raw (&ddy)[NT]) {
 #pragma unroll
-        for (int t = 0; t < NT; ++t) dx_[t] = __ldcs(xsrc + chunk_of<Geo, false>(w, t) * 32 + lane);
+        for (int t = 0; t < NT; ++t) dx_[t] = IO::load(x + r * ld, chunk_of<Geo, false>(w, t) * 32 + lane);
 #pragma unroll
-        for (int t = 0; t < NT; ++t) ddy[t] = __ldcs(dysrc + chunk_of<Geo, true>(w, t) * 32 + lane);
+        for (int t = 0; t < NT; ++t) ddy[t] = IO::load(dy + r * ld, chunk_of<Geo, true>(w, t) * 32 + lane);
     };
     for (long long row0 = static_cast<long long>(blockIdx.x) * RG + rg; row0 < T; row0 += U * stride) {
-        uint4 raws[U][NT], rawdys[U][NT];
+        Raw raws[U][NT], rawdys[U][NT];
 #pragma unroll
         for (int u = 0; u < U; ++u)
             if (row0 + u * stride < T) load_rows(row0 + u * stride, raws[u], rawdys[u]);  // uniform over the warp
@@ -505,7 +581,13 @@ mma_bwd_kernel(const __nv_bfloat16* dy, const __nv_bfloat16* x, const TP* __rest
             F2 m[NT][2][2];
             F2 v[NT][4];
             // u = x H, delivered in layout B
-            X::pass1_raw(raws[u], m, hf);
+            if constexpr (IO::kStoredBf16) {
+                X::pass1_raw(raws[u], m, hf);
+            } else {
+#pragma unroll
+                for (int t = 0; t < NT; ++t) IO::pairs(raws[u][t], v[t]);
+                X::pass1_f32(v, m, hf);
+            }
             X::mid_stages(m);
             X::pass2(m, v, hf);
             X::exchange_and_top(v, xbuf, w, lane, 1 + rg);
@@ -517,17 +599,16 @@ mma_bwd_kernel(const __nv_bfloat16* dy, const __nv_bfloat16* x, const TP* __rest
                 load_params8(a + (c * 32 + lane) * 8, as);
 #pragma unroll
                 for (int j = 0; j < 4; ++j) as[j] = mul2(as[j], rs2);
-                bwd_mid_chunk(v[idx], rawdys[u][idx], as, da_acc[idx], db_acc[idx]);
+                bwd_mid_chunk<TIO>(v[idx], rawdys[u][idx], as, da_acc[idx], db_acc[idx]);
             }
             // dx = (g H)/sqrt(d): layout B in, layout A out
             X::pass1_f32(v, m, hf);
             X::mid_stages(m);
             X::pass2(m, v, hf);
             X::exchange_and_top(v, xbuf + Geo::XCHG_ONE, w, lane, 1 + rg);
-            uint4* dst = reinterpret_cast<uint4*>(dx + row * ld);
 #pragma unroll
             for (int idx = 0; idx < NT; ++idx)
-                bwd_store_chunk(v[idx], dst + chunk_of<Geo, false>(w, idx) * 32 + lane);
+                IO::store(dx + row * ld, chunk_of<Geo, false>(w, idx) * 32 + lane, v[idx]);
         }
     }
     bwd_publish_partials<Geo>(da_acc, db_acc, smem, partials, rg, w, lane);

@@ -76,11 +76,11 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity
     return false;
 }
 
-template <int LOGD, int TB, int RG, int S_, bool BWD>
+template <int LOGD, int TB, int RG, int S_, bool BWD, int ELEM_BYTES = 2>
 struct PipeGeo : MmaGeo<LOGD, TB, RG> {
     using Base = MmaGeo<LOGD, TB, RG>;
     static constexpr int S = S_;                              // ring depth (rows in flight per row group)
-    static constexpr int ROW_BYTES = Base::D * 2;
+    static constexpr int ROW_BYTES = Base::D * ELEM_BYTES;
     static constexpr int STAGE_BYTES = ROW_BYTES * (BWD ? 2 : 1);  // bwd: x row then dy row
     static constexpr int RING_BYTES = RG * S * STAGE_BYTES;
     static constexpr int XCHG_BYTES = RG * Base::XCHG_FLOATS * 4;
@@ -122,12 +122,14 @@ __device__ __forceinline__ void read_staged8(const float* base, int c, int lane,
 }
 
 // ---- forward, streamed ----------------------------------------------------------
-template <int LOGD, int TB, int RG, int S, int MINB, typename TP>
+template <int LOGD, int TB, int RG, int S, int MINB, typename TP, typename TIO = __nv_bfloat16>
 __global__ void __launch_bounds__(MmaGeo<LOGD, TB, RG>::THREADS, MINB)
-mma_fwd_pipe_kernel(const __nv_bfloat16* x, const TP* __restrict__ a, const TP* __restrict__ b,
-                    const __nv_bfloat16* resid, __nv_bfloat16* y, long long T, long long ld, float inv_sqrt_d) {
-    using Geo = PipeGeo<LOGD, TB, RG, S, false>;
-    using X = MmaXform<Geo>;
+mma_fwd_pipe_kernel(const TIO* x, const TP* __restrict__ a, const TP* __restrict__ b,
+                    const TIO* resid, TIO* y, long long T, long long ld, float inv_sqrt_d) {
+    using Geo = PipeGeo<LOGD, TB, RG, S, false, sizeof(TIO)>;
+    using IO = MmaRowIO<TIO>;
+    using Raw = typename IO::Raw;
+    using X = MmaXform<Geo, IO::kStoredBf16 ? 2 : 3>;
     constexpr int NT = Geo::NT;
     extern __shared__ __align__(128) unsigned char smem_raw[];
     const int lane = threadIdx.x & 31;
@@ -178,13 +180,20 @@ mma_fwd_pipe_kernel(const __nv_bfloat16* x, const TP* __restrict__ a, const TP* 
     int parity = 0;
     for (long long row = first; row < T; row += stride) {
         mbar_wait_bounded(full + stage, phase);
-        const uint4* st = reinterpret_cast<const uint4*>(ring + stage * Geo::STAGE_BYTES);
-        uint4 raw[NT];
+        const unsigned char* st = ring + stage * Geo::STAGE_BYTES;
+        Raw raw[NT];
 #pragma unroll
-        for (int t = 0; t < NT; ++t) raw[t] = st[chunk_of<Geo, false>(w, t) * 32 + lane];
+        for (int t = 0; t < NT; ++t) raw[t] = IO::staged(st, chunk_of<Geo, false>(w, t) * 32 + lane);
         F2 m[NT][2][2];
         F2 v[NT][4];
-        X::pass1_raw(raw, m, hf);  // warp-synchronous: every lane's reads of the stage are done here
+        // pass 1 is warp-synchronous: every lane's reads of the stage are done after it
+        if constexpr (IO::kStoredBf16) {
+            X::pass1_raw(raw, m, hf);
+        } else {
+#pragma unroll
+            for (int t = 0; t < NT; ++t) IO::pairs(raw[t], v[t]);
+            X::pass1_f32(v, m, hf);
+        }
         const long long next_row = row + S * stride;
         if constexpr (Geo::WB == 0) {
             __syncwarp();
@@ -199,7 +208,7 @@ mma_fwd_pipe_kernel(const __nv_bfloat16* x, const TP* __restrict__ a, const TP* 
             // its pass 1: the stage is free
             if (elected && next_row < T) issue(stage, next_row);
         }
-        uint4* dst = reinterpret_cast<uint4*>(y + row * ld);
+        TIO* dst = y + row * ld;
 #pragma unroll
         for (int idx = 0; idx < NT; ++idx) {
             const int c = chunk_of<Geo, true>(w, idx);
@@ -207,10 +216,10 @@ mma_fwd_pipe_kernel(const __nv_bfloat16* x, const TP* __restrict__ a, const TP* 
             read_staged8(pa, c, lane, as);
             read_staged8(pb, c, lane, bs);
             if (resid != nullptr) {
-                const uint4 r = __ldcs(reinterpret_cast<const uint4*>(resid + row * ld) + c * 32 + lane);
-                fwd_store_chunk_res(v[idx], as, bs, r, dst + c * 32 + lane);
+                const Raw r = IO::load(resid + row * ld, c * 32 + lane);
+                fwd_store_chunk_res<TIO>(v[idx], as, bs, r, dst, c * 32 + lane);
             } else {
-                fwd_store_chunk(v[idx], as, bs, dst + c * 32 + lane);
+                fwd_store_chunk<TIO>(v[idx], as, bs, dst, c * 32 + lane);
             }
         }
         if (++stage == S) { stage = 0; phase ^= 1; }
@@ -218,12 +227,14 @@ mma_fwd_pipe_kernel(const __nv_bfloat16* x, const TP* __restrict__ a, const TP* 
 }
 
 // ---- backward, streamed -----------------------------------------------------------
-template <int LOGD, int TB, int RG, int S, int MINB, typename TP>
+template <int LOGD, int TB, int RG, int S, int MINB, typename TP, typename TIO = __nv_bfloat16>
 __global__ void __launch_bounds__(MmaGeo<LOGD, TB, RG>::THREADS, MINB)
-mma_bwd_pipe_kernel(const __nv_bfloat16* dy, const __nv_bfloat16* x, const TP* __restrict__ a,
-                    __nv_bfloat16* dx, float* __restrict__ partials, long long T, long long ld, float inv_sqrt_d) {
-    using Geo = PipeGeo<LOGD, TB, RG, S, true>;
-    using X = MmaXform<Geo>;
+mma_bwd_pipe_kernel(const TIO* dy, const TIO* x, const TP* __restrict__ a,
+                    TIO* dx, float* __restrict__ partials, long long T, long long ld, float inv_sqrt_d) {
+    using Geo = PipeGeo<LOGD, TB, RG, S, true, sizeof(TIO)>;
+    using IO = MmaRowIO<TIO>;
+    using Raw = typename IO::Raw;
+    using X = MmaXform<Geo, IO::kStoredBf16 ? 2 : 3>;
     constexpr int NT = Geo::NT;
     extern __shared__ __align__(128) unsigned char smem_raw[];
     const int lane = threadIdx.x & 31;
@@ -278,15 +289,21 @@ mma_bwd_pipe_kernel(const __nv_bfloat16* dy, const __nv_bfloat16* x, const TP* _
     uint32_t phase = 0;
     for (long long row = first; row < T; row += stride) {
         mbar_wait_bounded(full + stage, phase);
-        const uint4* stx = reinterpret_cast<const uint4*>(ring + stage * Geo::STAGE_BYTES);
-        const uint4* stdy = reinterpret_cast<const uint4*>(ring + stage * Geo::STAGE_BYTES + Geo::ROW_BYTES);
-        uint4 raw[NT];
-#pragma unroll
-        for (int t = 0; t < NT; ++t) raw[t] = stx[chunk_of<Geo, false>(w, t) * 32 + lane];
+        const unsigned char* stx = ring + stage * Geo::STAGE_BYTES;
+        const unsigned char* stdy = stx + Geo::ROW_BYTES;
         F2 m[NT][2][2];
         F2 v[NT][4];
         // u = x H, delivered in layout B
-        X::pass1_raw(raw, m, hf);
+        if constexpr (IO::kStoredBf16) {
+            Raw raw[NT];
+#pragma unroll
+            for (int t = 0; t < NT; ++t) raw[t] = IO::staged(stx, chunk_of<Geo, false>(w, t) * 32 + lane);
+            X::pass1_raw(raw, m, hf);
+        } else {
+#pragma unroll
+            for (int t = 0; t < NT; ++t) IO::pairs(IO::staged(stx, chunk_of<Geo, false>(w, t) * 32 + lane), v[t]);
+            X::pass1_f32(v, m, hf);
+        }
         X::mid_stages(m);
         X::pass2(m, v, hf);
         X::exchange_and_top(v, xbuf, w, lane, 1 + rg);
@@ -296,7 +313,7 @@ mma_bwd_pipe_kernel(const __nv_bfloat16* dy, const __nv_bfloat16* x, const TP* _
             const int c = chunk_of<Geo, true>(w, idx);
             F2 as[4];
             read_staged8(pa, c, lane, as);
-            bwd_mid_chunk(v[idx], stdy[c * 32 + lane], as, da_acc[idx], db_acc[idx]);
+            bwd_mid_chunk<TIO>(v[idx], IO::staged(stdy, c * 32 + lane), as, da_acc[idx], db_acc[idx]);
         }
         // dx = (g H)/sqrt(d): layout B in, layout A out
         X::pass1_f32(v, m, hf);  // warp-synchronous: this warp's reads of the stage are done here
@@ -311,10 +328,9 @@ mma_bwd_pipe_kernel(const __nv_bfloat16* dy, const __nv_bfloat16* x, const TP* _
         if constexpr (Geo::WB > 0) {
             if (elected && next_row < T) issue(stage, next_row);
         }
-        uint4* dst = reinterpret_cast<uint4*>(dx + row * ld);
+        TIO* dst = dx + row * ld;
 #pragma unroll
-        for (int idx = 0; idx < NT; ++idx)
-            bwd_store_chunk(v[idx], dst + chunk_of<Geo, false>(w, idx) * 32 + lane);
+        for (int idx = 0; idx < NT; ++idx) IO::store(dst, chunk_of<Geo, false>(w, idx) * 32 + lane, v[idx]);
         if (++stage == S) { stage = 0; phase ^= 1; }
     }
     bwd_publish_partials<Geo>(da_acc, db_acc, reinterpret_cast<float*>(smem_raw), partials, rg, w, lane);

@@ -119,8 +119,8 @@ int check_common(int64_t T, int32_t d, int dtype) {
 bool umma_fwd_supported(int logd, int dtype) { return dtype != WHT_F32 && logd >= 10 && logd <= 13; }
 bool umma_bwd_supported(int logd, int dtype) { return dtype != WHT_F32 && logd >= 10 && logd <= 13; }
 
-// bf16 rows of 256 ... 8192 elements (d = 256: two chained H_16 passes on one chunk per thread)
-bool mma_supported(int logd, int dtype) { return dtype != WHT_F32 && logd >= 8 && logd <= 13; }
+// Rows of 256 ... 8192 elements (d = 256: two chained H_16 passes on one chunk per thread), bf16 or fp32
+bool mma_supported(int logd, int /*dtype*/) { return logd >= 8 && logd <= 13; }
 
 // The persistent tcgen05 kernels win once there are a few hundred 32 KiB tiles (measured
 // cross-over against the direct-load kernels, CUDA-graph replay, d = 1024 ... 8192).
@@ -146,6 +146,17 @@ int select_fwd(const FwdArgs& f, int64_t T, int32_t d, int dtype, cudaStream_t s
         (g_variant >= 4 || (g_variant == 0 && enough_work_for_tiles(T, d)))) {
         return umma_fwd(logd, dtype, f, c);
     }
+    if (dtype == WHT_F32) {
+        // fp32 rows: streamed tensor-core passes beat the register butterflies from d = 1024 on once there are
+        // rows to pipeline (measured: d = 2048 0.73 -> 0.98 of the copy rate); below that the butterflies are at
+        // 0.94 ... 0.98 already.  A forced variant >= 2 takes the mma.sync kernels at every size.
+        const bool enough = !decode && enough_rows_to_stream(T, c.sms);
+        if (mma_supported(logd, dtype) && (g_variant >= 2 || (g_variant == 0 && logd >= 10 && enough))) {
+            const bool streamed = g_variant != 2;
+            return mma_fwd(logd, dtype, /*few_rows=*/decode, streamed, f, c);
+        }
+        return bfly_fwd(logd, dtype, f, c);
+    }
     if (g_variant != 1 && mma_supported(logd, dtype)) {
         // rows of 256 or 512 elements: the direct-load kernels (which request a warp's next row ahead) beat
         // the streamed ones at every size (measured)
@@ -170,6 +181,17 @@ int select_bwd(const BwdArgs& g, int64_t T, int32_t d, int dtype, cudaStream_t s
         // half-size products: measured 2-4 % faster in long runs at d = 1024 and 2048, 1 % slower at 4096
         const bool half_size = g_variant == 5 || (g_variant == 0 && logd <= 11);
         return umma_bwd(logd, dtype, g_bwd_operand_mode == 1, half_size, g, c);
+    }
+    if (dtype == WHT_F32) {
+        // fp32 rows: the streamed kernels win at every width they have the shared memory for (measured: d = 256
+        // 0.82 -> 0.93 of the copy rate, d = 2048 0.47 -> 0.91, d = 4096 0.37 -> 0.67).  At d = 8192 an x and a
+        // dy row take 64 KiB of the ring, one row group is all that fits, and neither it nor the direct-load
+        // kernel (within the 16 MiB of partial sums) beats the butterflies' 0.37.
+        if (mma_supported(logd, dtype) &&
+            (g_variant >= 2 || (g_variant == 0 && logd <= 12 && enough_rows_to_stream(T, c.sms)))) {
+            return mma_bwd(logd, dtype, /*streamed=*/g_variant != 2, g, c);
+        }
+        return bfly_bwd(logd, dtype, g, c);
     }
     if (g_variant != 1 && mma_supported(logd, dtype)) {
         // d = 256: direct loads (measured); wider rows are streamed once there are enough of them

@@ -372,6 +372,22 @@ def test_streamed_kernels_on_many_rows(B):
     B.wht_affine_device_status()
 
 
+def test_fp32_rows_on_the_tensor_core_passes(B):
+    # fp32 rows enter every H_16 pass as three bf16 terms; the fp32 bound (1e-5 of the row norm) must hold as
+    # for the register butterflies.  Direct loads (2), streamed (3: every ring wraps several times, ragged
+    # tail), and the automatic choice from the row count on at which it streams.
+    for d, T in [(256, 20011), (512, 9001), (1024, 9973), (2048, 5003), (4096, 3001), (8192, 1501)]:
+        w = wl.Workload("f32mma", T, d, wl.WHT_F32, "normal", 900 + d, True, "")
+        _run_case(B, w, 3)
+    for d, T in [(256, 1031), (1024, 2053), (2048, 1201), (8192, 301)]:
+        w = wl.Workload("f32mma", T, d, wl.WHT_F32, "normal", 950 + d, True, "")
+        _run_case(B, w, 2)
+    for d, T in [(512, 148 * 32 + 5), (1024, 148 * 32 + 1), (2048, 148 * 32 + 3)]:
+        w = wl.Workload("f32mma", T, d, wl.WHT_F32, "student_t3", 970 + d, True, "")
+        _run_case(B, w, 0)
+    B.wht_affine_device_status()
+
+
 def test_tcgen05_kernels_on_many_rows(B):
     # several tiles per CTA on every SM (the ring and both accumulator sets wrap), ragged last tile
     for d, dtype, T in [(1024, wl.WHT_BF16, 148 * 16 * 5 + 7), (2048, wl.WHT_BF16_PF32, 148 * 8 * 4 + 3),
@@ -422,7 +438,8 @@ def test_back_to_back_calls_see_each_others_results(B):
 @pytest.mark.parametrize("variant", VARIANTS)
 @pytest.mark.parametrize("d,dtype,T", [(256, wl.WHT_F32, 64), (64, wl.WHT_BF16, 1031), (1024, wl.WHT_BF16, 257),
                                        (2048, wl.WHT_BF16_PF32, 300), (4096, wl.WHT_BF16, 37),
-                                       (8192, wl.WHT_BF16_PF32, 21), (16384, wl.WHT_F32, 5)])
+                                       (8192, wl.WHT_BF16_PF32, 21), (16384, wl.WHT_F32, 5),
+                                       (2048, wl.WHT_F32, 300), (1024, wl.WHT_F32, 148 * 32 + 9)])
 def test_fwd_residual(B, d, dtype, T, variant):
     B.wht_affine_set_variant(variant)
     w = wl.Workload("res", T, d, dtype, "normal", 600 + d, True, "")
