@@ -423,10 +423,10 @@ def section_tensor_parallel_local(B, hbm_peak):
 
 
 def section_other_shapes(B, hbm_peak):
-    """Shapes outside the five configs, 256 MiB per row tensor: fp32 storage and the block-diagonal form
-    (butterfly kernels)."""
+    """Shapes outside the five configs, 256 MiB per row tensor: fp32 storage (butterfly kernels at d <= 512 in
+    the forward, streamed mma.sync kernels otherwise) and the block-diagonal form."""
     out = {}
-    for d in (256, 512, 2048):
+    for d in (256, 512, 1024, 2048, 4096):
         T = (256 << 20) // (4 * d)
         x = torch.randn(T, d, device="cuda")
         a = torch.rand(d, device="cuda") + 0.5

@@ -133,7 +133,7 @@ int dispatch_mma_bwd(int logd, bool streamed, const BwdArgs& g, const Ctx& c) {
     } else {
         switch (logd) {
             case 8: return launch_mma_bwd_pipe<8, 0, 8, 4, 3, TP>(g, c);
-            case 9: return launch_mma_bwd_pipe<9, 1, 8, 4, 2, TP>(g, c);
+            case 9: return launch_mma_bwd_pipe<9, 1, 16, 3, 1, TP>(g, c);
             case 10: return launch_mma_bwd_pipe<10, 2, 8, 3, 2, TP>(g, c);
             case 11: return launch_mma_bwd_pipe<11, 2, 4, 2, 2, TP>(g, c);
             case 12: return launch_mma_bwd_pipe<12, 2, 2, 2, 1, TP>(g, c);
