@@ -547,6 +547,8 @@ def run_ours(args, rank: int, world: int, local_rank: int):
     w = wl.CONFIGS[args.workload]
     if args.rows:
         w = w.with_rows(args.rows)  # a smaller case of the same kernels (profiler captures)
+    if args.fp32_rows:  # the same shape stored as fp32 (profiler captures of the fp32 kernels)
+        w = wl.Workload(w.name, w.T, w.d, wl.WHT_F32, w.dist, w.seed, w.has_bwd, w.note)
     # every rank draws its own rows (weak scaling): the seed is offset by the rank
     wr = wl.Workload(w.name, w.T, w.d, w.dtype, w.dist, w.seed + 1000 * rank, w.has_bwd, w.note)
     base_rows = min(w.T, 8192) if w.dist != "normal" else w.T
@@ -702,7 +704,8 @@ def run_ours(args, rank: int, world: int, local_rank: int):
     dom_sum = bwd_sum if w.has_bwd else fwd_sum
     dom_fig = bwd_fig if w.has_bwd else fwd_fig
     dom = "wht_affine_bwd (main kernel + the small second pass)" if w.has_bwd else "wht_affine_fwd"
-    traffic, traffic_source = ncu_traffic(w.name, w.T) if w.has_bwd else (None, "no capture recorded for this call")
+    traffic, traffic_source = (ncu_traffic(w.name, w.T) if w.has_bwd and not args.fp32_rows
+                               else (None, "no capture recorded for this call"))
     roofline = {"bound": "hbm", "kernel": dom, "achieved": dom_sum["GBps"], "peak": hbm_peak, "unit": "GB/s",
                 "frac": dom_sum["frac_of_measured_peak"], "frac_burst": dom_sum["burst"]["frac_of_measured_peak"],
                 "peak_source": peak_src, "traffic": traffic, "traffic_source": traffic_source,
@@ -861,6 +864,9 @@ def main():
     ap.add_argument("--rows", type=int, default=0,
                     help="override the workload's row count (small cases for profiler captures; "
                          "not the benchmark configuration)")
+    ap.add_argument("--fp32-rows", action="store_true",
+                    help="store the workload's rows and parameters as fp32 (profiler captures; not the "
+                         "benchmark configuration)")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
