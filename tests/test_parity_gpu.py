@@ -388,6 +388,77 @@ def test_fp32_rows_on_the_tensor_core_passes(B):
     B.wht_affine_device_status()
 
 
+@pytest.mark.parametrize("d,dtype,variants", [(1024, wl.WHT_BF16_PF32, [0, 1, 2, 3]), (1024, wl.WHT_F32, [0, 1, 2]),
+                                              (8192, wl.WHT_BF16_PF32, [0, 3]), (256, wl.WHT_BF16, [0, 1])])
+def test_tensors_past_two_to_the_31_elements(B, d, dtype, variants):
+    # e.g. 2^21 + 5 rows of 1024: 2^31 + 5120 elements per tensor, byte offsets past 4 GiB (bf16) and 8 GiB (fp32), so
+    # any 32-bit element or byte index in a kernel or on the way to it shows.  Only three blocks of rows are
+    # non-zero (the first rows, rows around the middle, the last 133): they are checked against the oracle row by
+    # row; a zero row must come out as b (forward) and as zero (backward), exactly; and da, db are sums over rows
+    # to which the zero rows add nothing, so the oracle on the three blocks alone gives them.
+    T = (1 << 31) // d + 5
+    blocks = [(0, 128), (T // 2 - 3, 128), (T - 133, 133)]
+    zero_rows = [128, 5000, T // 3, T // 2 + 200, T - 134]
+    proto = wl.Workload("big", 1, d, dtype, "normal", 1234, True, "")
+    a, b = wl.gen_params(proto)
+    tdt = proto.io_torch_dtype
+    x_d = torch.zeros(T, d, dtype=tdt, device="cuda")
+    dy_d = torch.zeros(T, d, dtype=tdt, device="cuda")
+    xs, dys = [], []
+    for i, (r0, n) in enumerate(blocks):
+        wb = wl.Workload("big", n, d, dtype, "normal", 1300 + i, True, "")
+        xs.append(wl.gen_full(wb, "x"))
+        dys.append(wl.gen_full(wb, "dy"))
+        x_d[r0:r0 + n].copy_(xs[-1])
+        dy_d[r0:r0 + n].copy_(dys[-1])
+    x_all, dy_all = torch.cat(xs), torch.cat(dys)
+    a64, b64 = to_f64(a), to_f64(b)
+    y_ref = oracle.wht_affine_fwd(to_f64(x_all), a64, b64)
+    dx_ref, da_ref, db_ref = oracle.wht_affine_bwd(to_f64(dy_all), to_f64(x_all), a64)
+    ad, bd = a.cuda(), b.cuda()
+    b_stored = bd.to(tdt)
+    y_d = torch.empty_like(x_d)
+    for variant in variants:
+        B.wht_affine_set_variant(variant)
+        y_d.fill_(7.0)
+        B.forward(x_d, ad, bd, out=y_d)
+        got = torch.cat([y_d[r0:r0 + n] for r0, n in blocks]).cpu()
+        what = f"2^31 elements, dtype {dtype}, v{variant}"
+        if dtype == wl.WHT_F32:
+            assert_rows_fp32(to_f64(got), y_ref, to_f64(x_all), what + " y")
+        else:
+            assert_rows_bf16(to_f64(got), y_ref, what + " y")
+        for r in zero_rows:
+            assert torch.equal(y_d[r], b_stored), f"{what}: y of zero row {r}"
+        # fused residual add, in place over the residual stream (here: dy)
+        y_d.copy_(dy_d)
+        B.forward(x_d, ad, bd, out=y_d, resid=y_d)
+        got = torch.cat([y_d[r0:r0 + n] for r0, n in blocks]).cpu()
+        res_ref = oracle.wht_affine_fwd_residual(to_f64(x_all), a64, b64, to_f64(dy_all))
+        if dtype == wl.WHT_F32:
+            err = np.max(np.abs(to_f64(got) - res_ref), axis=1)
+            assert np.all(err <= 1e-5 * (np.linalg.norm(to_f64(x_all), axis=1) + np.max(np.abs(to_f64(dy_all)), axis=1)))
+        else:
+            assert_rows_bf16(to_f64(got), res_ref, what + " y + resid")
+        for r in zero_rows:
+            assert torch.equal(y_d[r], b_stored), f"{what}: residual form, zero row {r}"
+        y_d.fill_(7.0)
+        da = torch.empty(d, dtype=torch.float32, device="cuda")
+        db = torch.empty(d, dtype=torch.float32, device="cuda")
+        B.wht_affine_bwd(dy_d, x_d, ad, y_d, da, db, T, d, dtype)
+        got = torch.cat([y_d[r0:r0 + n] for r0, n in blocks]).cpu()
+        if dtype == wl.WHT_F32:
+            assert_rows_fp32(to_f64(got), dx_ref, a64[None, :] * to_f64(dy_all), what + " dx")
+        else:
+            assert_rows_bf16(to_f64(got), dx_ref, what + " dx")
+        for r in zero_rows:
+            assert torch.count_nonzero(y_d[r]).item() == 0, f"{what}: dx of zero row {r}"
+        assert_grad_vec(to_f64(da.cpu()), da_ref, what + " da")
+        assert_grad_vec(to_f64(db.cpu()), db_ref, what + " db")
+    B.wht_affine_set_variant(0)
+    B.wht_affine_device_status()
+
+
 def test_tcgen05_kernels_on_many_rows(B):
     # several tiles per CTA on every SM (the ring and both accumulator sets wrap), ragged last tile
     for d, dtype, T in [(1024, wl.WHT_BF16, 148 * 16 * 5 + 7), (2048, wl.WHT_BF16_PF32, 148 * 8 * 4 + 3),
@@ -678,8 +749,9 @@ def test_bwd_bf16_operand_mode(B, name, rows, variant):
 
 # ------------------------------------------------------------------ grouped (block-diagonal) form
 
-@pytest.mark.parametrize("variant", [0, 1, 3])
+@pytest.mark.parametrize("variant", [0, 1, 2, 3])
 @pytest.mark.parametrize("d,block,dtype,T", [(768, 256, wl.WHT_F32, 70), (768, 256, wl.WHT_BF16, 300),
+                                             (1280, 256, wl.WHT_BF16_PF32, 1237), (3072, 512, wl.WHT_F32, 611),
                                              (1536, 512, wl.WHT_BF16_PF32, 129), (3072, 1024, wl.WHT_BF16, 33),
                                              (96, 32, wl.WHT_F32, 1000), (1024, 1024, wl.WHT_BF16, 40),
                                              (768, 256, wl.WHT_BF16_PF32, 148 * 32 + 77), (1536, 512, wl.WHT_BF16, 148 * 32 + 5),
