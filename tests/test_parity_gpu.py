@@ -795,6 +795,56 @@ def test_grouped_form(B, d, block, dtype, T, variant):
     B.wht_affine_set_variant(0)
 
 
+def test_grouped_form_past_two_to_the_31_elements(B):
+    # d = 768 = 3 blocks of 256, 2^31 / 768 + 7 rows: as in the plain test of that name, three blocks of rows are
+    # non-zero, the rest must come out as b and as zero, and da, db follow from the non-zero rows alone
+    d, block, dtype = 768, 256, wl.WHT_BF16_PF32
+    G = d // block
+    T = (1 << 31) // d + 7
+    rows = [(0, 96), (T // 2 + 1, 96), (T - 77, 77)]
+    zero_rows = [96, T // 3, T - 78]
+    gen = lambda n, seed, which: torch.cat(
+        [wl.gen_full(wl.Workload("grpbig", n, block, dtype, "normal", seed + g, True, ""), which) for g in range(G)],
+        dim=1).contiguous()
+    ab = [wl.gen_params(wl.Workload("grpbig", 1, block, dtype, "normal", 1500 + g, True, "")) for g in range(G)]
+    a = torch.cat([p[0] for p in ab]).contiguous()
+    b = torch.cat([p[1] for p in ab]).contiguous()
+    x_d = torch.zeros(T, d, dtype=torch.bfloat16, device="cuda")
+    dy_d = torch.zeros_like(x_d)
+    xs, dys = [], []
+    for i, (r0, n) in enumerate(rows):
+        xs.append(gen(n, 1600 + 10 * i, "x"))
+        dys.append(gen(n, 1600 + 10 * i, "dy"))
+        x_d[r0:r0 + n].copy_(xs[-1])
+        dy_d[r0:r0 + n].copy_(dys[-1])
+    x_all, dy_all = torch.cat(xs), torch.cat(dys)
+    ref_y = oracle.wht_affine_fwd_grouped(to_f64(x_all), to_f64(a), to_f64(b), block)
+    ref_dx, ref_da, ref_db = oracle.wht_affine_bwd_grouped(to_f64(dy_all), to_f64(x_all), to_f64(a), block)
+    ad, bd = a.cuda(), b.cuda()
+    out = torch.empty_like(x_d)
+    da = torch.empty(d, dtype=torch.float32, device="cuda")
+    db = torch.empty_like(da)
+    for variant in (0, 1):
+        B.wht_affine_set_variant(variant)
+        out.fill_(7.0)
+        B.wht_affine_fwd_grouped(x_d, ad, bd, out, T, d, block, dtype)
+        got = torch.cat([out[r0:r0 + n] for r0, n in rows]).cpu()
+        assert_rows_bf16(to_f64(got), ref_y, f"grouped y past 2^31, v{variant}")
+        for r in zero_rows:
+            assert torch.equal(out[r], bd.bfloat16())
+        ws = torch.empty(max(B.wht_affine_bwd_grouped_workspace_bytes(T, d, block, dtype), 16), dtype=torch.uint8,
+                         device="cuda")
+        out.fill_(7.0)
+        B.wht_affine_bwd_grouped(dy_d, x_d, ad, out, da, db, T, d, block, dtype, ws)
+        got = torch.cat([out[r0:r0 + n] for r0, n in rows]).cpu()
+        assert_rows_bf16(to_f64(got), ref_dx, f"grouped dx past 2^31, v{variant}")
+        for r in zero_rows:
+            assert torch.count_nonzero(out[r]).item() == 0
+        assert_grad_vec(to_f64(da.cpu()), ref_da, "grouped da past 2^31")
+        assert_grad_vec(to_f64(db.cpu()), ref_db, "grouped db past 2^31")
+    B.wht_affine_set_variant(0)
+
+
 def test_autograd_wrapper(B):
     from paper_2603_08343_b200.autograd import wht_affine
     B.wht_affine_set_variant(0)
