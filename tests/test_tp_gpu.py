@@ -139,6 +139,46 @@ def test_blocks_given_as_addresses_and_repeat_calls_are_bit_identical(B):
         assert torch.equal(u, v)
 
 
+@pytest.mark.parametrize("variant", [0, 1])
+def test_blocks_past_two_to_the_31_elements(B, variant):
+    # g = 2 ranks, blocks of 2^21 + 5 rows x 1024 columns: 2^31 + 5120 elements per block.  All rows are zero
+    # but the first and the last 100; those are checked against the full-width oracle, a zero row must come out
+    # as b and as zero, and da, db follow from the non-zero rows alone.
+    B.wht_affine_set_variant(variant)
+    g, w, dtype = 2, 1024, wl.WHT_BF16_PF32
+    d, T, n = g * w, (1 << 21) + 5, 100
+    wk = wl.Workload("tpbig", 2 * n, d, dtype, "normal", 990, True, "")
+    x, dy = wl.gen_full(wk, "x"), wl.gen_full(wk, "dy")
+    a, b = wl.gen_params(wk)
+    xs = [torch.zeros(T, w, dtype=torch.bfloat16, device="cuda") for _ in range(g)]
+    dys = [torch.zeros(T, w, dtype=torch.bfloat16, device="cuda") for _ in range(g)]
+    for s in range(g):
+        for blocks, src in ((xs, x), (dys, dy)):
+            blocks[s][:n].copy_(src[:n, s * w:(s + 1) * w])
+            blocks[s][T - n:].copy_(src[n:, s * w:(s + 1) * w])
+    as_ = [a[s * w:(s + 1) * w].contiguous().cuda() for s in range(g)]
+    bs = [b[s * w:(s + 1) * w].contiguous().cuda() for s in range(g)]
+    ref_y = oracle.wht_affine_fwd(to_f64(x), to_f64(a), to_f64(b))
+    ref_dx, ref_da, ref_db = oracle.wht_affine_bwd(to_f64(dy), to_f64(x), to_f64(a))
+    pick = lambda t: torch.cat([t[:n], t[T - n:]]).cpu()
+    ys, dxs, das, dbs = [], [], [], []
+    for r in range(g):
+        rank = tp.TpWht(g, r)
+        y = rank.forward(xs, as_[r], bs[r], T, w)
+        dx, da, db = rank.backward(dys, xs, as_, T, w)
+        torch.cuda.synchronize()
+        for row in (n, T // 2, T - n - 1):
+            assert torch.equal(y[row], bs[r].bfloat16()) and torch.count_nonzero(dx[row]).item() == 0
+        ys.append(pick(y)); dxs.append(pick(dx)); das.append(da.cpu()); dbs.append(db.cpu())
+        del y, dx
+    assert_rows_bf16(to_f64(torch.cat(ys, dim=1)), ref_y, "tp y past 2^31")
+    assert_rows_bf16(to_f64(torch.cat(dxs, dim=1)), ref_dx, "tp dx past 2^31")
+    assert_grad_vec(to_f64(torch.cat(das)), ref_da, "tp da past 2^31")
+    assert_grad_vec(to_f64(torch.cat(dbs)), ref_db, "tp db past 2^31")
+    B.wht_affine_set_variant(0)
+    B.wht_affine_device_status()
+
+
 def test_no_rows(B):
     g, w = 2, 256
     rank = tp.TpWht(g, 1)
