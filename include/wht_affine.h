@@ -332,6 +332,17 @@ int wht_affine_selftest_wait_expiry(uint32_t limit_us, unsigned int* out3, void*
 int wht_affine_debug_build(void);
 int wht_affine_debug_selftest_guard(int damage);
 
+/*
+ * Failure injection on the host, for test suites (the paper has no counterpart): the next `n`
+ * allocations the library would make for itself (the scratch of wht_affine_bwd; the guarded buffers
+ * of a debug build) fail as an out-of-memory answer of the allocator would, without the allocator
+ * being called.  The failing call returns WHT_ERR_WORKSPACE before anything is
+ * launched and leaves the caller's tensors and the library's state as they were; the call after the
+ * n-th failure allocates normally.  n = 0 clears the setting; n < 0 -> WHT_ERR_BAD_VARIANT.
+ * Returns the number of injected failures still pending before the call.  Process-wide.
+ */
+int wht_affine_test_fail_allocations(int n);
+
 /* cudaError_t of the most recent failing CUDA call on this thread (0 if none). */
 int wht_affine_last_cuda_error(void);
 

@@ -24,7 +24,8 @@ EXPORTS = (
     "wht_affine_bwd_workspace_bytes", "wht_affine_set_variant", "wht_affine_get_variant",
     "wht_affine_set_bwd_operand_mode", "wht_affine_get_bwd_operand_mode",
     "wht_copy_rows", "wht_affine_device_status", "wht_affine_selftest_wait_expiry",
-    "wht_affine_debug_build", "wht_affine_debug_selftest_guard", "wht_affine_last_cuda_error", "wht_affine_status_string",
+    "wht_affine_debug_build", "wht_affine_debug_selftest_guard", "wht_affine_test_fail_allocations",
+    "wht_affine_last_cuda_error", "wht_affine_status_string",
     "wht_affine_shutdown",
 )
 
@@ -77,6 +78,7 @@ def _load(path: str | None = None) -> ctypes.CDLL:
     lib.wht_affine_shutdown.argtypes = []
     lib.wht_affine_debug_build.argtypes = []
     lib.wht_affine_debug_selftest_guard.argtypes = [ci]
+    lib.wht_affine_test_fail_allocations.argtypes = [ci]
     for name in EXPORTS:
         fn = getattr(lib, name)
         if fn.restype is ctypes.c_int or fn.restype is None:
@@ -291,6 +293,15 @@ def wht_affine_selftest_wait_expiry(limit_us: int, out3, stream=None) -> None:
     _require_cuda(out3)
     _check(_lib.wht_affine_selftest_wait_expiry(limit_us, _ptr(out3), _stream(stream)),
            "wht_affine_selftest_wait_expiry")
+
+
+def wht_affine_test_fail_allocations(n: int) -> int:
+    """Test hook: the library's next n allocations of its own fail as out of memory; returns how many
+    injected failures were still pending."""
+    pending = _lib.wht_affine_test_fail_allocations(n)
+    if pending < 0:
+        raise WhtError(pending, "wht_affine_test_fail_allocations")
+    return pending
 
 
 def wht_affine_shutdown() -> None:

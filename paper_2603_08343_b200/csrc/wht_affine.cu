@@ -1,6 +1,7 @@
 // C ABI of the library (see include/wht_affine.h): argument checks, kernel selection and the
 // library-owned backward scratch buffer.  The kernels are instantiated and launched by the
 // family_*.cu files beside this one (one per kernel family, so that they compile in parallel).
+#include <atomic>
 #include <initializer_list>
 #include <mutex>
 
@@ -59,6 +60,18 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 
 size_t elem_bytes(int dtype) { return dtype == WHT_F32 ? 4 : 2; }
 
+// Every allocation the library makes for itself goes through here, so that tests can make it fail.
+std::atomic<int> g_fail_allocations{0};
+cudaError_t library_malloc(void** p, size_t bytes) {
+    int pending = g_fail_allocations.load();
+    while (pending > 0 && !g_fail_allocations.compare_exchange_weak(pending, pending - 1)) {}
+    if (pending > 0) {
+        *p = nullptr;
+        return cudaErrorMemoryAllocation;  // injected: the allocator is not called
+    }
+    return cudaMalloc(p, bytes);
+}
+
 #ifdef WHT_DEBUG
 // Debug build (-DWHT_DEBUG): every output and scratch buffer of a compute call is replaced by a device
 // buffer of the library's own with a guard region on either side, filled with a canary byte.  After the
@@ -79,7 +92,13 @@ class GuardedBuffer {
     int init(size_t bytes, cudaStream_t s) {
         bytes_ = bytes;
         padded_ = (bytes + 15) / 16 * 16;
-        if (cudaMalloc(&base_, padded_ + 2 * kGuardBytes) != cudaSuccess) return cuda_fail(cudaGetLastError());
+        const cudaError_t err = library_malloc(&base_, padded_ + 2 * kGuardBytes);
+        if (err != cudaSuccess) {
+            cudaGetLastError();
+            g_last_cuda_error = static_cast<int>(err);
+            base_ = nullptr;
+            return WHT_ERR_WORKSPACE;
+        }
         WHT_CUDA_TRY(cudaMemsetAsync(base_, kCanary, kGuardBytes, s));
         WHT_CUDA_TRY(cudaMemsetAsync(static_cast<unsigned char*>(base_) + kGuardBytes + padded_, kCanary, kGuardBytes, s));
         return WHT_OK;
@@ -437,8 +456,10 @@ int wht_affine_bwd(const void* dy, const void* x, const void* a, void* dx, float
             }
             void* p = nullptr;
             const size_t bytes = need < (1u << 20) ? (1u << 20) : need;
-            if (cudaMalloc(&p, bytes) != cudaSuccess) {
-                g_last_cuda_error = static_cast<int>(cudaGetLastError());
+            const cudaError_t err = library_malloc(&p, bytes);
+            if (err != cudaSuccess) {
+                cudaGetLastError();  // clear the runtime's sticky copy of an allocator failure
+                g_last_cuda_error = static_cast<int>(err);
                 return WHT_ERR_WORKSPACE;
             }
             st.scratch = p;
@@ -663,6 +684,11 @@ int wht_affine_debug_selftest_guard(int damage) {
     (void)damage;
     return WHT_ERR_BAD_VARIANT;
 #endif
+}
+
+int wht_affine_test_fail_allocations(int n) {
+    if (n < 0) return WHT_ERR_BAD_VARIANT;
+    return g_fail_allocations.exchange(n);
 }
 
 int wht_affine_last_cuda_error(void) { return g_last_cuda_error; }

@@ -157,3 +157,25 @@ def test_grouped_and_column_sharded_calls_through_the_guarded_build(libs):
                                      dtype, _p(ws), ws.numel(), s) == 0
         torch.cuda.synchronize()
         assert torch.equal(y, y_ref) and all(torch.equal(u, v) for u, v in zip(got, ref)), f"tp g={g_} w={w_}"
+
+
+def test_a_failed_guard_buffer_allocation_is_an_error(libs):
+    # the guarded build allocates on every call: an injected out-of-memory answer must surface as
+    # WHT_ERR_WORKSPACE, the output must stay as it was, and the next call must work
+    B, dbg = libs
+    w = wl.Workload("guard", 130, 1024, wl.WHT_BF16, "normal", 3300, True, "")
+    x = wl.gen_full(w, "x")
+    a, b = wl.gen_params(w)
+    xd, ad, bd = x.cuda(), a.cuda(), b.cuda()
+    s = ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+    y = torch.full_like(xd, 7.0)
+    assert dbg.wht_affine_test_fail_allocations(1) == 0
+    try:
+        assert dbg.wht_affine_fwd(_p(xd), _p(ad), _p(bd), _p(y), w.T, w.d, w.dtype, s) == -6
+        torch.cuda.synchronize()
+        assert torch.all(y == 7.0)
+    finally:
+        assert dbg.wht_affine_test_fail_allocations(0) == 0
+    assert dbg.wht_affine_fwd(_p(xd), _p(ad), _p(bd), _p(y), w.T, w.d, w.dtype, s) == 0
+    torch.cuda.synchronize()
+    assert_rows_bf16(to_f64(y.cpu()), oracle.wht_affine_fwd(to_f64(x), to_f64(a), to_f64(b)), "after the failed allocation")

@@ -63,3 +63,45 @@ def test_selftest_arguments_are_checked(B):
     torch.cuda.synchronize()
     assert out.cpu().tolist() == [0, 0, 0]
     B.wht_affine_device_status()
+
+
+def test_a_failed_scratch_allocation_is_an_error_and_nothing_runs(B):
+    # host-side injection: the library's next allocation answers "out of memory" without the allocator being
+    # called.  The backward that needs the scratch must return WHT_ERR_WORKSPACE before any launch, leave its
+    # outputs alone, and the next call must allocate and give the oracle's result.
+    from helpers import assert_grad_vec
+    w = wl.Workload("allocfail", 301, 2048, wl.WHT_BF16_PF32, "normal", 71, True, "")
+    x, dy = wl.gen_full(w, "x"), wl.gen_full(w, "dy")
+    a, _ = wl.gen_params(w)
+    xd, dyd, ad = x.cuda(), dy.cuda(), a.cuda()
+    dx = torch.full_like(xd, 7.0)
+    da = torch.full((w.d,), 7.0, device="cuda")
+    db = torch.full((w.d,), 7.0, device="cuda")
+    torch.cuda.synchronize()
+    B.wht_affine_shutdown()                      # the library owns no scratch now: the next backward allocates
+    assert B.wht_affine_test_fail_allocations(1) == 0
+    try:
+        with pytest.raises(B.WhtError) as err:
+            B.wht_affine_bwd(dyd, xd, ad, dx, da, db, w.T, w.d, w.dtype)
+        assert err.value.status == -6            # WHT_ERR_WORKSPACE
+        torch.cuda.synchronize()
+        assert torch.all(dx == 7.0) and torch.all(da == 7.0) and torch.all(db == 7.0)
+        assert B.wht_affine_test_fail_allocations(0) == 0   # the one injected failure was used up
+        # the calls that bring their own scratch, or need none, never allocate
+        B.wht_affine_test_fail_allocations(5)
+        if not B.lib().wht_affine_debug_build():
+            y = B.forward(xd, ad, ad)
+            B.wht_affine_bwd_noalloc(dyd, xd, ad, dx, da, db, w.T, w.d, w.dtype)
+            torch.cuda.synchronize()
+            assert B.wht_affine_test_fail_allocations(0) == 5
+    finally:
+        B.wht_affine_test_fail_allocations(0)
+    B.wht_affine_bwd(dyd, xd, ad, dx, da, db, w.T, w.d, w.dtype)
+    torch.cuda.synchronize()
+    ref_dx, ref_da, ref_db = oracle.wht_affine_bwd(to_f64(dy), to_f64(x), to_f64(a))
+    assert_rows_bf16(to_f64(dx.cpu()), ref_dx, "dx after the failed allocation")
+    assert_grad_vec(to_f64(da.cpu()), ref_da, "da after the failed allocation")
+    assert_grad_vec(to_f64(db.cpu()), ref_db, "db after the failed allocation")
+    with pytest.raises(B.WhtError):
+        B.wht_affine_test_fail_allocations(-1)
+    B.wht_affine_device_status()
