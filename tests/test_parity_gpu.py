@@ -895,6 +895,64 @@ def test_a_non_finite_row_stays_in_its_row(B, d, T, variant):
     B.wht_affine_set_variant(0)
 
 
+@pytest.mark.parametrize("d,dtype,T,decode", [(256, wl.WHT_F32, 64, False), (4096, wl.WHT_BF16, 8, True),
+                                              (1024, wl.WHT_BF16, 257, False), (2048, wl.WHT_BF16_PF32, 148 * 8 + 3, False),
+                                              (1024, wl.WHT_F32, 148 * 32 + 1, False)])
+def test_calls_captured_in_a_cuda_graph(B, d, dtype, T, decode):
+    # every compute call is asynchronous on its stream and, once its first call has sized the library's caches,
+    # free of allocation and synchronisation: a graph of forward, fused residual forward and the three backward
+    # entry points is captured once and replayed on NEW data in the same tensors; the replay must give the
+    # oracle's values for the new data (Eq. 1 and its chain rule)
+    B.wht_affine_set_variant(0)
+    w0 = wl.Workload("graph", T, d, dtype, "normal", 4100 + d, True, "")
+    w1 = wl.Workload("graph", T, d, dtype, "normal", 4200 + d, True, "")
+    a, b = wl.gen_params(w0)
+    ad, bd = a.cuda(), b.cuda()
+    x, dy = wl.gen_full(w0, "x").cuda(), wl.gen_full(w0, "dy").cuda()
+    y, yr = torch.empty_like(x), torch.empty_like(x)
+    dxs = [torch.empty_like(x) for _ in range(3)]
+    das = [torch.empty(d, dtype=torch.float32, device="cuda") for _ in range(3)]
+    dbs = [torch.empty(d, dtype=torch.float32, device="cuda") for _ in range(3)]
+    ws = torch.empty(max(B.wht_affine_bwd_workspace_bytes(T, d, dtype), 16), dtype=torch.uint8, device="cuda")
+
+    def calls():
+        (B.wht_affine_fwd_decode if decode else B.wht_affine_fwd)(x, ad, bd, y, T, d, dtype)
+        B.wht_affine_fwd_residual(x, ad, bd, dy, yr, T, d, dtype)
+        B.wht_affine_bwd(dy, x, ad, dxs[0], das[0], dbs[0], T, d, dtype)
+        B.wht_affine_bwd_ws(dy, x, ad, dxs[1], das[1], dbs[1], T, d, dtype, ws)
+        B.wht_affine_bwd_noalloc(dy, x, ad, dxs[2], das[2], dbs[2], T, d, dtype)
+
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        calls()                                 # sizes the scratch, looks up the built-in array, fills the caches
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        calls()
+    x1, dy1 = wl.gen_full(w1, "x"), wl.gen_full(w1, "dy")
+    x.copy_(x1)
+    dy.copy_(dy1)
+    for t in [y, yr] + dxs + das + dbs:
+        t.fill_(7.0)
+    graph.replay()
+    graph.replay()
+    torch.cuda.synchronize()
+    what = f"graph replay d={d} dtype={dtype} T={T}"
+    _check_fwd(w1, y.cpu(), x1, a, b, what + " fwd")
+    ref_r = oracle.wht_affine_fwd_residual(to_f64(x1), to_f64(a), to_f64(b), to_f64(dy1))
+    if dtype == wl.WHT_F32:
+        err = np.max(np.abs(to_f64(yr.cpu()) - ref_r), axis=1)
+        assert np.all(err <= 1e-5 * (np.linalg.norm(to_f64(x1), axis=1) + np.max(np.abs(to_f64(dy1)), axis=1)))
+    else:
+        assert_rows_bf16(to_f64(yr.cpu()), ref_r, what + " residual")
+    for k in range(3):
+        _check_bwd(w1, dxs[k].cpu(), das[k].cpu(), dbs[k].cpu(), dy1, x1, a, what + f" bwd entry {k}")
+    assert all(torch.equal(dxs[0], t) for t in dxs[1:]) and all(torch.equal(das[0], t) for t in das[1:])
+    B.wht_affine_device_status()
+
+
 def test_calls_on_two_streams_at_once(B):
     """A forward and a backward (caller-owned scratch) issued on two streams with no ordering between them
     give the bits of the serial calls: the kernels share SMs, tensor memory and the device-wide status word
