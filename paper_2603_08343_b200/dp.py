@@ -44,3 +44,47 @@ class GradBucket:
         if dist.is_available() and dist.is_initialized() and dist.get_world_size(group) > 1:
             dist.all_reduce(self.flat, op=dist.ReduceOp.SUM, group=group)
         return self.da, self.db
+
+
+class GradBucketRing:
+    """`n` GradBuckets used in turn, each step's all-reduce left in flight while the next step computes.
+
+    The sum over ranks is needed by whoever consumes the gradients (an optimizer), not by the next
+    forward pass, so a step need not wait for its own all-reduce: it is started asynchronously and
+    waited for only when its bucket comes round again (or at `drain`).  On GPU ranks the wait is a
+    stream dependency, not a host block.
+
+        bucket = ring.acquire()                 # its previous all-reduce, if any, is waited for
+        wht_affine_bwd(..., bucket.da, bucket.db, ...)
+        ring.all_reduce_async(bucket)           # returns at once
+        ...
+        ring.drain()                            # before reading the last steps' sums
+    """
+
+    def __init__(self, d: int, device="cpu", n: int = 2):
+        if n < 1:
+            raise ValueError("at least one bucket")
+        self.buckets = [GradBucket(d, device) for _ in range(n)]
+        self._pending = [None] * n
+        self._next = 0
+
+    def acquire(self) -> GradBucket:
+        i = self._next
+        self._next = (i + 1) % len(self.buckets)
+        self._wait(i)
+        return self.buckets[i]
+
+    def all_reduce_async(self, bucket: GradBucket, group=None) -> None:
+        i = next(k for k, b in enumerate(self.buckets) if b is bucket)
+        self._wait(i)
+        if dist.is_available() and dist.is_initialized() and dist.get_world_size(group) > 1:
+            self._pending[i] = dist.all_reduce(bucket.flat, op=dist.ReduceOp.SUM, group=group, async_op=True)
+
+    def drain(self) -> None:
+        for i in range(len(self.buckets)):
+            self._wait(i)
+
+    def _wait(self, i: int) -> None:
+        work, self._pending[i] = self._pending[i], None
+        if work is not None:
+            work.wait()

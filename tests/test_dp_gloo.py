@@ -70,3 +70,49 @@ def test_bucket_without_process_group_is_local():
     bucket.da.fill_(2.0)
     da, db = bucket.all_reduce()
     assert torch.all(da == 2.0) and torch.all(db == 0.0)
+
+
+def _ring_main(rank, world, port, out):
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        d, steps = 16, 5
+        ring = dp.GradBucketRing(d, n=2)
+        seen = []
+        for step in range(steps):
+            bucket = ring.acquire()          # the sum of step - 2 sits here until it is overwritten now
+            if step >= 2:
+                seen.append((step - 2, bucket.flat.clone()))
+            bucket.da.fill_(float(10 * step + rank + 1))
+            bucket.db.fill_(float(-(10 * step + rank + 1)))
+            ring.all_reduce_async(bucket)
+        ring.drain()
+        for k in (steps - 2, steps - 1):
+            seen.append((k, ring.buckets[k % 2].flat.clone()))
+        torch.save(seen, os.path.join(out, f"ring{rank}.pt"))
+    finally:
+        dist.destroy_process_group()
+
+
+def test_overlapped_bucket_ring_on_two_ranks(tmp_path):
+    # every step's all-reduce stays in flight until its bucket comes round again: each step's sum over the
+    # two ranks must be what that step wrote (1 + 2 + 20 * step), on both ranks, for all five steps
+    world = 2
+    mp.spawn(_ring_main, args=(world, _free_port(), str(tmp_path)), nprocs=world, join=True)
+    for rank in range(world):
+        seen = torch.load(os.path.join(tmp_path, f"ring{rank}.pt"), weights_only=False)
+        assert sorted(k for k, _ in seen) == [0, 1, 2, 3, 4]
+        for step, flat in seen:
+            want = float(20 * step + 3)
+            assert torch.all(flat[:16] == want) and torch.all(flat[16:] == -want), (rank, step)
+
+
+def test_bucket_ring_without_process_group_is_local():
+    ring = dp.GradBucketRing(8, n=3)
+    b0 = ring.acquire()
+    b0.da.fill_(5.0)
+    ring.all_reduce_async(b0)
+    assert ring.acquire() is ring.buckets[1] and ring.acquire() is ring.buckets[2] and ring.acquire() is b0
+    ring.drain()
+    assert torch.all(b0.da == 5.0)
