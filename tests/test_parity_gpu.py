@@ -867,13 +867,15 @@ def test_autograd_wrapper(B):
 
 
 @pytest.mark.parametrize("variant", VARIANTS)
-@pytest.mark.parametrize("d,T", [(2048, 301), (8192, 37), (256, 100)])
-def test_a_non_finite_row_stays_in_its_row(B, d, T, variant):
+@pytest.mark.parametrize("d,T,dtype", [(2048, 301, wl.WHT_BF16_PF32), (8192, 37, wl.WHT_BF16_PF32),
+                                       (256, 100, wl.WHT_BF16_PF32), (1024, 257, wl.WHT_F32),
+                                       (2048, 148 * 32 + 3, wl.WHT_F32)])
+def test_a_non_finite_row_stays_in_its_row(B, d, T, dtype, variant):
     """Rows are independent: Inf or NaN in one row of x (or dy) must leave every other row of y (dx)
     bit-identical -- tiles hold several rows side by side in shared and tensor memory -- while da, db,
     which sum over rows, follow the arithmetic (non-finite)."""
     B.wht_affine_set_variant(variant)
-    w = wl.Workload("poison", T, d, wl.WHT_BF16_PF32, "normal", 4242 + d, True, "")
+    w = wl.Workload("poison", T, d, dtype, "normal", 4242 + d, True, "")
     x, dy = wl.gen_full(w, "x").cuda(), wl.gen_full(w, "dy").cuda()
     a, b = (t.cuda() for t in wl.gen_params(w))
     y0 = B.forward(x, a, b)
