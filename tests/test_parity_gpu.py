@@ -755,7 +755,8 @@ def test_bwd_bf16_operand_mode(B, name, rows, variant):
                                              (1536, 512, wl.WHT_BF16_PF32, 129), (3072, 1024, wl.WHT_BF16, 33),
                                              (96, 32, wl.WHT_F32, 1000), (1024, 1024, wl.WHT_BF16, 40),
                                              (768, 256, wl.WHT_BF16_PF32, 148 * 32 + 77), (1536, 512, wl.WHT_BF16, 148 * 32 + 5),
-                                             (512, 256, wl.WHT_BF16, 3), (6144, 2048, wl.WHT_BF16_PF32, 21)])
+                                             (512, 256, wl.WHT_BF16, 3), (6144, 2048, wl.WHT_BF16_PF32, 21),
+                                             (768, 256, wl.WHT_F32, 148 * 32 + 9)])
 def test_grouped_form(B, d, block, dtype, T, variant):
     B.wht_affine_set_variant(variant)
     w = wl.Workload("grp", T, block, dtype, "normal", 800 + d, True, "")  # generators take a power of two:
