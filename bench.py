@@ -677,6 +677,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
     events = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(ev_steps)]
     for k in range(ev_steps):
         step(events[k])
+    ring.drain()
     torch.cuda.synchronize()
     fwd_ms = [e[0].elapsed_time(e[1]) for e in events]
     bwd_ms = [e[1].elapsed_time(e[2]) for e in events] if w.has_bwd else []
@@ -760,6 +761,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
     del xp, yp, staging
     if w.has_bwd:
         del dyp, dxp
+    ring.drain()
     if world > 1:
         dist.barrier()
     if rank != 0:
@@ -795,16 +797,18 @@ def run_ours(args, rank: int, world: int, local_rank: int):
 
     # ---- CPU baseline: the oracle as it stands, on a bounded sample of the same workload
     # (a short pilot sizes it: up to 16384 rows per pass, passes until about 12 s of CPU work)
-    pilot = {"tiny": 64, "prefill": 4096, "training": 2048, "large": 256}[w.name]
-    rate = pilot / oracle_step_seconds(w, pilot)
-    rows = min(w.T, 16384, max(pilot, int(rate * 4) // 256 * 256))
-    passes = max(1, min(16, math.ceil(12.0 * rate / rows)))
-    sec = sum(oracle_step_seconds(w, rows) for _ in range(passes))
-    out["cpu_baseline"] = {"value": rows * passes / sec, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
-                           "seconds": sec,
-                           "sample": f"{passes} passes over {rows} rows of the {w.name} workload (d={w.d}), fp64 dense "
-                                     f"product, fwd{'+bwd' if w.has_bwd else ''}; tokens/s from that sample "
-                                     "(per-row cost is constant)"}
+    # On one rank only: with several ranks the line is about scaling, and the other ranks have left.
+    if world == 1:
+        pilot = {"tiny": 64, "prefill": 4096, "training": 2048, "large": 256}[w.name]
+        rate = pilot / oracle_step_seconds(w, pilot)
+        rows = min(w.T, 16384, max(pilot, int(rate * 4) // 256 * 256))
+        passes = max(1, min(16, math.ceil(12.0 * rate / rows)))
+        sec = sum(oracle_step_seconds(w, rows) for _ in range(passes))
+        out["cpu_baseline"] = {"value": rows * passes / sec, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+                               "seconds": sec,
+                               "sample": f"{passes} passes over {rows} rows of the {w.name} workload (d={w.d}), fp64 "
+                                         f"dense product, fwd{'+bwd' if w.has_bwd else ''}; tokens/s from that sample "
+                                         "(per-row cost is constant)"}
 
     if not args.no_sections and world == 1:
         del xs, ys, dys, dxs, x, y, dy, dx
